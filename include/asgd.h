@@ -1,0 +1,160 @@
+/*
+ * libasgd -- K-Means ASGD worker loop on one NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The operations follow Keuper & Pfreundt, "Asynchronous Parallel Stochastic Gradient Descent"
+ * (arXiv 1505.04956):
+ *   - Algorithm 5 (ASGD): W workers, each owning a disjoint shard of the samples, repeat
+ *       draw mini-batch -> externally modified update -> send the new state to random peers.
+ *   - Eq. 8: assignment s_i(w) = index of the closest prototype; quantisation error E(w).
+ *   - Eq. 9: K-Means mini-batch gradient (per-centre sums and counts of the assigned samples).
+ *   - Eq. 3 / Eq. 4 / Eq. 6 / Eq. 7: N receive buffers per worker, the "buffer non-empty" indicator
+ *     lambda, the Parzen-window acceptance test delta, and the merged step.
+ *   - Section 1.2 / Section 3: single-sided communication; the sender never waits, the receiver
+ *     uses whatever has arrived.
+ *
+ * On the GPU a worker is a thread block, a receive buffer is a region of device memory, and a put
+ * is a sequence of global stores followed by a release-increment of the buffer's sequence number.
+ *
+ * General rules
+ *   - Every pointer argument says whether it is HOST or DEVICE memory.  Device pointers must
+ *     belong to the device that was current when asgd_init() ran.
+ *   - Every function returns 0 (ASGD_OK) or a negative asgd_status.  Nothing throws or aborts.
+ *   - The library allocates no device memory: the caller passes one workspace of
+ *     asgd_workspace_bytes() bytes and keeps it alive until asgd_destroy().
+ *   - All device work is enqueued on the stream given to asgd_init(); calls return after enqueue
+ *     unless stated otherwise.  A context is not thread-safe.
+ *   - There is no CPU fallback.  Without a CUDA device of compute capability 10.x asgd_init()
+ *     returns ASGD_EUNSUPPORTED.
+ */
+#ifndef ASGD_H_
+#define ASGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum asgd_status {
+  ASGD_OK = 0,
+  ASGD_EINVAL = -1,       /* NULL / out-of-range / misaligned argument                      */
+  ASGD_ENOMEM = -2,       /* workspace too small, or a host allocation failed               */
+  ASGD_ECUDA = -3,        /* a CUDA call failed; code via asgd_last_cuda_error()            */
+  ASGD_EUNSUPPORTED = -4, /* wrong device, or sizes outside what the chosen path supports   */
+  ASGD_ETIMEOUT = -5      /* a bounded device-side wait expired (reported by asgd_sync)     */
+} asgd_status;
+
+/* Distance paths (a2).  AUTO picks by k and d. */
+enum {
+  ASGD_PATH_AUTO = 0,
+  ASGD_PATH_FP32 = 1,       /* CUDA cores, fp32                                              */
+  ASGD_PATH_TC_3XTF32 = 2,  /* tcgen05, three TF32 products per fp32 product                 */
+  ASGD_PATH_TC_BF16 = 3     /* tcgen05, BF16 operands, fp32 accumulate                       */
+};
+
+/* Problem statement ASGD(X, T, eps, w0, b) of Algorithm 5 plus the communication parameters. */
+typedef struct asgd_config {
+  int64_t N;             /* rows of X                                                         */
+  int32_t d;             /* dimensions per sample                                             */
+  int32_t k;             /* centres (prototypes) per state                                    */
+  int32_t W;             /* workers; worker i owns rows [i*H, (i+1)*H), H = N / W (floor)     */
+  int32_t b;             /* mini-batch size, 1 <= b <= H.  A pass is B = H / b (floor) steps;  */
+                         /* rows beyond W*H and the last H - B*b rows of a shard are unused    */
+  float eps;             /* step size > 0                                                     */
+  int32_t comm_interval; /* c: put after step t iff c > 0 and (t+1) % c == 0; 0 = silent      */
+  int32_t fanout;        /* f: recipients per put, 0 <= f <= W-1                              */
+  int32_t slots;         /* S: receive buffers per worker, >= 1                               */
+  int32_t parzen;        /* 1 = Eq. 6 (acceptance test of Eq. 4), 0 = Eq. 3 (accept all)      */
+  int32_t dist_path;     /* ASGD_PATH_*                                                       */
+  int32_t shuffle;       /* 1 = seeded permutation of each worker's batch order, 0 = in order */
+  int32_t record_assign; /* 1 = keep the last step's assignments for asgd_get_assign()        */
+  int32_t reserved;      /* must be 0                                                         */
+  uint64_t seed;         /* batch order, recipients, buffer choice                            */
+} asgd_config;
+
+typedef struct asgd_ctx asgd_ctx; /* opaque; owned by the library, freed by asgd_destroy() */
+
+/* Bytes of device workspace asgd_init() needs for this configuration (256-byte aligned base). */
+int asgd_workspace_bytes(const asgd_config *cfg, size_t *bytes /* HOST out */);
+
+/*
+ * Initialisation step of Section 4: shards are fixed, w0 is copied into all W worker states,
+ * receive buffers are emptied, counters zeroed, batch orders drawn.
+ *   X_dev        DEVICE [N*d] fp32 row-major, 16-byte aligned.  BORROWED: never written, must stay
+ *                alive and unchanged until asgd_destroy().
+ *   X_bf16_dev   DEVICE [N*d] bf16 copy of X for ASGD_PATH_TC_BF16, or NULL.
+ *   w0_dev       DEVICE [k*d] fp32.  COPIED.
+ *   workspace    DEVICE, >= asgd_workspace_bytes(), 256-byte aligned.  BORROWED until destroy.
+ *   cuda_stream  a cudaStream_t (NULL = default stream).
+ */
+int asgd_init(asgd_ctx **out, const asgd_config *cfg, const float *X_dev, const void *X_bf16_dev,
+              const float *w0_dev, void *workspace_dev, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Deterministic mode.  `rounds` synchronous rounds: in a round every worker performs one step of
+ * Algorithm 5 (mini-batch, Eq. 8 assignment, Eq. 9 gradient, Eq. 4 tests, Eq. 6 update) from the
+ * states and receive buffers it had when the round began; then the round's puts are delivered as
+ * whole messages, senders in ascending order (the last sender into a buffer wins).
+ */
+int asgd_step(asgd_ctx *ctx, int64_t rounds);
+
+/*
+ * Free-running mode (Section 1.2): one persistent launch in which every worker performs
+ * `steps_per_worker` steps at its own pace; puts are plain stores into the recipient's buffer
+ * published by a release-increment of its sequence number, never acknowledged, never waited for.
+ * Messages may be lost or torn (Section 4.4).  Returns after enqueue.
+ */
+int asgd_run(asgd_ctx *ctx, int64_t steps_per_worker);
+
+/* State of one worker (worker 0 is the w^1 that Algorithm 5 returns); worker = -1 gives the mean
+ * over all workers (the aggregation variant of Section 4.3).  out_dev: DEVICE [k*d], caller's. */
+int asgd_get_state(asgd_ctx *ctx, int32_t worker, float *out_dev);
+/* Overwrite one worker's state (resume from an earlier run, Section 4 "Initialization"). */
+int asgd_set_state(asgd_ctx *ctx, int32_t worker, const float *w_dev /* DEVICE [k*d] */);
+/* A put from outside: write a whole message into receive buffer `slot` of `worker`. */
+int asgd_put(asgd_ctx *ctx, int32_t worker, int32_t slot, const float *payload_dev /* DEVICE [k*d] */);
+
+/* Eq. 8: E(w) of the given worker's state (-1 = mean state) over all N rows.  Synchronises. */
+int asgd_eval(asgd_ctx *ctx, int32_t worker, double *E_host /* HOST out */);
+
+/* out_host[5] = steps, messages sent, received, accepted ("good", delta = 1), overwritten unread.
+ * Synchronises. */
+int asgd_get_stats(asgd_ctx *ctx, int32_t worker, uint64_t *out_host /* HOST [5] */);
+
+/* Assignments s_i(w) of the last deterministic round, [W*b] int32 in worker-major order.
+ * Needs cfg.record_assign = 1.  out_dev: DEVICE, caller's. */
+int asgd_get_assign(asgd_ctx *ctx, int32_t *out_dev);
+/* Per-slot acceptance of the last step of `worker`: out_host[S], -1 nothing new, 0 rejected,
+ * 1 accepted.  Synchronises. */
+int asgd_get_accept(asgd_ctx *ctx, int32_t worker, int32_t *out_host /* HOST [S] */);
+
+/* Wait for the stream and return the device status word (ASGD_OK or ASGD_ETIMEOUT ...). */
+int asgd_sync(asgd_ctx *ctx);
+/* Number of kernels this context has launched so far. */
+int64_t asgd_launch_count(const asgd_ctx *ctx);
+/* Name of the distance path the context resolved to ("fp32-generic", "fp32-stream", ...). */
+const char *asgd_path_name(const asgd_ctx *ctx);
+/* cudaError_t of the last failed CUDA call in this context (0 if none). */
+int asgd_last_cuda_error(const asgd_ctx *ctx);
+const char *asgd_strerror(int status);
+void asgd_destroy(asgd_ctx *ctx);
+
+/*
+ * Whole job from HOST buffers (Algorithm 5 end to end): copies X and w0 to the device, runs
+ * `steps_per_worker` steps per worker (free-running if cfg is used with mode_async != 0, else
+ * deterministic rounds), copies worker 0's state back.  Synchronises before returning.
+ *   X_host       HOST [N*d] fp32 (pinned memory gives the best copy rate)
+ *   w0_host      HOST [k*d]
+ *   w_out_host   HOST [k*d] out
+ *   scratch_dev  DEVICE, >= asgd_fit_host_bytes(cfg) bytes, 256-byte aligned
+ */
+int asgd_fit_host_bytes(const asgd_config *cfg, size_t *bytes /* HOST out */);
+int asgd_fit_host(const asgd_config *cfg, const float *X_host, const float *w0_host,
+                  int64_t steps_per_worker, int32_t mode_async, float *w_out_host,
+                  void *scratch_dev, size_t scratch_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASGD_H_ */

@@ -1,0 +1,405 @@
+// C ABI of the K-Means ASGD library: context, argument checks, workspace layout, launches.
+// Declarations and argument contracts are in include/asgd.h.
+
+#include "../../include/asgd.h"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "asgd_aux.cuh"
+#include "asgd_generic.cuh"
+
+using namespace asgd;
+
+namespace {
+
+enum PathId { P_GENERIC = 0 };
+
+struct Layout {
+  size_t state, mail, seq, seen, arb_win, arb_cnt, stats, perm, status, assign_rec, accept_rec, gsum,
+      eval_partial, tmp_state, xmax, total;
+};
+
+constexpr size_t kAlign = 256;
+constexpr int kEvalBlocks = 148 * 8;
+constexpr size_t kMaxDynSmem = 227 * 1024;
+
+inline size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+bool config_ok(const asgd_config* c) {
+  if (!c) return false;
+  if (c->N <= 0 || c->d <= 0 || c->k <= 0 || c->W <= 0 || c->b <= 0) return false;
+  if (!(c->eps > 0.f)) return false;
+  if (c->comm_interval < 0 || c->fanout < 0 || c->fanout > c->W - 1 || c->fanout > MAX_FANOUT) return false;
+  if (c->slots < 1 || c->slots > MAX_SLOTS) return false;
+  if (c->reserved != 0) return false;
+  if (c->dist_path < ASGD_PATH_AUTO || c->dist_path > ASGD_PATH_TC_BF16) return false;
+  if ((long long)c->k * c->d > (1ll << 28)) return false;
+  const long long H = c->N / c->W;
+  if (H < c->b) return false;
+  if ((long long)c->W * c->fanout + 1 > 0x7fffffffll) return false;
+  return true;
+}
+
+Layout make_layout(const asgd_config* c) {
+  Layout L{};
+  const size_t W = c->W, S = c->slots;
+  const size_t kd = (size_t)c->k * c->d, kd_pad = (kd + 3) / 4 * 4;
+  const size_t H = c->N / c->W, B = H / c->b;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += up(bytes); return o; };
+  L.state = take(W * kd_pad * 4);
+  L.mail = take(W * S * kd_pad * 4);
+  L.seq = take(W * S * 4);
+  L.seen = take(W * S * 4);
+  L.arb_win = take(W * S * 4);
+  L.arb_cnt = take(W * S * 4);
+  L.stats = take(W * ST_STRIDE * 8);
+  L.perm = take(W * B * 4);
+  L.status = take(64);
+  L.assign_rec = take(c->record_assign ? W * (size_t)c->b * 4 : 4);
+  L.accept_rec = take(W * S * 4);
+  L.gsum = take(W * kd_pad * 4);
+  L.eval_partial = take((size_t)kEvalBlocks * 8);
+  L.tmp_state = take(kd_pad * 4);
+  L.xmax = take(64);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+
+struct asgd_ctx {
+  asgd_config cfg;
+  Params p;
+  Layout L;
+  unsigned char* ws;
+  cudaStream_t stream;
+  int path;
+  int state_on_chip;
+  size_t smem_bytes;
+  long long t_host;       // steps every worker has done (uniform across workers)
+  long long launches;
+  int last_cuda;
+  int sm_count;
+};
+
+namespace {
+
+int cuda_fail(asgd_ctx* c, cudaError_t e) {
+  if (c) c->last_cuda = (int)e;
+  return ASGD_ECUDA;
+}
+#define CU(ctx, call)                                   \
+  do {                                                  \
+    cudaError_t e_ = (call);                            \
+    if (e_ != cudaSuccess) return cuda_fail((ctx), e_); \
+  } while (0)
+
+// Batch order of one worker: Fisher-Yates from the top, driven by the schedule hash.
+void fill_perm(const asgd_config& c, long long B, int worker, int* perm) {
+  for (long long q = 0; q < B; ++q) perm[q] = (int)q;
+  if (!c.shuffle) return;
+  for (long long q = B - 1; q >= 1; --q) {
+    const unsigned long long r =
+        sched_draw(c.seed, TAG_PERM, (unsigned long long)worker, (unsigned long long)q, 0ull) % (unsigned long long)(q + 1);
+    std::swap(perm[q], perm[r]);
+  }
+}
+
+int launch_workers(asgd_ctx* c, bool det, long long steps) {
+  const Params& p = c->p;
+  switch (c->path) {
+    case P_GENERIC:
+    default:
+      if (det)
+        asgd_generic_kernel<true><<<p.W, GENERIC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->state_on_chip);
+      else
+        asgd_generic_kernel<false><<<p.W, GENERIC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->state_on_chip);
+      break;
+  }
+  c->launches += 1;
+  CU(c, cudaGetLastError());
+  return ASGD_OK;
+}
+
+int resolve_path(asgd_ctx* c) {
+  const asgd_config& cfg = c->cfg;
+  if (cfg.dist_path == ASGD_PATH_TC_3XTF32 || cfg.dist_path == ASGD_PATH_TC_BF16) return ASGD_EUNSUPPORTED;
+  c->path = P_GENERIC;
+  const int kd_pad = c->p.kd_pad;
+  size_t on = generic_smem_bytes(cfg.k, cfg.b, kd_pad, true);
+  size_t off = generic_smem_bytes(cfg.k, cfg.b, kd_pad, false);
+  if (on <= 200 * 1024) {
+    c->state_on_chip = 1;
+    c->smem_bytes = on;
+  } else if (off <= kMaxDynSmem) {
+    c->state_on_chip = 0;
+    c->smem_bytes = off;
+  } else {
+    return ASGD_EUNSUPPORTED;
+  }
+  CU(c, cudaFuncSetAttribute(asgd_generic_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  CU(c, cudaFuncSetAttribute(asgd_generic_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  return ASGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int asgd_workspace_bytes(const asgd_config* cfg, size_t* bytes) {
+  if (!bytes || !config_ok(cfg)) return ASGD_EINVAL;
+  *bytes = make_layout(cfg).total;
+  return ASGD_OK;
+}
+
+int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const void* X_bf16_dev,
+              const float* w0_dev, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
+  (void)X_bf16_dev;
+  if (!out) return ASGD_EINVAL;
+  *out = nullptr;
+  if (!config_ok(cfg) || !X_dev || !w0_dev || !workspace_dev) return ASGD_EINVAL;
+  if (((uintptr_t)X_dev & 15) || ((uintptr_t)workspace_dev & (kAlign - 1))) return ASGD_EINVAL;
+  Layout L = make_layout(cfg);
+  if (workspace_bytes < L.total) return ASGD_ENOMEM;
+
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return ASGD_EUNSUPPORTED;
+  if (prop.major != 10) return ASGD_EUNSUPPORTED;
+
+  asgd_ctx* c = new (std::nothrow) asgd_ctx();
+  if (!c) return ASGD_ENOMEM;
+  c->cfg = *cfg;
+  c->L = L;
+  c->ws = (unsigned char*)workspace_dev;
+  c->stream = (cudaStream_t)cuda_stream;
+  c->t_host = 0;
+  c->launches = 0;
+  c->last_cuda = 0;
+  c->sm_count = prop.multiProcessorCount;
+
+  Params& p = c->p;
+  p.X = X_dev; p.N = cfg->N; p.d = cfg->d; p.k = cfg->k; p.W = cfg->W; p.b = cfg->b; p.eps = cfg->eps;
+  p.c = cfg->comm_interval; p.f = cfg->fanout; p.S = cfg->slots; p.parzen = cfg->parzen ? 1 : 0;
+  p.seed = cfg->seed;
+  p.H = cfg->N / cfg->W; p.B = p.H / cfg->b;
+  p.kd = cfg->k * cfg->d; p.kd_pad = (p.kd + 3) / 4 * 4;
+  p.state = (float*)(c->ws + L.state);
+  p.mail = (float*)(c->ws + L.mail);
+  p.seq = (unsigned*)(c->ws + L.seq);
+  p.seen = (unsigned*)(c->ws + L.seen);
+  p.arb_win = (unsigned*)(c->ws + L.arb_win);
+  p.arb_cnt = (unsigned*)(c->ws + L.arb_cnt);
+  p.stats = (unsigned long long*)(c->ws + L.stats);
+  p.perm = (const int*)(c->ws + L.perm);
+  p.status = (int*)(c->ws + L.status);
+  p.assign_rec = cfg->record_assign ? (int*)(c->ws + L.assign_rec) : nullptr;
+  p.accept_rec = (int*)(c->ws + L.accept_rec);
+  p.gsum = (float*)(c->ws + L.gsum);
+  p.xmax2 = 0.f;
+
+  int rc = resolve_path(c);
+  if (rc != ASGD_OK) { delete c; return rc; }
+
+  // empty buffers, zero counters (everything between mail and perm, plus status/records)
+  cudaError_t e = cudaMemsetAsync(c->ws + L.mail, 0, L.perm - L.mail, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->ws + L.status, 0, L.total - L.status, c->stream);
+  if (e != cudaSuccess) { delete c; return ASGD_ECUDA; }
+  broadcast_state_kernel<<<256, 256, 0, c->stream>>>(p.state, w0_dev, p.W, p.kd, p.kd_pad);
+  c->launches += 1;
+
+  // batch orders
+  {
+    std::vector<int> perm;
+    try { perm.resize((size_t)p.W * p.B); } catch (...) { delete c; return ASGD_ENOMEM; }
+    for (int i = 0; i < p.W; ++i) fill_perm(*cfg, p.B, i, perm.data() + (size_t)i * p.B);
+    e = cudaMemcpyAsync(c->ws + L.perm, perm.data(), perm.size() * sizeof(int), cudaMemcpyHostToDevice, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // perm is a local: finish the copy
+    if (e != cudaSuccess) { delete c; return ASGD_ECUDA; }
+  }
+  *out = c;
+  return ASGD_OK;
+}
+
+int asgd_step(asgd_ctx* c, int64_t rounds) {
+  if (!c || rounds < 0) return ASGD_EINVAL;
+  const Params& p = c->p;
+  for (int64_t r = 0; r < rounds; ++r) {
+    int rc = launch_workers(c, true, 1);
+    if (rc != ASGD_OK) return rc;
+    if (p.c > 0 && p.f > 0 && p.W > 1 && (c->t_host + 1) % p.c == 0) {
+      deliver_kernel<<<p.W * p.S, 128, 0, c->stream>>>(p);
+      c->launches += 1;
+      CU(c, cudaGetLastError());
+    }
+    c->t_host += 1;
+  }
+  return ASGD_OK;
+}
+
+int asgd_run(asgd_ctx* c, int64_t steps_per_worker) {
+  if (!c || steps_per_worker < 0) return ASGD_EINVAL;
+  if (steps_per_worker == 0) return ASGD_OK;
+  int rc = launch_workers(c, false, steps_per_worker);
+  if (rc != ASGD_OK) return rc;
+  c->t_host += steps_per_worker;
+  return ASGD_OK;
+}
+
+int asgd_get_state(asgd_ctx* c, int32_t worker, float* out_dev) {
+  if (!c || !out_dev || worker < -1 || worker >= c->p.W) return ASGD_EINVAL;
+  const Params& p = c->p;
+  if (worker >= 0) {
+    CU(c, cudaMemcpyAsync(out_dev, p.state + (size_t)worker * p.kd_pad, (size_t)p.kd * 4, cudaMemcpyDeviceToDevice, c->stream));
+  } else {
+    mean_state_kernel<<<(p.kd + 255) / 256, 256, 0, c->stream>>>(p.state, p.W, p.kd, p.kd_pad, out_dev);
+    c->launches += 1;
+    CU(c, cudaGetLastError());
+  }
+  return ASGD_OK;
+}
+
+int asgd_set_state(asgd_ctx* c, int32_t worker, const float* w_dev) {
+  if (!c || !w_dev || worker < 0 || worker >= c->p.W) return ASGD_EINVAL;
+  const Params& p = c->p;
+  CU(c, cudaMemcpyAsync(p.state + (size_t)worker * p.kd_pad, w_dev, (size_t)p.kd * 4, cudaMemcpyDeviceToDevice, c->stream));
+  return ASGD_OK;
+}
+
+int asgd_put(asgd_ctx* c, int32_t worker, int32_t slot, const float* payload_dev) {
+  if (!c || !payload_dev || worker < 0 || worker >= c->p.W || slot < 0 || slot >= c->p.S) return ASGD_EINVAL;
+  const Params& p = c->p;
+  const size_t ri = (size_t)worker * p.S + slot;
+  external_put_kernel<<<1, 256, 0, c->stream>>>(p.mail + ri * (size_t)p.kd_pad, payload_dev, p.seq + ri, p.kd);
+  c->launches += 1;
+  CU(c, cudaGetLastError());
+  return ASGD_OK;
+}
+
+int asgd_eval(asgd_ctx* c, int32_t worker, double* E_host) {
+  if (!c || !E_host || worker < -1 || worker >= c->p.W) return ASGD_EINVAL;
+  const Params& p = c->p;
+  const float* w = nullptr;
+  if (worker >= 0) {
+    w = p.state + (size_t)worker * p.kd_pad;
+  } else {
+    float* tmp = (float*)(c->ws + c->L.tmp_state);
+    int rc = asgd_get_state(c, -1, tmp);
+    if (rc != ASGD_OK) return rc;
+    w = tmp;
+  }
+  const size_t wbytes = (size_t)p.kd * 4;
+  const int on_chip = wbytes <= 160 * 1024;
+  const size_t smem = 32 * sizeof(double) + (on_chip ? wbytes : 0);
+  CU(c, cudaFuncSetAttribute(eval_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  double* partial = (double*)(c->ws + c->L.eval_partial);
+  eval_kernel<<<kEvalBlocks, EVAL_THREADS, smem, c->stream>>>(p.X, p.N, p.d, p.k, w, on_chip, partial);
+  c->launches += 1;
+  CU(c, cudaGetLastError());
+  std::vector<double> host(kEvalBlocks);
+  CU(c, cudaMemcpyAsync(host.data(), partial, sizeof(double) * kEvalBlocks, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  double E = 0.0;
+  for (int q = 0; q < kEvalBlocks; ++q) E += host[q];
+  *E_host = E;
+  return ASGD_OK;
+}
+
+int asgd_get_stats(asgd_ctx* c, int32_t worker, uint64_t* out_host) {
+  if (!c || !out_host || worker < 0 || worker >= c->p.W) return ASGD_EINVAL;
+  unsigned long long row[ST_STRIDE];
+  CU(c, cudaMemcpyAsync(row, c->p.stats + (size_t)worker * ST_STRIDE, sizeof(row), cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  for (int q = 0; q < 5; ++q) out_host[q] = row[q];
+  return ASGD_OK;
+}
+
+int asgd_get_assign(asgd_ctx* c, int32_t* out_dev) {
+  if (!c || !out_dev || !c->p.assign_rec) return ASGD_EINVAL;
+  CU(c, cudaMemcpyAsync(out_dev, c->p.assign_rec, (size_t)c->p.W * c->p.b * 4, cudaMemcpyDeviceToDevice, c->stream));
+  return ASGD_OK;
+}
+
+int asgd_get_accept(asgd_ctx* c, int32_t worker, int32_t* out_host) {
+  if (!c || !out_host || worker < 0 || worker >= c->p.W) return ASGD_EINVAL;
+  CU(c, cudaMemcpyAsync(out_host, c->p.accept_rec + (size_t)worker * c->p.S, (size_t)c->p.S * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  return ASGD_OK;
+}
+
+int asgd_sync(asgd_ctx* c) {
+  if (!c) return ASGD_EINVAL;
+  int st[4] = {0, 0, 0, 0};
+  CU(c, cudaMemcpyAsync(st, c->p.status, sizeof(st), cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  if (st[0] == DEV_TIMEOUT) return ASGD_ETIMEOUT;
+  return ASGD_OK;
+}
+
+int64_t asgd_launch_count(const asgd_ctx* c) { return c ? c->launches : 0; }
+
+const char* asgd_path_name(const asgd_ctx* c) {
+  if (!c) return "none";
+  switch (c->path) {
+    case P_GENERIC: return c->state_on_chip ? "fp32-generic" : "fp32-generic-offchip";
+    default: return "unknown";
+  }
+}
+
+int asgd_last_cuda_error(const asgd_ctx* c) { return c ? c->last_cuda : 0; }
+
+const char* asgd_strerror(int s) {
+  switch (s) {
+    case ASGD_OK: return "ok";
+    case ASGD_EINVAL: return "invalid argument";
+    case ASGD_ENOMEM: return "workspace too small or host allocation failed";
+    case ASGD_ECUDA: return "CUDA call failed";
+    case ASGD_EUNSUPPORTED: return "unsupported device or problem size";
+    case ASGD_ETIMEOUT: return "a bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+void asgd_destroy(asgd_ctx* c) { delete c; }
+
+int asgd_fit_host_bytes(const asgd_config* cfg, size_t* bytes) {
+  if (!bytes || !config_ok(cfg)) return ASGD_EINVAL;
+  const size_t kd = (size_t)cfg->k * cfg->d;
+  *bytes = up((size_t)cfg->N * cfg->d * 4) + up(kd * 4) + up(kd * 4) + make_layout(cfg).total;
+  return ASGD_OK;
+}
+
+int asgd_fit_host(const asgd_config* cfg, const float* X_host, const float* w0_host, int64_t steps_per_worker,
+                  int32_t mode_async, float* w_out_host, void* scratch_dev, size_t scratch_bytes, void* cuda_stream) {
+  size_t need = 0;
+  if (asgd_fit_host_bytes(cfg, &need) != ASGD_OK || !X_host || !w0_host || !w_out_host || !scratch_dev ||
+      steps_per_worker < 0)
+    return ASGD_EINVAL;
+  if (scratch_bytes < need) return ASGD_ENOMEM;
+  if ((uintptr_t)scratch_dev & (kAlign - 1)) return ASGD_EINVAL;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  const size_t kd = (size_t)cfg->k * cfg->d, xb = (size_t)cfg->N * cfg->d * 4;
+  unsigned char* base = (unsigned char*)scratch_dev;
+  float* Xd = (float*)base;
+  float* w0d = (float*)(base + up(xb));
+  float* wod = (float*)(base + up(xb) + up(kd * 4));
+  void* ws = base + up(xb) + 2 * up(kd * 4);
+  if (cudaMemcpyAsync(Xd, X_host, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return ASGD_ECUDA;
+  if (cudaMemcpyAsync(w0d, w0_host, kd * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return ASGD_ECUDA;
+  asgd_ctx* c = nullptr;
+  int rc = asgd_init(&c, cfg, Xd, nullptr, w0d, ws, scratch_bytes - (size_t)((unsigned char*)ws - base), st);
+  if (rc != ASGD_OK) return rc;
+  rc = mode_async ? asgd_run(c, steps_per_worker) : asgd_step(c, steps_per_worker);
+  if (rc == ASGD_OK) rc = asgd_get_state(c, 0, wod);
+  if (rc == ASGD_OK && cudaMemcpyAsync(w_out_host, wod, kd * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) rc = ASGD_ECUDA;
+  if (rc == ASGD_OK) rc = asgd_sync(c);
+  asgd_destroy(c);
+  return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,107 @@
+// Small kernels around the worker loop: initial broadcast of w0, delivery of a synchronous round's
+// puts, external put, mean of the worker states, and the evaluation of E(w) (Eq. 8).
+#pragma once
+
+#include "asgd_common.cuh"
+
+namespace asgd {
+
+// Initialisation step of Section 4: the control thread's w0 goes to every worker.
+__global__ void broadcast_state_kernel(float* state, const float* w0, int W, int kd, int kd_pad) {
+  const size_t total = (size_t)W * kd_pad;
+  for (size_t g = (size_t)blockIdx.x * blockDim.x + threadIdx.x; g < total; g += (size_t)gridDim.x * blockDim.x) {
+    const int e = (int)(g % kd_pad);
+    state[g] = (e < kd) ? w0[e] : 0.f;
+  }
+}
+
+// Delivery of one synchronous round (deterministic mode).  One block per receive buffer; the
+// buffer takes the whole state of the last announcing sender (ascending sender, then recipient
+// index), and its sequence number advances by the number of messages that were aimed at it.
+__global__ void deliver_kernel(const Params p) {
+  const size_t ri = blockIdx.x;           // receiver * S + slot
+  const unsigned win = p.arb_win[ri];
+  if (win == 0) return;
+  const int sender = (int)((win - 1u) / (unsigned)p.f);
+  const float4* src = reinterpret_cast<const float4*>(p.state + (size_t)sender * p.kd_pad);
+  float4* dst = reinterpret_cast<float4*>(p.mail + ri * (size_t)p.kd_pad);
+  for (int e = threadIdx.x; e < p.kd_pad / 4; e += blockDim.x) dst[e] = src[e];
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    p.seq[ri] += p.arb_cnt[ri];
+    p.arb_win[ri] = 0;
+    p.arb_cnt[ri] = 0;
+  }
+}
+
+// A put from the host side of the library: whole message, then the sequence number.
+__global__ void external_put_kernel(float* dst, const float* src, unsigned* seq, int kd) {
+  for (int e = threadIdx.x; e < kd; e += blockDim.x) dst[e] = src[e];
+  __syncthreads();
+  if (threadIdx.x == 0) red_release_gpu_inc(seq);
+}
+
+// Aggregation variant of Section 4.3: out = (1/W) sum_i w^i, summed in ascending worker order.
+__global__ void mean_state_kernel(const float* state, int W, int kd, int kd_pad, float* out) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= kd) return;
+  double acc = 0.0;
+  for (int i = 0; i < W; ++i) acc += (double)state[(size_t)i * kd_pad + e];
+  out[e] = (float)(acc / (double)W);
+}
+
+// Eq. 8: E(w) = sum_i 1/2 min_k ||x_i - w_k||^2.  Direct difference form in fp32 per sample,
+// fp64 from the per-thread sum on.  One partial per block; the host adds them in block order.
+constexpr int EVAL_THREADS = 256;
+__global__ void __launch_bounds__(EVAL_THREADS)
+eval_kernel(const float* __restrict__ X, long long N, int d, int k, const float* __restrict__ wg,
+            int w_on_chip, double* partial) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* red = reinterpret_cast<double*>(smem_raw);
+  float* ws = reinterpret_cast<float*>(smem_raw + 32 * sizeof(double));
+  const float* w = wg;
+  if (w_on_chip) {
+    for (int e = threadIdx.x; e < k * d; e += blockDim.x) ws[e] = wg[e];
+    w = ws;
+  }
+  __syncthreads();
+  double acc = 0.0;
+  for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < N; r += (long long)gridDim.x * blockDim.x) {
+    const float* x = X + (size_t)r * d;
+    float bd = __int_as_float(0x7f800000);
+    for (int a = 0; a < k; ++a) {
+      const float* wa = w + (size_t)a * d;
+      float s = 0.f;
+      for (int j = 0; j < d; ++j) {
+        const float df = __ldg(x + j) - wa[j];
+        s = fmaf(df, df, s);
+      }
+      bd = fminf(bd, s);
+    }
+    acc += 0.5 * (double)bd;
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w_ = 0; w_ < (int)(blockDim.x >> 5); ++w_) s += red[w_];
+    partial[blockIdx.x] = s;
+  }
+}
+
+// max_i ||x_i||^2 over the rows the workers can touch (one pass at initialisation).
+__global__ void xmax2_kernel(const float* __restrict__ X, long long N, int d, unsigned* out_bits) {
+  float m = 0.f;
+  for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < N; r += (long long)gridDim.x * blockDim.x) {
+    const float* x = X + (size_t)r * d;
+    float s = 0.f;
+    for (int j = 0; j < d; ++j) { const float v = __ldg(x + j); s = fmaf(v, v, s); }
+    m = fmaxf(m, s);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) atomicMax(out_bits, __float_as_uint(m));   // non-negative floats order as uints
+}
+
+}  // namespace asgd

@@ -1,0 +1,232 @@
+"""CUDA library against the CPU oracle, element by element, on the same seeded inputs (C ABI calls)."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import paper_1505_04956_b200 as pkg
+from oracle import asgd_oracle as orc
+from tests.gpu_util import CENTRE_TOL, PARITY_WORKLOADS, Pair, decided, scaled
+
+pytestmark = pytest.mark.gpu
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _compare_stats(pr, exact_accept=True):
+    for i in range(pr.wl.W):
+        g, c = pr.gpu.get_stats(i), pr.cpu.stats(i)
+        for key in ("steps", "sent", "received", "overwritten"):
+            assert g[key] == c[key], (i, key, g, c)
+        if exact_accept:
+            assert g["accepted"] == c["accepted"], (i, g, c)
+
+
+def _accept_decided(tr, s, eps_rel=1e-5):
+    """True when the oracle's Eq. 4 comparison is decided beyond the relative gap."""
+    return abs(tr["lhs"][s] - tr["rhs"][s]) >= eps_rel * tr["rhs"][s]
+
+
+@pytest.mark.parametrize("name", list(PARITY_WORKLOADS))
+def test_trajectory_matches_oracle(name):
+    wl, rounds = PARITY_WORKLOADS[name]
+    pr = Pair(wl)
+    step = max(1, rounds // 8)
+    done = 0
+    undecided_accepts = 0
+    while done < rounds:
+        n = min(step, rounds - done)
+        pr.rounds(n)
+        done += n
+        pr.gpu.sync()
+        assert pr.max_rel_l2() < CENTRE_TOL, (name, done, pr.max_rel_l2())
+        for i in range(wl.W):
+            tr = pr.cpu.last_step(i)
+            acc = pr.gpu.get_accept(i)
+            for s in range(pr.S):
+                if tr["accept"][s] < 0:
+                    assert acc[s] == -1
+                elif _accept_decided(tr, s):
+                    assert acc[s] == tr["accept"][s], (name, done, i, s, tr["lhs"][s], tr["rhs"][s])
+                else:
+                    undecided_accepts += 1
+    _compare_stats(pr, exact_accept=False)
+    tot_g = sum(pr.gpu.get_stats(i)["accepted"] for i in range(wl.W))
+    tot_c = sum(pr.cpu.stats(i)["accepted"] for i in range(wl.W))
+    tot_r = sum(pr.cpu.stats(i)["received"] for i in range(wl.W))
+    assert abs(tot_g - tot_c) <= max(2, 0.01 * tot_r), (tot_g, tot_c, tot_r)
+    if wl.comm_interval > 0 and wl.fanout > 0:
+        assert tot_r > 0
+    pr.close()
+
+
+@pytest.mark.parametrize("name", list(PARITY_WORKLOADS))
+def test_single_step_assignments_bit_exact(name):
+    wl, rounds = PARITY_WORKLOADS[name]
+    pr = Pair(wl)
+    warm = min(rounds, 5)
+    pr.cpu.rounds(warm)
+    pr.gpu.step(warm)
+    # restart the GPU from the oracle's states so that an earlier rounding difference cannot matter
+    pr.load_oracle_states_into_gpu()
+    pr.rounds(1)
+    pr.gpu.sync()
+    got = pr.gpu.get_assign().cpu().numpy()
+    checked = 0
+    for i in range(wl.W):
+        tr = pr.cpu.last_step(i)
+        ok = decided(tr["d1"], tr["d2"])
+        assert (got[i][ok] == tr["assign"][ok]).all(), (name, i)
+        checked += int(ok.sum())
+        if ok.all():
+            assert np.bincount(got[i], minlength=wl.k).tolist() == tr["counts"].tolist()
+    assert checked >= 0.99 * wl.W * wl.b
+    assert pr.max_rel_l2() < CENTRE_TOL
+    pr.close()
+
+
+def test_parzen_hand_cases_on_gpu():
+    for line in open(os.path.join(GOLD, "parzen_1d_cases.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        w, x, eps, v, parzen, delta, w_new = (float(s) for s in line.split())
+        wl = scaled("tiny", N=8, d=1, k=1, W=2, b=4, eps=eps, comm_interval=0, fanout=1)
+        X = np.full((8, 1), x, np.float32)
+        pr = Pair(wl, parzen=int(parzen), X=X, w0=np.array([[w]], np.float32), oracle=False)
+        pr.gpu.put(0, 0, torch.tensor([[v]], dtype=torch.float32, device="cuda"))
+        pr.gpu.step(1)
+        pr.gpu.sync()
+        assert pr.gpu.get_accept(0) == [int(delta)], line
+        assert pr.gpu.get_accept(1) == [-1]
+        assert abs(float(pr.gpu.get_state(0).cpu()[0, 0]) - w_new) < 2e-6, line
+        assert abs(float(pr.gpu.get_state(1).cpu()[0, 0]) - (w - eps * (w - x))) < 2e-6
+        st = pr.gpu.get_stats(0)
+        assert st["received"] == 1 and st["accepted"] == int(delta) and st["steps"] == 1
+        pr.close()
+
+
+EDGE_CASES = {
+    "one_worker": dict(N=997, d=3, k=4, W=1, b=33, comm_interval=1, fanout=0),
+    "batch_of_one": dict(N=64, d=5, k=3, W=4, b=1, comm_interval=1, fanout=1),
+    "one_centre": dict(N=640, d=7, k=1, W=4, b=40, comm_interval=2, fanout=2),
+    "one_dim": dict(N=640, d=1, k=5, W=4, b=40, comm_interval=1, fanout=1),
+    "more_centres_than_samples": dict(N=400, d=6, k=50, W=4, b=10, comm_interval=1, fanout=1),
+    "silent": dict(N=4000, d=10, k=10, W=8, b=100, comm_interval=0, fanout=1),
+    "fanout_all_peers": dict(N=4000, d=10, k=10, W=5, b=50, comm_interval=1, fanout=4),
+    "ragged_rows": dict(N=4003, d=9, k=7, W=7, b=37, comm_interval=3, fanout=2),
+    "odd_kd": dict(N=3000, d=3, k=3, W=3, b=97, comm_interval=1, fanout=1),
+}
+
+
+@pytest.mark.parametrize("case", list(EDGE_CASES))
+@pytest.mark.parametrize("parzen", [1, 0])
+def test_edge_cases(case, parzen):
+    kw = dict(EDGE_CASES[case])
+    wl = scaled("tiny", eps=0.1, **kw)
+    slots = 3 if case in ("fanout_all_peers", "ragged_rows") else None
+    pr = Pair(wl, parzen=parzen, slots=slots)
+    rounds = 2 * wl.B + 3
+    pr.rounds(rounds)
+    pr.gpu.sync()
+    assert pr.max_rel_l2() < CENTRE_TOL, (case, pr.max_rel_l2())
+    _compare_stats(pr, exact_accept=(parzen == 0))
+    pr.close()
+
+
+def test_unshuffled_batches_and_many_slots():
+    wl = scaled("tiny", N=6000, W=6, comm_interval=1, fanout=3)
+    pr = Pair(wl, shuffle=0, slots=2)
+    pr.rounds(25)
+    pr.gpu.sync()
+    assert pr.max_rel_l2() < CENTRE_TOL
+    _compare_stats(pr, exact_accept=False)
+    assert sum(pr.cpu.stats(i)["overwritten"] for i in range(wl.W)) > 0     # collisions did happen
+    pr.close()
+
+
+def test_eval_and_mean_state():
+    wl = scaled("tiny", N=50_000)
+    pr = Pair(wl)
+    pr.rounds(30)
+    E = pr.gpu.eval(0)
+    want = orc.quantization_error(pr.Xh, pr.gpu.get_state(0).cpu().numpy())
+    assert abs(E - want) <= 1e-5 * want
+    mean = pr.gpu.get_state(-1).cpu().numpy()
+    assert np.allclose(mean, pr.gpu_states().astype(np.float64).mean(0), rtol=1e-6, atol=1e-6)
+    Em = pr.gpu.eval(-1)
+    assert abs(Em - orc.quantization_error(pr.Xh, mean)) <= 1e-5 * Em
+    pr.close()
+
+
+def test_free_running_mode_reaches_the_oracles_error():
+    wl = scaled("tiny")
+    pr = Pair(wl, record_assign=0)
+    steps = wl.steps_per_worker()
+    pr.gpu.run(steps)
+    pr.gpu.sync()
+    pr.cpu.rounds(steps)
+    E_gpu = orc.quantization_error(pr.Xh, pr.gpu.get_state(0).cpu().numpy())
+    E_cpu = orc.quantization_error(pr.Xh, pr.cpu.state(0))
+    assert abs(E_gpu - E_cpu) <= 0.01 * E_cpu, (E_gpu, E_cpu)
+    tot = {key: sum(pr.gpu.get_stats(i)[key] for i in range(wl.W)) for key in
+           ("steps", "sent", "received", "accepted", "overwritten")}
+    assert tot["steps"] == wl.W * steps
+    assert tot["sent"] == wl.W * wl.fanout * (steps // wl.comm_interval)
+    assert tot["received"] + tot["overwritten"] <= tot["sent"]
+    assert tot["accepted"] <= tot["received"]
+    pr.close()
+
+
+def test_mixing_deterministic_rounds_and_free_running():
+    wl = scaled("tiny", N=20_000)
+    pr = Pair(wl, record_assign=0)
+    pr.rounds(10)
+    pr.gpu.sync()
+    assert pr.max_rel_l2() < CENTRE_TOL
+    pr.gpu.run(15)
+    pr.gpu.step(5)
+    pr.gpu.sync()
+    assert all(pr.gpu.get_stats(i)["steps"] == 30 for i in range(wl.W))
+    pr.close()
+
+
+def test_fit_host_end_to_end():
+    wl = scaled("tiny", N=20_000)
+    pr = Pair(wl, record_assign=0)
+    rounds = 40
+    pr.rounds(rounds)
+    cfg = pr.cfg
+    cfg.record_assign = 0
+    Xp = torch.from_numpy(pr.Xh).pin_memory()
+    w0p = torch.from_numpy(pr.w0h).pin_memory()
+    out = torch.empty((wl.k, wl.d), dtype=torch.float32).pin_memory()
+    scratch = torch.empty(pkg.asgd_fit_host_bytes(cfg) + 256, dtype=torch.uint8, device="cuda")
+    off = (-scratch.data_ptr()) % 256
+    pkg.asgd_fit_host(cfg, Xp, w0p, rounds, False, out, scratch[off:])
+    assert np.array_equal(out.numpy(), pr.gpu.get_state(0).cpu().numpy())
+    pr.close()
+
+
+def test_error_returns():
+    import ctypes as C
+    L = pkg.load()
+    wl = scaled("tiny", N=2000)
+    pr = Pair(wl, oracle=False)
+    cfg = pr.cfg
+    need = pkg.asgd_workspace_bytes(cfg)
+    ws = torch.empty(need + 512, dtype=torch.uint8, device="cuda")
+    base = (ws.data_ptr() + 255) // 256 * 256
+    h = C.c_void_p()
+    st = C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    args = (C.byref(cfg), C.c_void_p(pr.X.data_ptr()), None, C.c_void_p(pr.w0.data_ptr()))
+    assert L.asgd_init(C.byref(h), *args, C.c_void_p(base), need - 1, st) == pkg.binding.ASGD_ENOMEM
+    assert L.asgd_init(C.byref(h), *args, C.c_void_p(base + 8), need, st) == pkg.binding.ASGD_EINVAL
+    assert L.asgd_init(C.byref(h), C.byref(cfg), C.c_void_p(pr.X.data_ptr() + 4), None, C.c_void_p(pr.w0.data_ptr()),
+                       C.c_void_p(base), need, st) == pkg.binding.ASGD_EINVAL
+    with pytest.raises(pkg.AsgdError):
+        pr.gpu.get_state(wl.W)
+    with pytest.raises(pkg.AsgdError):
+        pr.gpu.put(0, pr.S, pr.w0)
+    with pytest.raises(ValueError):
+        pkg.Asgd(cfg, pr.X.cpu(), pr.w0.cpu())
+    pr.close()
