@@ -1,0 +1,281 @@
+#!/usr/bin/env python
+"""Throughput of the K-Means ASGD worker loop on B200: samples/s, achieved HBM GB/s, roofline fraction.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload stream]
+
+One bench "step" is one full pass of every worker over its shard in free-running mode (a single
+asgd_run launch: mini-batch draw, assignment, per-centre sums, gradient, receive buffers with the
+Parzen test, update, puts).  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "K-Means ASGD samples/s"
+UNIT = "samples/s"
+CPU_SAMPLE_ROWS = 1 << 25          # prefix of the workload the CPU baseline runs on
+NOMINAL_HBM_GBS = 8000.0
+
+
+def env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        return float(pk["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle samples while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes_per_pass(wl, steps):
+    """One read of every used sample (d*4 B) plus the put payloads (k*d*4 B per recipient per put)."""
+    sample_bytes = wl.W * steps * wl.b * wl.d * 4
+    puts = wl.W * wl.fanout * (steps // wl.comm_interval if wl.comm_interval > 0 else 0)
+    return sample_bytes + puts * wl.k * wl.d * 4
+
+
+def cpu_baseline(wl, sample_rows, threads=None, min_seconds=0.0):
+    """The oracle, as it stands, on a prefix of the workload; returns (samples/s, description, threads)."""
+    import numpy as np  # noqa: F401
+    from oracle import asgd_oracle as orc
+    from paper_1505_04956_b200 import inputs
+    sub = wl.scaled(N=min(sample_rows, wl.N))
+    X, _ = inputs.make_samples(sub, device="cpu")
+    w0 = inputs.initial_centres(sub, X)
+    th = threads or min(os.cpu_count() or 1, orc.max_threads(), sub.W)
+    o = orc.Oracle(X.numpy(), w0.numpy(), W=sub.W, b=sub.b, eps=sub.eps, comm_interval=sub.comm_interval,
+                   fanout=sub.fanout, seed=sub.seed, threads=th)
+    rounds = sub.B
+    t0 = time.perf_counter()
+    done = 0
+    while True:
+        o.rounds(rounds)
+        done += rounds
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds:
+            break
+    val = sub.W * done * sub.b / dt
+    desc = "first %d rows of the workload (W=%d, b=%d), %d synchronous rounds, %.1f s" % (sub.N, sub.W, sub.b, done, dt)
+    o.close()
+    return val, desc, o.threads
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on bounded samples of the same workload."""
+    from paper_1505_04956_b200 import inputs
+    rank = env_int("RANK", 0)
+    if rank != 0:
+        return 0
+    from oracle import asgd_oracle as orc
+    wl = inputs.WORKLOADS[args.workload]
+    sub = wl.scaled(N=min(args.reference_rows, wl.N))
+    X, _ = inputs.make_samples(sub, device="cpu")
+    w0 = inputs.initial_centres(sub, X)
+    th = min(os.cpu_count() or 1, orc.max_threads(), sub.W)
+    o = orc.Oracle(X.numpy(), w0.numpy(), W=sub.W, b=sub.b, eps=sub.eps, comm_interval=sub.comm_interval,
+                   fanout=sub.fanout, seed=sub.seed, threads=th)
+    for _ in range(args.warmup):
+        o.rounds(sub.B)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        o.rounds(sub.B)
+    dt = time.perf_counter() - t0
+    val = sub.W * sub.B * sub.b * args.steps / dt
+    sample = "each step = one pass over the first %d rows (W=%d, b=%d, %d rounds)" % (sub.N, sub.W, sub.b, sub.B)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(1, args.steps), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "k": wl.k, "W": wl.W, "b": wl.b},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": o.threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="stream")
+    ap.add_argument("--rows", type=int, default=0, help="use only the first ROWS rows (profiling of a small case)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--reference-rows", type=int, default=1 << 23)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import paper_1505_04956_b200 as pkg
+    from paper_1505_04956_b200 import dist, inputs
+
+    args.warmup = max(args.warmup, 3)
+    rank, world, local = dist.init_from_env(backend="nccl")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    pkg.load()
+
+    wl = inputs.WORKLOADS[args.workload]
+    if args.rows:
+        wl = wl.scaled(N=args.rows)
+    # each rank owns an independent group of W workers on its own seeded shard (no cross-GPU exchange)
+    wl_rank = wl.scaled(seed=dist.shard_seed(wl.seed, rank, world))
+    X, _ = inputs.make_samples(wl_rank, device=dev)
+    w0 = inputs.initial_centres(wl_rank, X)
+    cfg = pkg.make_config(N=wl.N, d=wl.d, k=wl.k, W=wl.W, b=wl.b, eps=wl.eps, comm_interval=wl.comm_interval,
+                          fanout=wl.fanout, seed=wl_rank.seed)
+    ctx = pkg.Asgd(cfg, X, w0)
+    steps = wl.B                                   # one pass
+    samples_per_pass = wl.W * steps * wl.b
+
+    for _ in range(args.warmup):
+        ctx.run(steps)
+    ctx.sync()
+    sampler = ClockSampler(local)
+    l0 = ctx.launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    ev[0].record()
+    for s in range(args.steps):
+        ctx.run(steps)
+        ev[s + 1].record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    clocks = sampler.stop()
+    ctx.sync()
+    launches = ctx.launch_count() - l0
+    per_launch_ms = [ev[s].elapsed_time(ev[s + 1]) for s in range(args.steps)]
+    total_ms = dist.max_over_ranks(ev[0].elapsed_time(ev[-1]))
+    value = world * samples_per_pass * args.steps / (total_ms * 1e-3)
+    E_final = ctx.eval(0)
+
+    # roofline of the dominant kernel (the persistent worker kernel: one launch per bench step)
+    peak, peak_kind = measured_peaks()
+    launch_ms = statistics.mean(per_launch_ms)
+    bytes_per_launch = algorithmic_bytes_per_pass(wl, steps)
+    achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": None, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "kernel": ctx.path_name(), "launch_ms": launch_ms, "algorithmic_bytes_per_launch": bytes_per_launch}
+
+    # end to end through the host-buffer entry point: H2D of X and w0, the pass, D2H of w^1
+    e2e = None
+    if not args.no_e2e:
+        try:
+            path = ctx.path_name()
+            ctx.destroy()
+            del ctx
+            Xh = torch.empty(X.shape, dtype=torch.float32, pin_memory=True)
+            Xh.copy_(X)
+            w0h = w0.cpu().pin_memory()
+            del X
+            torch.cuda.empty_cache()
+            out = torch.empty((wl.k, wl.d), dtype=torch.float32).pin_memory()
+            scratch = torch.empty(pkg.asgd_fit_host_bytes(cfg) + 256, dtype=torch.uint8, device=dev)
+            off = (-scratch.data_ptr()) % 256
+            pkg.asgd_fit_host(cfg, Xh, w0h, steps, True, out, scratch[off:])       # warm-up
+            dist.barrier()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(args.e2e_steps):
+                pkg.asgd_fit_host(cfg, Xh, w0h, steps, True, out, scratch[off:])   # synchronises itself
+            dt = dist.max_over_ranks(time.perf_counter() - t0)
+            e2e = {"value": world * samples_per_pass * args.e2e_steps / dt, "unit": UNIT,
+                   "h2d_bytes_per_step": int(Xh.numel() * 4 + w0h.numel() * 4), "d2h_bytes_per_step": int(out.numel() * 4),
+                   "steps": args.e2e_steps, "path": path}
+            del scratch, Xh
+        except Exception as exc:      # e.g. not enough pinned host memory on this machine
+            e2e = {"value": None, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0, "error": repr(exc)[:200]}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, desc, th = cpu_baseline(wl, CPU_SAMPLE_ROWS)
+        cpu = {"value": v, "unit": UNIT, "cores": th, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "k": wl.k, "W": wl.W, "b": wl.b, "eps": wl.eps,
+                       "comm_interval": wl.comm_interval, "fanout": wl.fanout, "mode": "free-running",
+                       "steps_per_worker_per_bench_step": steps, "parallelism": "dp%d" % world,
+                       "l2": "inputs larger than L2 (%.2f GB per pass)" % (bytes_per_launch / 1e9)},
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "quantization_error_worker0": E_final,
+        }
+        print(json.dumps(line), flush=True)
+    dist.shutdown()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

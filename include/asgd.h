@@ -48,9 +48,10 @@ typedef enum asgd_status {
 /* Distance paths (a2).  AUTO picks by k and d. */
 enum {
   ASGD_PATH_AUTO = 0,
-  ASGD_PATH_FP32 = 1,       /* CUDA cores, fp32                                              */
+  ASGD_PATH_FP32 = 1,       /* CUDA cores, fp32 (the specialised kernel for the shape, if any) */
   ASGD_PATH_TC_3XTF32 = 2,  /* tcgen05, three TF32 products per fp32 product                 */
-  ASGD_PATH_TC_BF16 = 3     /* tcgen05, BF16 operands, fp32 accumulate                       */
+  ASGD_PATH_TC_BF16 = 3,    /* tcgen05, BF16 operands, fp32 accumulate                       */
+  ASGD_PATH_FP32_GENERAL = 4 /* CUDA cores, fp32, the shape-independent kernel                */
 };
 
 /* Problem statement ASGD(X, T, eps, w0, b) of Algorithm 5 plus the communication parameters. */

@@ -11,12 +11,16 @@
 
 #include "asgd_aux.cuh"
 #include "asgd_generic.cuh"
+#include "asgd_stream.cuh"
 
 using namespace asgd;
 
 namespace {
 
-enum PathId { P_GENERIC = 0 };
+enum PathId { P_GENERIC = 0, P_STREAM = 1 };
+
+// (d, k) shapes the streaming path is compiled for
+#define ASGD_STREAM_SHAPES(X) X(10, 10) X(16, 16) X(4, 5) X(3, 3)
 
 struct Layout {
   size_t state, mail, seq, seen, arb_win, arb_cnt, stats, perm, status, assign_rec, accept_rec, gsum,
@@ -36,7 +40,7 @@ bool config_ok(const asgd_config* c) {
   if (c->comm_interval < 0 || c->fanout < 0 || c->fanout > c->W - 1 || c->fanout > MAX_FANOUT) return false;
   if (c->slots < 1 || c->slots > MAX_SLOTS) return false;
   if (c->reserved != 0) return false;
-  if (c->dist_path < ASGD_PATH_AUTO || c->dist_path > ASGD_PATH_TC_BF16) return false;
+  if (c->dist_path < ASGD_PATH_AUTO || c->dist_path > ASGD_PATH_FP32_GENERAL) return false;
   if ((long long)c->k * c->d > (1ll << 28)) return false;
   const long long H = c->N / c->W;
   if (H < c->b) return false;
@@ -110,9 +114,29 @@ void fill_perm(const asgd_config& c, long long B, int worker, int* perm) {
   }
 }
 
+template <int D, int K>
+int stream_prepare(asgd_ctx* c) {
+  c->smem_bytes = stream_smem_bytes<D, K>(c->cfg.b);
+  CU(c, cudaFuncSetAttribute(asgd_stream_kernel<D, K, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  CU(c, cudaFuncSetAttribute(asgd_stream_kernel<D, K, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  return ASGD_OK;
+}
+template <int D, int K>
+void stream_launch(asgd_ctx* c, bool det, long long steps) {
+  if (det)
+    asgd_stream_kernel<D, K, true><<<c->p.W, STREAM_THREADS, c->smem_bytes, c->stream>>>(c->p, steps);
+  else
+    asgd_stream_kernel<D, K, false><<<c->p.W, STREAM_THREADS, c->smem_bytes, c->stream>>>(c->p, steps);
+}
+
 int launch_workers(asgd_ctx* c, bool det, long long steps) {
   const Params& p = c->p;
   switch (c->path) {
+    case P_STREAM:
+#define X(D_, K_) if (p.d == D_ && p.k == K_) stream_launch<D_, K_>(c, det, steps);
+      ASGD_STREAM_SHAPES(X)
+#undef X
+      break;
     case P_GENERIC:
     default:
       if (det)
@@ -129,6 +153,17 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
 int resolve_path(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
   if (cfg.dist_path == ASGD_PATH_TC_3XTF32 || cfg.dist_path == ASGD_PATH_TC_BF16) return ASGD_EUNSUPPORTED;
+  // streaming path: small state, both ring slots and the state within a quarter of an SM's shared memory
+  if (cfg.dist_path == ASGD_PATH_AUTO || cfg.dist_path == ASGD_PATH_FP32) {
+#define X(D_, K_)                                                                     \
+  if (cfg.d == D_ && cfg.k == K_ && stream_smem_bytes<D_, K_>(cfg.b) <= 56 * 1024) { \
+    c->path = P_STREAM;                                                               \
+    c->state_on_chip = 1;                                                             \
+    return stream_prepare<D_, K_>(c);                                                 \
+  }
+    ASGD_STREAM_SHAPES(X)
+#undef X
+  }
   c->path = P_GENERIC;
   const int kd_pad = c->p.kd_pad;
   size_t on = generic_smem_bytes(cfg.k, cfg.b, kd_pad, true);
@@ -347,6 +382,7 @@ const char* asgd_path_name(const asgd_ctx* c) {
   if (!c) return "none";
   switch (c->path) {
     case P_GENERIC: return c->state_on_chip ? "fp32-generic" : "fp32-generic-offchip";
+    case P_STREAM: return "fp32-stream";
     default: return "unknown";
   }
 }

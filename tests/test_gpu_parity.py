@@ -115,6 +115,12 @@ EDGE_CASES = {
     "fanout_all_peers": dict(N=4000, d=10, k=10, W=5, b=50, comm_interval=1, fanout=4),
     "ragged_rows": dict(N=4003, d=9, k=7, W=7, b=37, comm_interval=3, fanout=2),
     "odd_kd": dict(N=3000, d=3, k=3, W=3, b=97, comm_interval=1, fanout=1),
+    # shapes of the streaming kernel: misaligned batch starts, a batch that ends on X's last row
+    "stream_3x3_to_the_last_row": dict(N=582, d=3, k=3, W=3, b=97, comm_interval=1, fanout=1),
+    "stream_4x5": dict(N=5 * 333 + 2, d=4, k=5, W=5, b=111, comm_interval=2, fanout=2),
+    "stream_16x16": dict(N=6 * 700, d=16, k=16, W=6, b=175, comm_interval=1, fanout=1),
+    "stream_10x10_one_sample": dict(N=40, d=10, k=10, W=4, b=1, comm_interval=1, fanout=1),
+    "stream_10x10_to_the_last_row": dict(N=4 * 33 * 3, d=10, k=10, W=4, b=33, comm_interval=1, fanout=3),
 }
 
 
@@ -131,6 +137,22 @@ def test_edge_cases(case, parzen):
     assert pr.max_rel_l2() < CENTRE_TOL, (case, pr.max_rel_l2())
     _compare_stats(pr, exact_accept=(parzen == 0))
     pr.close()
+
+
+def test_specialised_and_general_kernels_agree():
+    wl = scaled("tiny", N=30_000)
+    a = Pair(wl, oracle=False)
+    g = Pair(wl, oracle=False, dist_path=pkg.PATH_FP32_GENERAL)
+    assert a.gpu.path_name() == "fp32-stream" and g.gpu.path_name() == "fp32-generic"
+    a.gpu.step(60)
+    g.gpu.step(60)
+    assert (a.gpu.get_assign() == g.gpu.get_assign()).all()
+    sa, sg = a.gpu_states().astype(np.float64), g.gpu_states().astype(np.float64)
+    assert np.sqrt(((sa - sg) ** 2).sum()) / np.sqrt((sg ** 2).sum()) < 1e-5
+    for i in range(wl.W):
+        assert a.gpu.get_stats(i) == g.gpu.get_stats(i)
+    a.close()
+    g.close()
 
 
 def test_unshuffled_batches_and_many_slots():
