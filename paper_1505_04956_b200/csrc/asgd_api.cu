@@ -20,7 +20,7 @@ namespace {
 enum PathId { P_GENERIC = 0, P_STREAM = 1 };
 
 // (d, k) shapes the streaming path is compiled for
-#define ASGD_STREAM_SHAPES(X) X(10, 10) X(16, 16) X(4, 5) X(3, 3)
+#define ASGD_STREAM_SHAPES(X) X(10, 10) X(16, 16) X(4, 5) X(2, 3)
 
 struct Layout {
   size_t state, mail, seq, seen, arb_win, arb_cnt, stats, perm, status, assign_rec, accept_rec, gsum,
@@ -153,10 +153,11 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
 int resolve_path(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
   if (cfg.dist_path == ASGD_PATH_TC_3XTF32 || cfg.dist_path == ASGD_PATH_TC_BF16) return ASGD_EUNSUPPORTED;
-  // streaming path: small state, both ring slots and the state within a quarter of an SM's shared memory
+  // streaming path: small state, a mini-batch of at most 4 samples per thread
   if (cfg.dist_path == ASGD_PATH_AUTO || cfg.dist_path == ASGD_PATH_FP32) {
 #define X(D_, K_)                                                                     \
-  if (cfg.d == D_ && cfg.k == K_ && stream_smem_bytes<D_, K_>(cfg.b) <= 56 * 1024) { \
+  if (cfg.d == D_ && cfg.k == K_ && cfg.b <= STREAM_MAX_B &&                         \
+      stream_smem_bytes<D_, K_>(cfg.b) <= 100 * 1024) {                             \
     c->path = P_STREAM;                                                               \
     c->state_on_chip = 1;                                                             \
     return stream_prepare<D_, K_>(c);                                                 \

@@ -56,7 +56,7 @@ constexpr int EVAL_THREADS = 256;
 __global__ void __launch_bounds__(EVAL_THREADS)
 eval_kernel(const float* __restrict__ X, long long N, int d, int k, const float* __restrict__ wg,
             int w_on_chip, double* partial) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   double* red = reinterpret_cast<double*>(smem_raw);
   float* ws = reinterpret_cast<float*>(smem_raw + 32 * sizeof(double));
   const float* w = wg;

@@ -41,7 +41,7 @@ __device__ inline void warp0_exclusive_scan(const int* cnt, int k, int* start) {
 template <bool kDet>
 __global__ void __launch_bounds__(GENERIC_THREADS)
 asgd_generic_kernel(const Params p, const long long steps, const int state_on_chip) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   TailScratch* ts = reinterpret_cast<TailScratch*>(smem_raw);
   unsigned char* cur = smem_raw + sizeof(TailScratch);
   float* w;

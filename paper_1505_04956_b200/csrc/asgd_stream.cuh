@@ -1,15 +1,20 @@
-// Streaming fp32 path for small states (k, d <= 16): the HBM-bound shape of the method.
+// Streaming fp32 path for small states (k <= 16, even d <= 16, b <= 512): the HBM-bound shape.
 //
 // One worker = one 128-thread block, 4 blocks per SM.  The worker's mini-batches are pulled into a
 // two-slot shared-memory ring with bulk asynchronous copies (one elected thread issues them, an
 // mbarrier per slot counts the bytes), so the next batch streams in while the current one is used.
-// Assignment: one thread per sample, expanded form  score_a = ||w_a||^2 - 2 x.w_a  (exactly k*d
-// FMAs), with the centre index packed into the low mantissa bits so that min/max instructions carry
-// the argmin; a sample whose two best scores are closer than the rounding bound of that form is
-// decided again in the direct difference form.  Per-centre sums: lanes of a warp that share a centre
-// add their rows with a pointer-jumping shuffle reduction, the group's first lane adds the result
-// to the warp's private accumulators in shared memory.  The order of every sum is fixed by sample
-// position, so a step is reproducible.
+//
+// Assignment (Eq. 8): a warp owns 128 consecutive rows of the batch, a thread 4 of them (row =
+// 32*q + lane of the warp's block).  Scores use the expanded form  ||w_a||^2 - 2 x.w_a  with packed
+// two-wide FMAs (even and odd dimensions accumulate in the two halves).  The centre index rides in
+// the low mantissa bits so that min/max instructions carry the argmin and the runner-up; a sample
+// whose two best scores are closer than the rounding bound of this form is decided again in the
+// direct difference form.
+//
+// Per-centre sums (Eq. 9): for each of its four 32-row blocks a warp lists the lanes that chose each
+// centre (rank inside the block from a match, so a list is in row order); then lane (block, centre)
+// adds the listed rows from the shared-memory tile.  Every sum has a fixed order, so a step is
+// reproducible.  The plain local step needs two block-wide barriers.
 #pragma once
 
 #include "asgd_step_tail.cuh"
@@ -19,7 +24,11 @@ namespace asgd {
 constexpr int STREAM_THREADS = 128;
 constexpr int STREAM_WARPS = STREAM_THREADS / 32;
 constexpr int STREAM_STAGES = 2;
-constexpr unsigned STREAM_WAIT_LIMIT = 1u << 22;   // bounded mbarrier wait (iterations of try_wait)
+constexpr int STREAM_SPT = 4;                          // samples per thread = 32-row blocks per warp
+constexpr int STREAM_MAX_B = STREAM_THREADS * STREAM_SPT;
+constexpr int STREAM_WARP_SAMPLES = 32 * STREAM_SPT;
+constexpr int STREAM_PARTS = STREAM_WARPS * STREAM_SPT;   // partial sums per centre
+constexpr unsigned STREAM_WAIT_LIMIT = 1u << 22;       // bounded mbarrier wait (iterations of try_wait)
 
 __device__ inline unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 __device__ inline void mbar_init(unsigned long long* bar, unsigned count) {
@@ -46,96 +55,95 @@ __device__ inline void bulk_g2s(void* dst, const void* src, unsigned bytes, unsi
                ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 __device__ inline void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ inline unsigned ld_relaxed_gpu(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 
 template <int D, int K>
 struct StreamLayout {
+  static_assert(D % 2 == 0 && D <= 16 && K <= 16, "streaming path: even d <= 16, k <= 16");
   static constexpr int DP = (D + 3) / 4 * 4;        // padded row of -2w for 128-bit loads
-  static constexpr int SP = D + 1;                  // row stride of the per-warp accumulators
+  static constexpr int D2 = D / 2;                  // dimension pairs
   static constexpr int INDEX_BITS = (K <= 2) ? 1 : (K <= 4) ? 2 : (K <= 8) ? 3 : 4;
   static constexpr unsigned INDEX_MASK = (1u << INDEX_BITS) - 1u;
+  static constexpr int CPW = 32 / D;                // centres a warp updates at a time
+  static constexpr int LISTS = STREAM_SPT * K;      // lists per warp: (32-row block, centre)
 };
-
-inline size_t stream_slot_bytes(int b, int d) { return ((size_t)b * d * 4 + 32 + 127) / 128 * 128; }
 
 // Shared-memory map of the streaming kernel (byte offsets, every region 16-byte aligned).
 template <int D, int K>
 struct StreamSmem {
   using L = StreamLayout<D, K>;
-  size_t ring, bars, flags, tail, wneg2, cnorm, w, sd, sw, cw, cnt, total;
+  size_t ring, bars, flags, zero, tail, wneg2, cnorm, w, sd, sw, cw, cnt, seen, lists, total;
   __host__ __device__ explicit StreamSmem(int b) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) / 16 * 16; return o; };
     ring = take(STREAM_STAGES * (((size_t)b * D * 4 + 32 + 127) / 128 * 128));
     bars = take(64);
     flags = take(64);
+    zero = take(64);                                            // a row of zeros
     tail = take(sizeof(TailScratch));
     wneg2 = take((size_t)K * L::DP * 4);
-    cnorm = take((size_t)K * 4);
+    cnorm = take((size_t)K * 8);                                // (||w_a||^2, 0) pairs
     w = take((size_t)K * D * 4);
     sd = take((size_t)K * D * 4);
-    sw = take((size_t)STREAM_WARPS * K * L::SP * 4);
-    cw = take((size_t)STREAM_WARPS * K * 4);
+    sw = take((size_t)STREAM_PARTS * K * D * 4);                // partial sums
+    cw = take((size_t)STREAM_WARPS * L::LISTS * 4);             // list lengths
     cnt = take((size_t)K * 4);
+    seen = take((size_t)MAX_SLOTS * 4);
+    lists = take((size_t)STREAM_WARPS * L::LISTS * 32);         // u8 lane numbers
     total = (off + 127) / 128 * 128;
   }
 };
 template <int D, int K>
 inline size_t stream_smem_bytes(int b) { return StreamSmem<D, K>(b).total; }
 
-// Squared distances of one sample in the direct difference form; strict "<" keeps the lowest index.
-template <int D, int K>
-__device__ inline int direct_argmin(const float (&x)[D], const float* wneg2, int DP) {
-  int best = 0;
-  float bd = __int_as_float(0x7f800000);
-#pragma unroll
-  for (int a = 0; a < K; ++a) {
-    float s = 0.f;
-#pragma unroll
-    for (int j = 0; j < D; ++j) {
-      const float df = x[j] + 0.5f * wneg2[a * DP + j];     // -0.5 * (-2w) = w, exact
-      s = fmaf(df, df, s);
-    }
-    if (s < bd) { bd = s; best = a; }
-  }
-  return best;
-}
-
 template <int D, int K, bool kDet>
 __global__ void __launch_bounds__(STREAM_THREADS, 4)
 asgd_stream_kernel(const Params p, const long long steps) {
   using L = StreamLayout<D, K>;
-  constexpr int DP = L::DP, SP = L::SP, KD = K * D;
+  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, LISTS = L::LISTS;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int b = p.b;
-  const size_t slot_bytes = ((size_t)b * D * 4 + 32 + 127) / 128 * 128;
+  const unsigned slot_bytes = ((unsigned)b * D * 4 + 32 + 127) / 128 * 128;
   const StreamSmem<D, K> map(b);
   unsigned char* ring = smem_raw + map.ring;
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + map.bars);   // [STAGES]
-  int* flags = reinterpret_cast<int*>(smem_raw + map.flags);                               // [0] any fresh buffer
+  int* flags = reinterpret_cast<int*>(smem_raw + map.flags);                               // [0] a buffer has news
+  const float* zero_row = reinterpret_cast<const float*>(smem_raw + map.zero);
   TailScratch* ts = reinterpret_cast<TailScratch*>(smem_raw + map.tail);
   float* wneg2 = reinterpret_cast<float*>(smem_raw + map.wneg2);
-  float* cnorm = reinterpret_cast<float*>(smem_raw + map.cnorm);
+  float2* cnorm = reinterpret_cast<float2*>(smem_raw + map.cnorm);
   float* w = reinterpret_cast<float*>(smem_raw + map.w);
   float* SD = reinterpret_cast<float*>(smem_raw + map.sd);
   float* Sw = reinterpret_cast<float*>(smem_raw + map.sw);
   int* Cw = reinterpret_cast<int*>(smem_raw + map.cw);
   int* cnt = reinterpret_cast<int*>(smem_raw + map.cnt);
+  unsigned* seen_s = reinterpret_cast<unsigned*>(smem_raw + map.seen);
+  unsigned char* lists = smem_raw + map.lists;
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int i = blockIdx.x;
   float* wglob = p.state + (size_t)i * p.kd_pad;
-  const float* Xend = p.X + (size_t)p.N * D;
+  const unsigned char* Xend = reinterpret_cast<const unsigned char*>(p.X + (size_t)p.N * D);
+  const unsigned char* shard = reinterpret_cast<const unsigned char*>(p.X + (size_t)i * p.H * D);
+  const unsigned batch_bytes = (unsigned)b * D * 4;
+  const float inv_b = 1.0f / (float)b;
+  const float eps = p.eps;
 
-  // state on chip: w, -2w (padded rows), ||w_a||^2
+  // state on chip: w, -2w (padded rows), (||w_a||^2, 0)
   for (int e = tid; e < K * DP; e += STREAM_THREADS) wneg2[e] = 0.f;
+  if (tid < 16) reinterpret_cast<float*>(smem_raw + map.zero)[tid] = 0.f;
   __syncthreads();
   for (int e = tid; e < KD; e += STREAM_THREADS) {
     const float v = wglob[e];
     w[e] = v;
     wneg2[(e / D) * DP + (e % D)] = -2.f * v;
   }
-  for (int e = tid; e < STREAM_WARPS * K * SP; e += STREAM_THREADS) Sw[e] = 0.f;
-  for (int e = tid; e < STREAM_WARPS * K; e += STREAM_THREADS) Cw[e] = 0;
+  if (tid < K) cnt[tid] = 0;
+  if (tid < p.S) seen_s[tid] = p.seen[(size_t)i * p.S + tid];
   if (tid == 0) {
     for (int q = 0; q < STREAM_STAGES; ++q) mbar_init(bars + q, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -146,27 +154,29 @@ asgd_stream_kernel(const Params p, const long long steps) {
     float s = 0.f;
 #pragma unroll
     for (int j = 0; j < D; ++j) s = fmaf(w[tid * D + j], w[tid * D + j], s);
-    cnorm[tid] = s;
+    cnorm[tid] = make_float2(s, 0.f);
   }
 
   unsigned long long t = p.stats[(size_t)i * ST_STRIDE + ST_STEPS];
+  // 32-bit running positions: place in the batch order, steps left until the next put
+  const int* myperm = p.perm + (size_t)i * p.B;
+  const int nB = (int)p.B;
+  const int pos = (int)(t % (unsigned long long)p.B);
+  const bool puts_on = p.c > 0 && p.f > 0 && p.W > 1;
+  int to_put = puts_on ? p.c - (int)(t % (unsigned long long)p.c) : 0x7fffffff;   // a put is due at 1
+  auto next_pos = [&](int q) { return q + 1 == nB ? 0 : q + 1; };
 
   // a batch's copy: source rounded down to 16 bytes, size rounded up; `head` = bytes to skip
-  const int* myperm = p.perm + (size_t)i * p.B;
-  auto tile_src = [&](long long batch, unsigned& head, unsigned& bytes) -> const unsigned char* {
-    const unsigned char* src = reinterpret_cast<const unsigned char*>(p.X + ((size_t)i * p.H + (size_t)batch * b) * D);
+  auto tile_src = [&](int batch, unsigned& head, unsigned& bytes) -> const unsigned char* {
+    const unsigned char* src = shard + (size_t)batch * batch_bytes;
     head = (unsigned)((uintptr_t)src & 15);
-    bytes = (head + (unsigned)b * D * 4 + 15u) & ~15u;
+    bytes = (head + batch_bytes + 15u) & ~15u;
     return src - head;
   };
-  // true when the rounded copy stays inside X (else the tile is fetched with plain loads)
-  auto tile_bulk_ok = [&](const unsigned char* src, unsigned bytes) {
-    return src + bytes <= reinterpret_cast<const unsigned char*>(Xend);
-  };
-  auto issue = [&](long long batch, int slot) {
+  auto issue = [&](int batch, int slot) {
     unsigned head, bytes;
     const unsigned char* src = tile_src(batch, head, bytes);
-    if (tile_bulk_ok(src, bytes)) {
+    if (src + bytes <= Xend) {
       mbar_expect_tx(bars + slot, bytes);
       bulk_g2s(ring + (size_t)slot * slot_bytes, src, bytes, bars + slot);
     } else {
@@ -175,33 +185,36 @@ asgd_stream_kernel(const Params p, const long long steps) {
   };
 
   // batch indices are read one step ahead so that no step waits on that load
-  long long batch_cur = myperm[t % (unsigned long long)p.B];
-  long long batch_nxt = myperm[(t + 1) % (unsigned long long)p.B];
+  int pos1 = next_pos(pos);
+  int batch_cur = myperm[pos];
+  int batch_nxt = myperm[pos1];
   if (tid == 0 && steps > 0) issue(batch_cur, 0);
   __syncthreads();
 
+  const float tau_scale = (float)(4 * D + 72) * 5.9604645e-8f;
+  int* myCw = Cw + wid * LISTS;
+  unsigned char* myLists = lists + (size_t)wid * (LISTS * 32);
   int abort = 0;
   for (long long step = 0; step < steps; ++step, ++t) {
     const int slot = (int)(step & 1);
     const unsigned parity = (unsigned)((step >> 1) & 1);
 
-    // thread 0: look at the receive buffers' sequence numbers early, start the next batch's copy
-    if (tid == 0) {
-      int any = 0;
-      for (int s = 0; s < p.S; ++s) any |= (ld_acquire_gpu(p.seq + (size_t)i * p.S + s) != p.seen[(size_t)i * p.S + s]);
-      flags[0] = any;
-      if (step + 1 < steps) {
-        fence_proxy_async_smem();
-        issue(batch_nxt, slot ^ 1);
-      }
+    // start the next batch's copy; peek at the receive buffers' sequence numbers (used after the sums)
+    if (tid == 0 && step + 1 < steps) {
+      fence_proxy_async_smem();
+      issue(batch_nxt, slot ^ 1);
     }
-    const long long batch_nn = myperm[(t + 2) % (unsigned long long)p.B];
+    unsigned my_seq = 0;
+    if (tid < p.S) my_seq = ld_relaxed_gpu(p.seq + (size_t)i * p.S + tid);
+    const int pos2 = next_pos(pos1);
+    const int batch_nn = myperm[pos2];
+    for (int e = lane; e < LISTS; e += 32) myCw[e] = 0;
 
     unsigned head, bytes;
     const unsigned char* src = tile_src(batch_cur, head, bytes);
     unsigned char* tile = ring + (size_t)slot * slot_bytes;
     if (!mbar_wait_bounded(bars + slot, parity)) abort = 1;
-    if (!tile_bulk_ok(src, bytes)) {
+    if (src + bytes > Xend) {
       // last rows of X: a rounded bulk copy would run past the array, use plain loads
       const float* g = reinterpret_cast<const float*>(src + head);
       float* sdst = reinterpret_cast<float*>(tile + head);
@@ -209,135 +222,178 @@ asgd_stream_kernel(const Params p, const long long steps) {
       __syncthreads();
     }
     const float* xs = reinterpret_cast<const float*>(tile + head);
+    const float* wblk = xs + (size_t)wid * STREAM_WARP_SAMPLES * D;      // this warp's 128 rows
 
-    float cn[K];
+    // ---- Eq. 8: scores of this thread's samples against every centre ----
+    float2 xv[STREAM_SPT][D2];
+    float x2[STREAM_SPT];
+#pragma unroll
+    for (int q = 0; q < STREAM_SPT; ++q) {
+      const int r = min(wid * STREAM_WARP_SAMPLES + q * 32 + lane, b - 1);   // rows past the batch re-read its last row
+      const float2* xrow = reinterpret_cast<const float2*>(xs + (size_t)r * D);
+#pragma unroll
+      for (int jp = 0; jp < D2; ++jp) xv[q][jp] = xrow[jp];
+      float2 n2 = __fmul2_rn(xv[q][0], xv[q][0]);
+#pragma unroll
+      for (int jp = 1; jp < D2; ++jp) n2 = __ffma2_rn(xv[q][jp], xv[q][jp], n2);
+      x2[q] = n2.x + n2.y;
+    }
+    float s1[STREAM_SPT], s2[STREAM_SPT];
+#pragma unroll
+    for (int q = 0; q < STREAM_SPT; ++q) { s1[q] = __int_as_float(0x7f800000); s2[q] = __int_as_float(0x7f800000); }
     float wmax2 = 0.f;
+#pragma unroll 2
+    for (int a = 0; a < K; ++a) {
+      float2 wr[DP / 2];
 #pragma unroll
-    for (int a = 0; a < K; ++a) { cn[a] = cnorm[a]; wmax2 = fmaxf(wmax2, cn[a]); }
-    const float tau_scale = (float)(4 * D + 72) * 5.9604645e-8f;
-
-    for (int base = 0; base < b; base += STREAM_THREADS) {
-      const int s = base + tid;
-      const bool valid = s < b;
-      float x[D];
-      if (valid) {
-        if (D % 2 == 0) {
-#pragma unroll
-          for (int j = 0; j < D; j += 2) {
-            const float2 v = *reinterpret_cast<const float2*>(xs + (size_t)s * D + j);
-            x[j] = v.x; x[j + 1] = v.y;
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < D; ++j) x[j] = xs[(size_t)s * D + j];
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < D; ++j) x[j] = 0.f;
+      for (int j4 = 0; j4 < DP / 4; ++j4) {
+        const float4 v = *reinterpret_cast<const float4*>(wneg2 + a * DP + 4 * j4);
+        wr[2 * j4] = make_float2(v.x, v.y);
+        wr[2 * j4 + 1] = make_float2(v.z, v.w);
       }
-      float x2 = 0.f;
+      const float2 cn = cnorm[a];                       // (||w_a||^2, 0)
+      wmax2 = fmaxf(wmax2, cn.x);
 #pragma unroll
-      for (int j = 0; j < D; ++j) x2 = fmaf(x[j], x[j], x2);
-
-      // Eq. 8 in expanded form; index in the low mantissa bits
-      float s1 = __int_as_float(0x7f800000), s2 = __int_as_float(0x7f800000);
+      for (int q = 0; q < STREAM_SPT; ++q) {
+        float2 acc = cn;
 #pragma unroll
-      for (int a = 0; a < K; ++a) {
-        float acc = cn[a];
-        const float4* wr = reinterpret_cast<const float4*>(wneg2 + a * DP);
-#pragma unroll
-        for (int j4 = 0; j4 < DP / 4; ++j4) {
-          const float4 wv = wr[j4];
-          if (4 * j4 + 0 < D) acc = fmaf(x[4 * j4 + 0 < D ? 4 * j4 + 0 : 0], wv.x, acc);
-          if (4 * j4 + 1 < D) acc = fmaf(x[4 * j4 + 1 < D ? 4 * j4 + 1 : 0], wv.y, acc);
-          if (4 * j4 + 2 < D) acc = fmaf(x[4 * j4 + 2 < D ? 4 * j4 + 2 : 0], wv.z, acc);
-          if (4 * j4 + 3 < D) acc = fmaf(x[4 * j4 + 3 < D ? 4 * j4 + 3 : 0], wv.w, acc);
-        }
-        const float sp = __uint_as_float((__float_as_uint(acc) & ~L::INDEX_MASK) | (unsigned)a);
-        s2 = fmaxf(s1, fminf(s2, sp));
-        s1 = fminf(s1, sp);
+        for (int jp = 0; jp < D2; ++jp) acc = __ffma2_rn(xv[q][jp], wr[jp], acc);
+        const float sc = acc.x + acc.y;
+        const float sp = __uint_as_float((__float_as_uint(sc) & ~L::INDEX_MASK) | (unsigned)a);
+        s2[q] = fmaxf(s1[q], fminf(s2[q], sp));
+        s1[q] = fminf(s1[q], sp);
       }
-      int best = (int)(__float_as_uint(s1) & L::INDEX_MASK);
-      if (K > 1 && (s2 - s1) <= tau_scale * (wmax2 + x2)) best = direct_argmin<D, K>(x, wneg2, DP);
-      if (!valid) best = K;                              // padding lanes form their own group
-      if (valid && p.assign_rec) p.assign_rec[(size_t)i * b + s] = best;
-
-      // Eq. 9: sum the rows of the lanes that chose the same centre (pointer jumping over the
-      // group's lanes in ascending order), then the group's first lane adds to the warp's row
-      const unsigned grp = __match_any_sync(0xffffffffu, best);
-      const unsigned above = grp & ~((2u << lane) - 1u);
-      int nxt = above ? (__ffs(above) - 1) : lane;
-      const bool leader = (grp & ((1u << lane) - 1u)) == 0;
-      const int gsize = __popc(grp);
-      int rounds = 32 - __clz(__reduce_max_sync(0xffffffffu, (unsigned)gsize) - 1);   // ceil(log2(max size))
-      for (int r = 0; r < rounds; ++r) {
-        const bool have = nxt != lane;
-#pragma unroll
-        for (int j = 0; j < D; ++j) {
-          const float o = __shfl_sync(0xffffffffu, x[j], nxt);
-          if (have) x[j] += o;
-        }
-        const int nn = __shfl_sync(0xffffffffu, nxt, nxt);
-        nxt = (!have || nn == nxt) ? lane : nn;
-      }
-      if (leader && best < K) {
-        float* row = Sw + (wid * K + best) * SP;
-#pragma unroll
-        for (int j = 0; j < D; ++j) row[j] += x[j];
-        Cw[wid * K + best] += gsize;
-      }
-      __syncwarp();
     }
 
-    // ---- barrier A: every warp's sums are in shared memory, the slot is free again ----
+    // ---- decide: index from the packed minimum; direct differences when the runner-up is too close ----
+    int best[STREAM_SPT];
+#pragma unroll
+    for (int q = 0; q < STREAM_SPT; ++q) {
+      best[q] = (int)(__float_as_uint(s1[q]) & L::INDEX_MASK);
+      if (K > 1 && (s2[q] - s1[q]) <= tau_scale * (wmax2 + x2[q])) {
+        float bd = __int_as_float(0x7f800000);
+        int bb = 0;
+        for (int a = 0; a < K; ++a) {
+          float acc = 0.f;
+#pragma unroll
+          for (int jp = 0; jp < D2; ++jp) {
+            const float d0 = xv[q][jp].x + 0.5f * wneg2[a * DP + 2 * jp];        // -0.5 * (-2w) = w, exact
+            const float d1 = xv[q][jp].y + 0.5f * wneg2[a * DP + 2 * jp + 1];
+            acc = fmaf(d0, d0, acc);
+            acc = fmaf(d1, d1, acc);
+          }
+          if (acc < bd) { bd = acc; bb = a; }          // strict "<": the lowest index keeps a tie
+        }
+        best[q] = bb;
+      }
+      const int r = wid * STREAM_WARP_SAMPLES + q * 32 + lane;
+      if (r >= b) best[q] = K;                                   // rows past the batch form their own group
+      else if (p.assign_rec) p.assign_rec[(size_t)i * b + r] = best[q];
+    }
+    // ---- lists: per 32-row block, the lanes that chose each centre, in lane order ----
+    __syncwarp();
+#pragma unroll
+    for (int q = 0; q < STREAM_SPT; ++q) {
+      const unsigned grp = __match_any_sync(0xffffffffu, best[q]);
+      const unsigned below = grp & ((1u << lane) - 1u);
+      if (best[q] < K) {
+        myLists[(q * K + best[q]) * 32 + __popc(below)] = (unsigned char)lane;
+        if (below == 0) myCw[q * K + best[q]] = __popc(grp);
+      }
+    }
+    if (tid < p.S && my_seq != seen_s[tid]) flags[0] = 1;
+    __syncwarp();
+
+    // ---- Eq. 9: lane (block, centre) adds its list's rows; up to 8 independent row loads at a time ----
+    for (int l = lane; l < LISTS; l += 32) {
+      const int q = l / K, a = l % K;
+      const int n = myCw[l];
+      const float* blk = wblk + (size_t)q * 32 * D;
+      const uint2* ent = reinterpret_cast<const uint2*>(myLists + l * 32);
+      float2 acc[D2];
+#pragma unroll
+      for (int jp = 0; jp < D2; ++jp) acc[jp] = make_float2(0.f, 0.f);
+      const int nmax = (int)__reduce_max_sync(__activemask(), (unsigned)n);
+      for (int e0 = 0; e0 < nmax; e0 += 8) {
+        const uint2 pk = ent[e0 >> 3];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const unsigned word = (u < 4) ? pk.x : pk.y;
+          const int li = (int)((word >> (8 * (u & 3))) & 0xffu);
+          const float2* row = reinterpret_cast<const float2*>((e0 + u < n) ? blk + li * D : zero_row);
+#pragma unroll
+          for (int jp = 0; jp < D2; ++jp) acc[jp] = __fadd2_rn(acc[jp], row[jp]);
+        }
+      }
+      float2* out = reinterpret_cast<float2*>(Sw + (size_t)((wid * STREAM_SPT + q) * K + a) * D);
+#pragma unroll
+      for (int jp = 0; jp < D2; ++jp) out[jp] = acc[jp];
+      if (n) atomicAdd(cnt + a, n);
+    }
+
+    // ---- barrier B: partial sums and counts complete, the ring slot is free again ----
     if (__syncthreads_or(abort)) { abort = 1; break; }
 
-    // per-centre totals and the local gradient (Eq. 9), in place of the generic tail's first loop
-    for (int e = tid; e < KD; e += STREAM_THREADS) {
-      float ssum = 0.f;
-#pragma unroll
-      for (int q = 0; q < STREAM_WARPS; ++q) ssum += Sw[(q * K + e / D) * SP + (e % D)];
-      SD[e] = ssum;
-    }
-    if (tid < K) {
-      int c = 0;
-#pragma unroll
-      for (int q = 0; q < STREAM_WARPS; ++q) c += Cw[q * K + tid];
-      cnt[tid] = c;
-    }
-    __syncthreads();
-    for (int e = tid; e < STREAM_WARPS * K * SP; e += STREAM_THREADS) Sw[e] = 0.f;
-    for (int e = tid; e < STREAM_WARPS * K; e += STREAM_THREADS) Cw[e] = 0;
-
-    const bool put_now = p.c > 0 && p.f > 0 && p.W > 1 && (t + 1) % (unsigned long long)p.c == 0;
-    if (flags[0] || put_now) {
-      // a message is waiting or a put is due: the general tail handles both
-      step_tail<kDet>(p, i, t, w, SD, cnt, wglob, ts);
-    } else {
-      // common case: plain local step  w <- w - eps * D
+    const bool put_now = (to_put == 1);
+    if (flags[0] != 0 || put_now) {
+      // a message is waiting or a put is due: totals into SD, then the general tail handles both
       for (int e = tid; e < KD; e += STREAM_THREADS) {
-        const float ww = w[e];
-        const float Dg = ((float)cnt[e / D] * ww - SD[e]) * (1.0f / (float)b);
-        const float nw = ww - p.eps * Dg;
-        w[e] = nw;
-        wglob[e] = nw;
-      }
-      if (tid == 0) {
-        for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
-        p.stats[(size_t)i * ST_STRIDE + ST_STEPS] = t + 1;
+        float ssum = 0.f;
+#pragma unroll
+        for (int q = 0; q < STREAM_PARTS; ++q) ssum += Sw[(size_t)(q * K + e / D) * D + (e % D)];
+        SD[e] = ssum;
       }
       __syncthreads();
-    }
-    for (int e = tid; e < KD; e += STREAM_THREADS) wneg2[(e / D) * DP + (e % D)] = -2.f * w[e];
-    if (tid < K) {
-      float s = 0.f;
+      step_tail<kDet>(p, i, t, w, SD, cnt, wglob, ts);
+      if (tid < p.S) seen_s[tid] = p.seen[(size_t)i * p.S + tid];
+      if (tid == 0) flags[0] = 0;
+      if (tid < K) cnt[tid] = 0;
+      for (int e = tid; e < KD; e += STREAM_THREADS) wneg2[(e / D) * DP + (e % D)] = -2.f * w[e];
+      if (tid < K) {
+        float s = 0.f;
 #pragma unroll
-      for (int j = 0; j < D; ++j) s = fmaf(w[tid * D + j], w[tid * D + j], s);
-      cnorm[tid] = s;
+        for (int j = 0; j < D; ++j) s = fmaf(w[tid * D + j], w[tid * D + j], s);
+        cnorm[tid] = make_float2(s, 0.f);
+      }
+    } else {
+      // common case: plain local step  w <- w - eps * D,  D = (n_a w - S) / b.  A warp updates CPW
+      // centres at a time, lane = (centre, dimension), and reduces ||w_a||^2 over the centre's lanes.
+      for (int a0 = wid * L::CPW; a0 < K; a0 += STREAM_WARPS * L::CPW) {
+        const int a = a0 + lane / D, j = lane % D;
+        const bool on = (lane < L::CPW * D) && (a < K);
+        float sq = 0.f;
+        if (on) {
+          const int n = cnt[a];
+          float ssum = 0.f;
+#pragma unroll
+          for (int q = 0; q < STREAM_PARTS; ++q) ssum += Sw[(size_t)(q * K + a) * D + j];
+          const float ww = w[a * D + j];
+          const float Dg = ((float)n * ww - ssum) * inv_b;
+          const float nw = ww - eps * Dg;
+          w[a * D + j] = nw;
+          wneg2[a * DP + j] = -2.f * nw;
+          wglob[a * D + j] = nw;
+          sq = nw * nw;
+        }
+#pragma unroll
+        for (int o = 1; o < D; o <<= 1) {
+          const float up = __shfl_down_sync(0xffffffffu, sq, o);
+          if (j + o < D) sq += up;
+        }
+        __syncwarp();
+        if (on && j == 0) { cnorm[a] = make_float2(sq, 0.f); cnt[a] = 0; }
+      }
+      if (tid == 0) {
+        if (kDet)
+          for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
+        p.stats[(size_t)i * ST_STRIDE + ST_STEPS] = t + 1;
+      }
     }
     batch_cur = batch_nxt;
     batch_nxt = batch_nn;
-    __syncthreads();
+    pos1 = pos2;
+    if (puts_on) to_put = (to_put == 1) ? p.c : to_put - 1;
+    __syncthreads();                                   // barrier E: w, -2w, ||w||^2 ready for the next step
   }
 
   if (abort) {

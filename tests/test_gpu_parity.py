@@ -116,11 +116,14 @@ EDGE_CASES = {
     "ragged_rows": dict(N=4003, d=9, k=7, W=7, b=37, comm_interval=3, fanout=2),
     "odd_kd": dict(N=3000, d=3, k=3, W=3, b=97, comm_interval=1, fanout=1),
     # shapes of the streaming kernel: misaligned batch starts, a batch that ends on X's last row
-    "stream_3x3_to_the_last_row": dict(N=582, d=3, k=3, W=3, b=97, comm_interval=1, fanout=1),
+    "stream_2x3_to_the_last_row": dict(N=582, d=2, k=3, W=3, b=97, comm_interval=1, fanout=1),
     "stream_4x5": dict(N=5 * 333 + 2, d=4, k=5, W=5, b=111, comm_interval=2, fanout=2),
     "stream_16x16": dict(N=6 * 700, d=16, k=16, W=6, b=175, comm_interval=1, fanout=1),
     "stream_10x10_one_sample": dict(N=40, d=10, k=10, W=4, b=1, comm_interval=1, fanout=1),
     "stream_10x10_to_the_last_row": dict(N=4 * 33 * 3, d=10, k=10, W=4, b=33, comm_interval=1, fanout=3),
+    "stream_10x10_full_block": dict(N=3 * 512 * 3 + 7, d=10, k=10, W=3, b=512, comm_interval=2, fanout=1),
+    "stream_10x10_odd_batch": dict(N=3 * 129 * 5, d=10, k=10, W=3, b=129, comm_interval=2, fanout=1),
+    "general_10x10_big_batch": dict(N=2 * 700 * 3, d=10, k=10, W=2, b=700, comm_interval=2, fanout=1),
 }
 
 
