@@ -155,6 +155,41 @@ int asgd_fit_host(const asgd_config *cfg, const float *X_host, const float *w0_h
                   int64_t steps_per_worker, int32_t mode_async, float *w_out_host,
                   void *scratch_dev, size_t scratch_bytes, void *cuda_stream);
 
+/*
+ * E(w) of Eq. 8 for callers that must not allocate device memory.  (The paper has no counterpart
+ * to this entry point; it exists for the sake of the caller, not of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a latency-critical serving
+ * loop whose memory was carved up at start-up, under a framework's caching allocator whose pool the
+ * caller may not grow, or in a process whose device memory is fully budgeted to someone else.  Such
+ * a caller can own X, w and one double for the result, but cannot hand the library a workspace, so
+ * asgd_eval() (which keeps its per-block partial sums in the context's workspace) is closed to it.
+ * Here the partial sums live in a fixed array compiled into the library:
+ * ASGD_EVAL_NOALLOC_MAX_BLOCKS doubles (32 KB) on every GPU that loads the library, until exit.
+ *
+ *   X_dev   DEVICE [N*d] fp32 row-major (input)       w_dev  DEVICE [k*d] fp32 (input)
+ *   E_dev   DEVICE, one double (output): sum over rows of 1/2 min_k ||x - w_k||^2
+ *
+ * Limits: N <= ASGD_EVAL_NOALLOC_MAX_BLOCKS * ASGD_EVAL_NOALLOC_ROWS_PER_BLOCK (2^28 rows) and
+ * k*d <= ASGD_EVAL_NOALLOC_MAX_KD (the centres are kept in shared memory); anything larger returns
+ * ASGD_EUNSUPPORTED and launches nothing.  Rows are summed in blocks of a fixed size and the blocks
+ * in ascending order, so the value does not depend on the GPU's size.
+ *
+ * The call enqueues two kernels on `cuda_stream` and returns; it calls no cudaMalloc, no cudaFree
+ * and no allocating routine of any library.  The first call on each device also looks up the
+ * array's device address (cudaGetSymbolAddress) and raises the kernel's shared-memory limit, with
+ * that device current; make that first call before starting any stream capture.
+ *
+ * All calls on a device share the one array.  Nothing in it has to start at zero (a call writes
+ * every entry it later reads), but two calls that overlap on the GPU -- different streams, or
+ * different host threads -- race on it: keep calls on one device in stream order.
+ */
+#define ASGD_EVAL_NOALLOC_ROWS_PER_BLOCK 65536
+#define ASGD_EVAL_NOALLOC_MAX_BLOCKS 4096
+#define ASGD_EVAL_NOALLOC_MAX_KD 40960
+int asgd_eval_noalloc(const float *X_dev, int64_t N, int32_t d, int32_t k, const float *w_dev,
+                      double *E_dev, void *cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

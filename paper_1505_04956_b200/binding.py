@@ -18,7 +18,7 @@ EXPORTS = (
     "asgd_workspace_bytes", "asgd_init", "asgd_step", "asgd_run", "asgd_get_state", "asgd_set_state",
     "asgd_put", "asgd_eval", "asgd_get_stats", "asgd_get_assign", "asgd_get_accept", "asgd_sync",
     "asgd_launch_count", "asgd_path_name", "asgd_last_cuda_error", "asgd_strerror", "asgd_destroy",
-    "asgd_fit_host_bytes", "asgd_fit_host",
+    "asgd_fit_host_bytes", "asgd_fit_host", "asgd_eval_noalloc",
 )
 
 
@@ -78,6 +78,7 @@ def load():
     L.asgd_destroy.restype = None
     L.asgd_fit_host_bytes.argtypes = [cfgp, C.POINTER(sz)]
     L.asgd_fit_host.argtypes = [cfgp, vp, vp, i64, i32, vp, vp, sz, vp]
+    L.asgd_eval_noalloc.argtypes = [vp, i64, i32, i32, vp, vp, vp]
     _lib = L
     return L
 
@@ -123,6 +124,16 @@ def asgd_fit_host(cfg: AsgdConfig, X_host, w0_host, steps_per_worker: int, mode_
                               C.c_void_p(scratch_dev.data_ptr()), scratch_dev.numel(), _stream_handle(stream))
     if rc != ASGD_OK:
         raise AsgdError(rc, "asgd_fit_host")
+
+
+def asgd_eval_noalloc(X, w, E_out, stream=None) -> int:
+    """E(w) over the rows of X into the one-element float64 CUDA tensor `E_out`, using only the
+    library's built-in scratch array (for callers that may not allocate device memory).  Returns the
+    status code instead of raising, so that a caller can probe the size limits."""
+    n, d = X.shape
+    return int(load().asgd_eval_noalloc(C.c_void_p(X.data_ptr()), int(n), int(d), int(w.shape[0]),
+                                        C.c_void_p(w.data_ptr()), C.c_void_p(E_out.data_ptr()),
+                                        _stream_handle(stream)))
 
 
 class Asgd:
