@@ -25,6 +25,10 @@ METRIC = "K-Means ASGD samples/s"
 UNIT = "samples/s"
 CPU_SAMPLE_ROWS = 1 << 25          # prefix of the workload the CPU baseline runs on
 NOMINAL_HBM_GBS = 8000.0
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the stream kernel per algorithmic byte, from one ncu
+# capture of a 2^24-row case (profiles/asgd_stream_kernel__stream_workload.md); it grows in proportion to the rows
+# a launch processes.  Valid only for the kernel source it was taken on (first 12 hex digits of its SHA-1).
+TRAFFIC_CAPTURE = {"kernel_sha1": "3a2112266150", "traffic_per_algorithmic_byte": 670.90 / 663.51}
 
 
 def env_int(name, default):
@@ -228,8 +232,13 @@ def main():
     launch_ms = statistics.mean(per_launch_ms)
     bytes_per_launch = algorithmic_bytes_per_pass(wl, steps)
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    traffic = None
+    with open(os.path.join(ROOT, "paper_1505_04956_b200", "csrc", "asgd_stream.cuh"), "rb") as f:
+        import hashlib
+        if ctx.path_name() == "fp32-stream" and hashlib.sha1(f.read()).hexdigest()[:12] == TRAFFIC_CAPTURE["kernel_sha1"]:
+            traffic = bytes_per_launch * TRAFFIC_CAPTURE["traffic_per_algorithmic_byte"]
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "traffic": traffic, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "kernel": ctx.path_name(), "launch_ms": launch_ms, "algorithmic_bytes_per_launch": bytes_per_launch}
 
     # end to end through the host-buffer entry point: H2D of X and w0, the pass, D2H of w^1
