@@ -12,15 +12,20 @@
 #include "asgd_aux.cuh"
 #include "asgd_generic.cuh"
 #include "asgd_stream.cuh"
+#include "asgd_tiled.cuh"
 
 using namespace asgd;
 
 namespace {
 
-enum PathId { P_GENERIC = 0, P_STREAM = 1 };
+enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2 };
 
 // (d, k) shapes the streaming path is compiled for
 #define ASGD_STREAM_SHAPES(X) X(10, 10) X(16, 16) X(4, 5) X(2, 3)
+
+// (d, padded k, warps along samples, warps along centres, blocks per SM) the tiled path is compiled for;
+// the first shape with the same d and enough centres is taken
+#define ASGD_TILED_SHAPES(X) X(32, 64, 4, 2, 2) X(128, 128, 4, 4, 1)
 
 struct Layout {
   size_t state, mail, seq, seen, arb_win, arb_cnt, stats, perm, status, assign_rec, accept_rec, gsum,
@@ -84,6 +89,7 @@ struct asgd_ctx {
   cudaStream_t stream;
   int path;
   int state_on_chip;
+  int grid;               // blocks of the worker kernel (tiled path: a block may serve several workers)
   size_t smem_bytes;
   long long t_host;       // steps every worker has done (uniform across workers)
   long long launches;
@@ -129,9 +135,38 @@ void stream_launch(asgd_ctx* c, bool det, long long steps) {
     asgd_stream_kernel<D, K, false><<<c->p.W, STREAM_THREADS, c->smem_bytes, c->stream>>>(c->p, steps);
 }
 
+template <int D, int KP, int WS, int WK, int MINB>
+int tiled_prepare(asgd_ctx* c) {
+  c->smem_bytes = tiled_smem_bytes<D, KP, WS, WK>(c->cfg.k);
+  CU(c, cudaFuncSetAttribute(asgd_tiled_kernel<D, KP, WS, WK, MINB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  CU(c, cudaFuncSetAttribute(asgd_tiled_kernel<D, KP, WS, WK, MINB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  int per_sm = 0;
+  CU(c, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, asgd_tiled_kernel<D, KP, WS, WK, MINB, false>, 32 * WS * WK, c->smem_bytes));
+  if (per_sm < 1) return ASGD_EUNSUPPORTED;
+  const int resident = per_sm * c->sm_count;
+  const int V = (c->cfg.W + resident - 1) / resident;          // workers per block, served in turn
+  if (V > TILED_MAX_V) return ASGD_EUNSUPPORTED;
+  c->grid = (c->cfg.W + V - 1) / V;
+  return ASGD_OK;
+}
+template <int D, int KP, int WS, int WK, int MINB>
+void tiled_launch(asgd_ctx* c, bool det, long long steps) {
+  if (det)
+    asgd_tiled_kernel<D, KP, WS, WK, MINB, true><<<c->grid, 32 * WS * WK, c->smem_bytes, c->stream>>>(c->p, steps);
+  else
+    asgd_tiled_kernel<D, KP, WS, WK, MINB, false><<<c->grid, 32 * WS * WK, c->smem_bytes, c->stream>>>(c->p, steps);
+}
+
 int launch_workers(asgd_ctx* c, bool det, long long steps) {
   const Params& p = c->p;
   switch (c->path) {
+    case P_TILED: {
+      bool done = false;
+#define X(D_, KP_, WS_, WK_, MB_) if (!done && p.d == D_ && p.k <= KP_) { tiled_launch<D_, KP_, WS_, WK_, MB_>(c, det, steps); done = true; }
+      ASGD_TILED_SHAPES(X)
+#undef X
+      break;
+    }
     case P_STREAM:
 #define X(D_, K_) if (p.d == D_ && p.k == K_) stream_launch<D_, K_>(c, det, steps);
       ASGD_STREAM_SHAPES(X)
@@ -163,6 +198,16 @@ int resolve_path(asgd_ctx* c) {
     return stream_prepare<D_, K_>(c);                                                 \
   }
     ASGD_STREAM_SHAPES(X)
+#undef X
+  }
+  if (cfg.dist_path == ASGD_PATH_AUTO || cfg.dist_path == ASGD_PATH_FP32) {
+#define X(D_, KP_, WS_, WK_, MB_)                                                                  \
+  if (cfg.d == D_ && cfg.k <= KP_ && tiled_smem_bytes<D_, KP_, WS_, WK_>(cfg.k) <= kMaxDynSmem) { \
+    c->path = P_TILED;                                                                             \
+    c->state_on_chip = 0;                                                                          \
+    return tiled_prepare<D_, KP_, WS_, WK_, MB_>(c);                                               \
+  }
+    ASGD_TILED_SHAPES(X)
 #undef X
   }
   c->path = P_GENERIC;
@@ -384,6 +429,7 @@ const char* asgd_path_name(const asgd_ctx* c) {
   switch (c->path) {
     case P_GENERIC: return c->state_on_chip ? "fp32-generic" : "fp32-generic-offchip";
     case P_STREAM: return "fp32-stream";
+    case P_TILED: return "fp32-tiled";
     default: return "unknown";
   }
 }

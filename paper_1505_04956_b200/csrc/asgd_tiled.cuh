@@ -1,0 +1,325 @@
+// Register-tiled fp32 path for mid-size states (k <= KP, d = D, -2w resident in shared memory):
+// the shapes that are bound by the fp32 pipe, not by HBM.
+//
+// A thread block serves one or more workers in turn (worker = blockIdx.x + v * gridDim.x): a step
+// loads the worker's state from HBM/L2, streams the mini-batch through a two-slot ring of sample
+// tiles (one bulk copy per row; rows and centres are padded by 4 floats so that the rows a warp
+// reads at once fall in different banks), and writes the state back through the shared step tail.
+//
+// Assignment (Eq. 8): the tile's scores  ||w_a||^2 - 2 x.w_a  are a small GEMM.  A warp covers
+// 16 samples x 32 centres, a lane 4 x 4 of them (interleaved: rows sg + 4*m, centres cg + 8*i):
+// per four dimensions it reads four 128-bit pieces of x rows and four of -2w rows and issues 64
+// FMAs.  The centre index rides in the low mantissa bits; minimum and runner-up are reduced over
+// the lanes and warps that share a sample; a sample whose two best scores are closer than the
+// rounding bound of this form is decided again by a warp with direct differences in fp64.
+//
+// Per-centre sums (Eq. 9): every warp owns the centres a = warp (mod warps); it finds the tile's
+// rows of a centre with ballots and adds them, lane = dimension, into the centre's row of S in
+// shared memory.  The order of every sum is fixed by row position.
+#pragma once
+
+#include "asgd_step_tail.cuh"
+#include "asgd_stream.cuh"   // bulk-copy and mbarrier helpers
+
+namespace asgd {
+
+constexpr int TILED_MAX_V = 32;     // workers one block can serve
+
+template <int D, int KP, int WS, int WK>
+struct TiledShape {
+  static_assert(D % 32 == 0 && KP % 32 == 0 && KP == 32 * WK, "tiled path: d a multiple of 32, KP = 32 * WK");
+  static constexpr int THREADS = 32 * WS * WK;
+  static constexpr int WARPS = WS * WK;
+  static constexpr int TS = 16 * WS;              // samples per tile
+  static constexpr int XS = D + 4;                // padded row stride of x tiles and of -2w (floats)
+  static constexpr int INDEX_BITS = (KP <= 32) ? 5 : (KP <= 64) ? 6 : (KP <= 128) ? 7 : 8;
+  static constexpr unsigned INDEX_MASK = (1u << INDEX_BITS) - 1u;
+  static constexpr int DR = D / 32;               // dimensions per lane in the sums
+};
+
+template <int D, int KP, int WS, int WK>
+struct TiledSmem {
+  using T = TiledShape<D, KP, WS, WK>;
+  size_t wR, cn, S, cnt, xt, best, x2, red, flagged, tbase, bars, misc, tail, total;
+  __host__ __device__ explicit TiledSmem(int k) {
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) / 16 * 16; return o; };
+    wR = take((size_t)KP * T::XS * 4);
+    cn = take((size_t)KP * 4);
+    S = take((size_t)k * D * 4);
+    cnt = take((size_t)KP * 4);
+    xt = take((size_t)2 * T::TS * T::XS * 4);
+    best = take((size_t)T::TS * 4);
+    x2 = take((size_t)T::TS * 4);
+    red = take((size_t)WK * T::TS * 8);
+    flagged = take((size_t)(T::TS + 4) * 4);
+    tbase = take((size_t)TILED_MAX_V * 8);
+    bars = take(64);
+    misc = take(64);
+    tail = take(sizeof(TailScratch));
+    total = (off + 127) / 128 * 128;
+  }
+};
+template <int D, int KP, int WS, int WK>
+inline size_t tiled_smem_bytes(int k) { return TiledSmem<D, KP, WS, WK>(k).total; }
+
+template <int D, int KP, int WS, int WK, int MINB, bool kDet>
+__global__ void __launch_bounds__(32 * WS * WK, MINB)
+asgd_tiled_kernel(const Params p, const long long steps) {
+  using T = TiledShape<D, KP, WS, WK>;
+  constexpr int TS = T::TS, XS = T::XS, THREADS = T::THREADS, WARPS = T::WARPS, DR = T::DR;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  const int k = p.k, b = p.b;
+  const TiledSmem<D, KP, WS, WK> map(k);
+  float* wR = reinterpret_cast<float*>(smem_raw + map.wR);          // [KP][XS]  -2 w
+  float* cn = reinterpret_cast<float*>(smem_raw + map.cn);          // [KP]      ||w_a||^2 (+inf for padding)
+  float* S = reinterpret_cast<float*>(smem_raw + map.S);            // [k][D]
+  int* cnt = reinterpret_cast<int*>(smem_raw + map.cnt);            // [KP]
+  float* xt = reinterpret_cast<float*>(smem_raw + map.xt);          // [2][TS][XS]
+  int* best = reinterpret_cast<int*>(smem_raw + map.best);          // [TS]
+  float* x2s = reinterpret_cast<float*>(smem_raw + map.x2);         // [TS]
+  float2* red = reinterpret_cast<float2*>(smem_raw + map.red);      // [WK][TS] (minimum, runner-up)
+  int* flagged = reinterpret_cast<int*>(smem_raw + map.flagged);    // [0] count, [1..] tile rows to decide again
+  unsigned long long* tbase = reinterpret_cast<unsigned long long*>(smem_raw + map.tbase);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + map.bars);
+  float* misc = reinterpret_cast<float*>(smem_raw + map.misc);      // [0] max_a ||w_a||^2
+  TailScratch* ts = reinterpret_cast<TailScratch*>(smem_raw + map.tail);
+
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int wk = wid % WK, wsi = wid / WK;        // the warp's centre block and sample block
+  const int cg = lane & 7, sg = lane >> 3;        // the lane's centres cg + 8*i and rows sg + 4*m of the warp tile
+  const int tiles = (b + TS - 1) / TS;
+  const float tau_scale = (float)(4 * D + 8 + 4 * (1 << T::INDEX_BITS)) * 5.9604645e-8f;
+  const float INF = __int_as_float(0x7f800000);
+
+  const int G = (int)gridDim.x;
+  const int nv = (p.W - (int)blockIdx.x + G - 1) / G;              // workers of this block
+  if (tid < nv) tbase[tid] = p.stats[(size_t)((int)blockIdx.x + tid * G) * ST_STRIDE + ST_STEPS];
+  if (tid == 0) {
+    mbar_init(bars + 0, 1);
+    mbar_init(bars + 1, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // The launch consumes tiles in the order (step, worker slot, tile of the batch); tile g uses ring slot g & 1.
+  const long long total_tiles = steps * nv * tiles;
+  auto issue_tile = [&](long long g) {            // called by all lanes of warp 0
+    const int tl = (int)(g % tiles);
+    const long long sv = g / tiles;
+    const int v = (int)(sv % nv);
+    const int i = (int)blockIdx.x + v * G;
+    const unsigned long long t = tbase[v] + (unsigned long long)(sv / nv);
+    const long long batch = p.perm[(size_t)i * p.B + (size_t)(t % (unsigned long long)p.B)];
+    const int rows = min(TS, b - tl * TS);
+    const int slot = (int)(g & 1);
+    float* dst = xt + (size_t)slot * TS * XS;
+    const float* src = p.X + ((size_t)i * p.H + (size_t)batch * b + (size_t)tl * TS) * D;
+    if (lane == 0) mbar_expect_tx(bars + slot, (unsigned)rows * D * 4);
+    __syncwarp();
+    for (int r = lane; r < rows; r += 32) bulk_g2s(dst + (size_t)r * XS, src + (size_t)r * D, D * 4, bars + slot);
+  };
+  if (wid == 0 && total_tiles > 0) issue_tile(0);
+
+  int abort = 0;
+  long long g = 0;
+  for (long long st = 0; st < steps && !abort; ++st) {
+    for (int v = 0; v < nv && !abort; ++v) {
+      const int i = (int)blockIdx.x + v * G;
+      const unsigned long long t = tbase[v] + (unsigned long long)st;
+      float* wglob = p.state + (size_t)i * p.kd_pad;
+
+      // ---- the worker's state: -2w rows, ||w_a||^2, empty sums ----
+      for (int e = tid; e < KP * (D / 4); e += THREADS) {
+        const int a = e / (D / 4), j4 = e % (D / 4);
+        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (a < k) {
+          v4 = *reinterpret_cast<const float4*>(wglob + (size_t)a * D + 4 * j4);
+          v4.x *= -2.f; v4.y *= -2.f; v4.z *= -2.f; v4.w *= -2.f;
+        }
+        *reinterpret_cast<float4*>(wR + (size_t)a * XS + 4 * j4) = v4;
+      }
+      for (int e = tid; e < k * D; e += THREADS) S[e] = 0.f;
+      for (int e = tid; e < KP; e += THREADS) cnt[e] = 0;
+      __syncthreads();
+      for (int a = wid; a < KP; a += WARPS) {
+        float s = 0.f;
+#pragma unroll
+        for (int q = 0; q < DR; ++q) { const float u = wR[(size_t)a * XS + lane + 32 * q]; s = fmaf(u, u, s); }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) cn[a] = (a < k) ? 0.25f * s : INF;
+      }
+      __syncthreads();
+      if (wid == 0) {
+        float m = 0.f;
+        for (int a = lane; a < k; a += 32) m = fmaxf(m, cn[a]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) misc[0] = m;
+      }
+
+      for (int tl = 0; tl < tiles; ++tl, ++g) {
+        const int slot = (int)(g & 1);
+        const unsigned parity = (unsigned)((g >> 1) & 1);
+        const int rows = min(TS, b - tl * TS);
+        const float* xb = xt + (size_t)slot * TS * XS;
+        if (wid == 0 && g + 1 < total_tiles) {
+          fence_proxy_async_smem();
+          issue_tile(g + 1);
+        }
+        if (tid == 0) flagged[0] = 0;
+        if (!mbar_wait_bounded(bars + slot, parity)) abort = 1;
+
+        // ---- scores of the warp's 16 x 32 block: acc[m][i] = sum_j x[row m][j] * (-2 w[centre i][j]) ----
+        float acc[4][4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc[m][c] = 0.f;
+        const float* xrow = xb + (size_t)(wsi * 16 + sg) * XS;
+        const float* wrow = wR + (size_t)(wk * 32 + cg) * XS;
+#pragma unroll 2
+        for (int j = 0; j < D; j += 4) {
+          float4 xv[4], wv[4];
+#pragma unroll
+          for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xrow + (size_t)(4 * m) * XS + j);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) wv[c] = *reinterpret_cast<const float4*>(wrow + (size_t)(8 * c) * XS + j);
+#pragma unroll
+          for (int m = 0; m < 4; ++m)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              acc[m][c] = fmaf(xv[m].x, wv[c].x, acc[m][c]);
+              acc[m][c] = fmaf(xv[m].y, wv[c].y, acc[m][c]);
+              acc[m][c] = fmaf(xv[m].z, wv[c].z, acc[m][c]);
+              acc[m][c] = fmaf(xv[m].w, wv[c].w, acc[m][c]);
+            }
+        }
+        // minimum and runner-up over the lane's 4 centres, then over the 8 lanes that share the rows
+        float cnv[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) cnv[c] = cn[wk * 32 + 8 * c + cg];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+          float s1 = INF, s2 = INF;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const float sc = acc[m][c] + cnv[c];
+            const float sp = __uint_as_float((__float_as_uint(sc) & ~T::INDEX_MASK) | (unsigned)(wk * 32 + 8 * c + cg));
+            s2 = fmaxf(s1, fminf(s2, sp));
+            s1 = fminf(s1, sp);
+          }
+#pragma unroll
+          for (int o = 1; o < 8; o <<= 1) {
+            const float o1 = __shfl_xor_sync(0xffffffffu, s1, o);
+            const float o2 = __shfl_xor_sync(0xffffffffu, s2, o);
+            s2 = fminf(fmaxf(s1, o1), fminf(s2, o2));
+            s1 = fminf(s1, o1);
+          }
+          if (cg == 0) red[(size_t)wk * TS + wsi * 16 + 4 * m + sg] = make_float2(s1, s2);
+        }
+        __syncthreads();                                         // (1) red complete
+
+        // ---- one thread per tile row: merge over the centre blocks, decide or flag ----
+        if (tid < TS) {
+          int bst = -1;
+          if (tid < rows) {
+            float s1 = INF, s2 = INF;
+#pragma unroll
+            for (int q = 0; q < WK; ++q) {
+              const float2 r = red[(size_t)q * TS + tid];
+              s2 = fminf(fmaxf(s1, r.x), fminf(s2, r.y));
+              s1 = fminf(s1, r.x);
+            }
+            float xx = 0.f;
+            const float4* xr = reinterpret_cast<const float4*>(xb + (size_t)tid * XS);
+            for (int j4 = 0; j4 < D / 4; ++j4) {
+              const float4 u = xr[j4];
+              xx = fmaf(u.x, u.x, xx); xx = fmaf(u.y, u.y, xx); xx = fmaf(u.z, u.z, xx); xx = fmaf(u.w, u.w, xx);
+            }
+            bst = (int)(__float_as_uint(s1) & T::INDEX_MASK);
+            if (k > 1 && (s2 - s1) <= tau_scale * (misc[0] + xx)) flagged[1 + atomicAdd(flagged, 1)] = tid;
+          }
+          best[tid] = bst;
+        }
+        __syncthreads();                                         // (2) best, flagged complete
+
+        // ---- rows too close for the expanded form: a warp per row, direct differences in fp64 ----
+        const int nflag = flagged[0];
+        if (nflag > 0) {
+          for (int f = wid; f < nflag; f += WARPS) {
+            const int r = flagged[1 + f];
+            const float* xr = xb + (size_t)r * XS;
+            double bd = 1e300;
+            int bi = 0x7fffffff;
+            for (int a = lane; a < k; a += 32) {
+              const float* wa = wR + (size_t)a * XS;
+              double s = 0.0;
+              for (int j = 0; j < D; ++j) {
+                const double df = (double)xr[j] + 0.5 * (double)wa[j];     // -0.5 * (-2w) = w, exact
+                s = fma(df, df, s);
+              }
+              if (s < bd) { bd = s; bi = a; }                    // ascending a: the lowest index keeps a tie
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+              const double od = __shfl_xor_sync(0xffffffffu, bd, o);
+              const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+              if (od < bd || (od == bd && oi < bi)) { bd = od; bi = oi; }
+            }
+            if (lane == 0) best[r] = bi;
+          }
+          __syncthreads();                                       // (2b) uniform: nflag is the same for all threads
+        }
+        if (p.assign_rec && tid < rows) p.assign_rec[(size_t)i * b + (size_t)tl * TS + tid] = best[tid];
+
+        // ---- Eq. 9: the warp adds the tile's rows of the centres it owns, lane = dimension ----
+        {
+          const int b0 = (lane < TS) ? best[lane] : -1;
+          const int b1 = (TS > 32 && 32 + lane < TS) ? best[32 + lane] : -1;
+          const int b2 = (TS > 64 && 64 + lane < TS) ? best[64 + lane] : -1;
+          const int b3 = (TS > 96 && 96 + lane < TS) ? best[96 + lane] : -1;
+          for (int a = wid; a < k; a += WARPS) {
+            unsigned msk[4];
+            msk[0] = __ballot_sync(0xffffffffu, b0 == a);
+            msk[1] = (TS > 32) ? __ballot_sync(0xffffffffu, b1 == a) : 0u;
+            msk[2] = (TS > 64) ? __ballot_sync(0xffffffffu, b2 == a) : 0u;
+            msk[3] = (TS > 96) ? __ballot_sync(0xffffffffu, b3 == a) : 0u;
+            const int n = __popc(msk[0]) + __popc(msk[1]) + __popc(msk[2]) + __popc(msk[3]);
+            if (n == 0) continue;
+            float sum[DR];
+#pragma unroll
+            for (int q = 0; q < DR; ++q) sum[q] = 0.f;
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+              unsigned m = msk[h];
+              while (m) {
+                const int r = 32 * h + __ffs(m) - 1;
+                m &= m - 1;
+#pragma unroll
+                for (int q = 0; q < DR; ++q) sum[q] += xb[(size_t)r * XS + lane + 32 * q];
+              }
+            }
+#pragma unroll
+            for (int q = 0; q < DR; ++q) S[(size_t)a * D + lane + 32 * q] += sum[q];
+            if (lane == 0) cnt[a] += n;
+          }
+        }
+        if (__syncthreads_or(abort)) { abort = 1; break; }      // (3) tile consumed
+      }
+      if (abort) break;
+
+      step_tail<kDet>(p, i, t, wglob, S, cnt, nullptr, ts);
+      __syncthreads();
+    }
+  }
+
+  if (abort) {
+    if (tid == 0) atomicExch(p.status, DEV_TIMEOUT);
+    mbar_wait_bounded(bars + 0, 0); mbar_wait_bounded(bars + 0, 1);
+    mbar_wait_bounded(bars + 1, 0); mbar_wait_bounded(bars + 1, 1);
+  }
+}
+
+}  // namespace asgd

@@ -123,6 +123,11 @@ EDGE_CASES = {
     "stream_10x10_to_the_last_row": dict(N=4 * 33 * 3, d=10, k=10, W=4, b=33, comm_interval=1, fanout=3),
     "stream_10x10_full_block": dict(N=3 * 512 * 3 + 7, d=10, k=10, W=3, b=512, comm_interval=2, fanout=1),
     "stream_10x10_odd_batch": dict(N=3 * 129 * 5, d=10, k=10, W=3, b=129, comm_interval=2, fanout=1),
+    # shapes of the register-tiled kernel: padded centres, ragged last tile, several workers per block
+    "tiled_32_k37_ragged_tile": dict(N=5 * 100 * 3 + 1, d=32, k=37, W=5, b=100, comm_interval=2, fanout=2),
+    "tiled_32_many_workers": dict(N=700 * 12, d=32, k=8, W=700, b=4, comm_interval=1, fanout=1),
+    "tiled_128_k128": dict(N=3 * 200 * 2, d=128, k=128, W=3, b=200, comm_interval=1, fanout=1),
+    "tiled_128_k5_tiny_batch": dict(N=4 * 7 * 3, d=128, k=5, W=4, b=7, comm_interval=1, fanout=3),
     "general_10x10_big_batch": dict(N=2 * 700 * 3, d=10, k=10, W=2, b=700, comm_interval=2, fanout=1),
 }
 
