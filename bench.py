@@ -237,6 +237,18 @@ def main():
         import hashlib
         if ctx.path_name() == "fp32-stream" and hashlib.sha1(f.read()).hexdigest()[:12] == TRAFFIC_CAPTURE["kernel_sha1"]:
             traffic = bytes_per_launch * TRAFFIC_CAPTURE["traffic_per_algorithmic_byte"]
+    if ctx.path_name() in ("fp32-tiled",):
+        # bound by the fp32 pipe: 2*k*d flops per sample against SMs x 128 lanes x 2 x max SM clock
+        props = torch.cuda.get_device_properties(dev)
+        alu_peak = props.multi_processor_count * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
+        flops = 2.0 * wl.k * wl.d * samples_per_pass
+        ach = flops / (launch_ms * 1e-3) / 1e12
+        roofline_alu = {"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "TFLOP/s", "frac": ach / alu_peak,
+                        "traffic": None, "peak_kind": "SMs x 128 fp32 lanes x 2 x max SM clock", "kernel": ctx.path_name(),
+                        "launch_ms": launch_ms, "algorithmic_flops_per_launch": flops,
+                        "hbm_GBs": achieved}
+    else:
+        roofline_alu = None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                 "kernel": ctx.path_name(), "launch_ms": launch_ms, "algorithmic_bytes_per_launch": bytes_per_launch}
@@ -284,7 +296,7 @@ def main():
                        "comm_interval": wl.comm_interval, "fanout": wl.fanout, "mode": "free-running",
                        "steps_per_worker_per_bench_step": steps, "parallelism": "dp%d" % world,
                        "l2": "inputs larger than L2 (%.2f GB per pass)" % (bytes_per_launch / 1e9)},
-            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "roofline": roofline_alu or roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "quantization_error_worker0": E_final,
         }
         print(json.dumps(line), flush=True)

@@ -115,7 +115,7 @@ asgd_generic_kernel(const Params p, const long long steps, const int state_on_ch
     }
     __syncthreads();
 
-    step_tail<kDet>(p, i, t, w, SD, cnt, state_on_chip ? wglob : nullptr, ts);
+    step_tail<kDet>(p, i, t, w, d, SD, cnt, state_on_chip ? wglob : nullptr, ts);
     __syncthreads();
   }
 }

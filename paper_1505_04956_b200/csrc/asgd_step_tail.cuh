@@ -14,48 +14,52 @@ constexpr int MAX_SLOTS = 16;
 struct TailScratch {
   double red[96];
   int accept[MAX_SLOTS];
+  int fresh[MAX_SLOTS];
   int peers[MAX_FANOUT];
   int pslots[MAX_FANOUT];
   int flag;
   int m;
 };
 
-// w     [kd]  this worker's state (shared or global memory), updated in place
+// w     [k rows of d, row stride wstride]  this worker's state (shared or global memory), updated in place
 // SD    [kd]  in: per-centre sums S_k of the mini-batch; out: the local gradient D
 // cnt   [k]   per-centre counts n_k
 // wglob       the worker's row of Params::state when w lives in shared memory, else nullptr
 template <bool kDet>
-__device__ inline void step_tail(const Params& p, int i, unsigned long long t, float* w, float* SD,
+__device__ inline void step_tail(const Params& p, int i, unsigned long long t, float* w, int wstride, float* SD,
                                  const int* cnt, float* wglob, TailScratch* ts) {
   const int tid = threadIdx.x, nt = blockDim.x;
   const int kd = p.kd, d = p.d;
+  const bool dense_rows = (wstride == d);
+  auto widx = [&](int e) { return dense_rows ? e : (e / d) * wstride + (e % d); };
   const float inv_b = 1.0f / (float)p.b;
   const float eps = p.eps;
 
   // Eq. 9 (true-gradient sign, mean over the mini-batch size): D_k = (n_k w_k - S_k) / b
   for (int e = tid; e < kd; e += nt) {
     const int a = e / d;
-    SD[e] = ((float)cnt[a] * w[e] - SD[e]) * inv_b;
+    SD[e] = ((float)cnt[a] * w[widx(e)] - SD[e]) * inv_b;
   }
   __syncthreads();
 
-  // receive buffers
+  // receive buffers: thread s looks at buffer s (all buffers at once, one L2 round trip)
   int m = 0;
-  unsigned long long n_recv = 0, n_over = 0;
+  if (tid < p.S) {
+    const size_t si = (size_t)i * p.S + tid;
+    const unsigned sq = ld_acquire_gpu(p.seq + si);
+    const unsigned sn = p.seen[si];
+    ts->fresh[tid] = (sq != sn);
+    if (sq != sn) {
+      p.seen[si] = sq;
+      unsigned long long* st = p.stats + (size_t)i * ST_STRIDE;
+      atomicAdd(st + ST_RECV, 1ull);
+      if (sq - sn > 1u) atomicAdd(st + ST_OVERWRITTEN, (unsigned long long)(sq - sn - 1u));
+    }
+  }
+  __syncthreads();
   for (int s = 0; s < p.S; ++s) {
     const size_t si = (size_t)i * p.S + s;
-    if (tid == 0) {
-      const unsigned sq = ld_acquire_gpu(p.seq + si);
-      const unsigned sn = p.seen[si];
-      ts->flag = (sq != sn);
-      if (sq != sn) {
-        p.seen[si] = sq;
-        n_recv += 1;
-        n_over += (unsigned long long)(sq - sn - 1u);
-      }
-    }
-    __syncthreads();
-    const bool fresh = ts->flag != 0;
+    const bool fresh = ts->fresh[s] != 0;
     int acc = -1;
     if (fresh) {
       const float* v = p.mail + si * (size_t)p.kd_pad;
@@ -63,7 +67,7 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
       for (int e = tid; e < kd; e += nt) {
         const float vv = __ldcg(v + e);
         const float D = SD[e];
-        const float df = w[e] - vv;
+        const float df = w[widx(e)] - vv;
         dot += (double)D * (double)df;
         dd += (double)D * (double)D;
         nv += (double)vv * (double)vv;
@@ -84,10 +88,11 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
     float sumv = 0.f;
     for (int s = 0; s < p.S; ++s)
       if (ts->accept[s] == 1) sumv += __ldcg(p.mail + ((size_t)i * p.S + s) * (size_t)p.kd_pad + e);
-    const float ww = w[e];
+    const int we = widx(e);
+    const float ww = w[we];
     const float Dbar = (ww - (ww + sumv) * inv_m1) + SD[e];
     const float nw = ww - eps * Dbar;
-    w[e] = nw;
+    w[we] = nw;
     if (wglob) wglob[e] = nw;
   }
   __syncthreads();
@@ -114,7 +119,7 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
       for (int j = 0; j < p.f; ++j) {
         const size_t ri = (size_t)ts->peers[j] * p.S + ts->pslots[j];
         float* dst = p.mail + ri * (size_t)p.kd_pad;
-        for (int e = tid; e < kd; e += nt) dst[e] = w[e];
+        for (int e = tid; e < kd; e += nt) dst[e] = w[widx(e)];
         __syncthreads();
         if (tid == 0) red_release_gpu_inc(p.seq + ri);
       }
@@ -125,10 +130,8 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
   if (tid == 0) {
     unsigned long long* st = p.stats + (size_t)i * ST_STRIDE;
     st[ST_STEPS] = t + 1;
-    st[ST_SENT] += n_sent;
-    st[ST_RECV] += n_recv;
-    st[ST_ACCEPT] += (unsigned long long)m;
-    st[ST_OVERWRITTEN] += n_over;
+    if (n_sent) atomicAdd(st + ST_SENT, n_sent);
+    if (m) atomicAdd(st + ST_ACCEPT, (unsigned long long)m);
   }
 }
 

@@ -344,7 +344,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
         SD[e] = ssum;
       }
       __syncthreads();
-      step_tail<kDet>(p, i, t, w, SD, cnt, wglob, ts);
+      step_tail<kDet>(p, i, t, w, D, SD, cnt, wglob, ts);
       if (tid < p.S) seen_s[tid] = p.seen[(size_t)i * p.S + tid];
       if (tid == 0) flags[0] = 0;
       if (tid < K) cnt[tid] = 0;

@@ -3,11 +3,11 @@
 //
 // A thread block serves one or more workers in turn (worker = blockIdx.x + v * gridDim.x): a step
 // loads the worker's state from HBM/L2, streams the mini-batch through a two-slot ring of sample
-// tiles (one bulk copy per row; rows and centres are padded by 4 floats so that the rows a warp
-// reads at once fall in different banks), and writes the state back through the shared step tail.
+// tiles (four bulk copies per tile, one per quarter of its rows, each quarter shifted by one bank
+// group; the -2w rows are padded by 4 floats: the rows a warp reads at once fall in different banks), and writes the state back through the shared step tail.
 //
 // Assignment (Eq. 8): the tile's scores  ||w_a||^2 - 2 x.w_a  are a small GEMM.  A warp covers
-// 16 samples x 32 centres, a lane 4 x 4 of them (interleaved: rows sg + 4*m, centres cg + 8*i):
+// 16 samples x 32 centres, a lane 4 x 4 of them (rows m of quarter sg, centres cg + 8*i):
 // per four dimensions it reads four 128-bit pieces of x rows and four of -2w rows and issues 64
 // FMAs.  The centre index rides in the low mantissa bits; minimum and runner-up are reduced over
 // the lanes and warps that share a sample; a sample whose two best scores are closer than the
@@ -27,13 +27,17 @@ constexpr int TILED_MAX_V = 32;     // workers one block can serve
 
 template <int D, int KP, int WS, int WK>
 struct TiledShape {
-  static_assert(D % 32 == 0 && KP % 32 == 0 && KP == 32 * WK, "tiled path: d a multiple of 32, KP = 32 * WK");
+  static_assert(D % 32 == 0 && KP == 32 * WK && WK <= 4, "tiled path: d a multiple of 32, KP = 32 * WK, WK <= 4");
   static constexpr int THREADS = 32 * WS * WK;
   static constexpr int WARPS = WS * WK;
   static constexpr int TS = 16 * WS;              // samples per tile
-  static constexpr int XS = D + 4;                // padded row stride of x tiles and of -2w (floats)
-  static constexpr int INDEX_BITS = (KP <= 32) ? 5 : (KP <= 64) ? 6 : (KP <= 128) ? 7 : 8;
-  static constexpr unsigned INDEX_MASK = (1u << INDEX_BITS) - 1u;
+  static constexpr int XS = D;                    // row stride inside a quarter of a sample tile (floats)
+  static constexpr int QR = 4 * WS;               // rows per quarter; a lane's sample group sg reads quarter sg
+  static constexpr int QS = QR * D + 4;           // quarter stride: each quarter starts 4 floats (one bank group) later,
+                                                  // so the four rows a warp reads at once fall in different banks
+  static constexpr int WST = D + 4;               // padded row stride of -2w: the 8 rows a quarter-warp reads fall in different banks
+  static constexpr int INDEX_BITS = 5;            // index inside the warp's block of 32 centres
+  static constexpr unsigned INDEX_MASK = 31u;
   static constexpr int DR = D / 32;               // dimensions per lane in the sums
 };
 
@@ -44,11 +48,11 @@ struct TiledSmem {
   __host__ __device__ explicit TiledSmem(int k) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) / 16 * 16; return o; };
-    wR = take((size_t)KP * T::XS * 4);
+    wR = take((size_t)KP * T::WST * 4);
     cn = take((size_t)KP * 4);
     S = take((size_t)k * D * 4);
     cnt = take((size_t)KP * 4);
-    xt = take((size_t)2 * T::TS * T::XS * 4);
+    xt = take((size_t)2 * 4 * T::QS * 4);
     best = take((size_t)T::TS * 4);
     x2 = take((size_t)T::TS * 4);
     red = take((size_t)WK * T::TS * 8);
@@ -67,15 +71,15 @@ template <int D, int KP, int WS, int WK, int MINB, bool kDet>
 __global__ void __launch_bounds__(32 * WS * WK, MINB)
 asgd_tiled_kernel(const Params p, const long long steps) {
   using T = TiledShape<D, KP, WS, WK>;
-  constexpr int TS = T::TS, XS = T::XS, THREADS = T::THREADS, WARPS = T::WARPS, DR = T::DR;
+  constexpr int TS = T::TS, XS = T::XS, QR = T::QR, QS = T::QS, WST = T::WST, THREADS = T::THREADS, WARPS = T::WARPS, DR = T::DR;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int k = p.k, b = p.b;
   const TiledSmem<D, KP, WS, WK> map(k);
-  float* wR = reinterpret_cast<float*>(smem_raw + map.wR);          // [KP][XS]  -2 w
+  float* wR = reinterpret_cast<float*>(smem_raw + map.wR);          // [KP][WST]  -2 w
   float* cn = reinterpret_cast<float*>(smem_raw + map.cn);          // [KP]      ||w_a||^2 (+inf for padding)
   float* S = reinterpret_cast<float*>(smem_raw + map.S);            // [k][D]
   int* cnt = reinterpret_cast<int*>(smem_raw + map.cnt);            // [KP]
-  float* xt = reinterpret_cast<float*>(smem_raw + map.xt);          // [2][TS][XS]
+  float* xt = reinterpret_cast<float*>(smem_raw + map.xt);          // [2][4 quarters][QR][XS] (+4 floats per quarter)
   int* best = reinterpret_cast<int*>(smem_raw + map.best);          // [TS]
   float* x2s = reinterpret_cast<float*>(smem_raw + map.x2);         // [TS]
   float2* red = reinterpret_cast<float2*>(smem_raw + map.red);      // [WK][TS] (minimum, runner-up)
@@ -104,22 +108,29 @@ asgd_tiled_kernel(const Params p, const long long steps) {
 
   // The launch consumes tiles in the order (step, worker slot, tile of the batch); tile g uses ring slot g & 1.
   const long long total_tiles = steps * nv * tiles;
-  auto issue_tile = [&](long long g) {            // called by all lanes of warp 0
-    const int tl = (int)(g % tiles);
-    const long long sv = g / tiles;
-    const int v = (int)(sv % nv);
+  // (tile, worker slot, step) of the next tile to fetch, advanced by the issuing warp only
+  int nx_tl = 0, nx_v = 0;
+  long long nx_st = 0, nx_g = 0;
+  auto issue_next = [&]() {                       // called by all lanes of the issuing warp
+    const int tl = nx_tl, v = nx_v;
     const int i = (int)blockIdx.x + v * G;
-    const unsigned long long t = tbase[v] + (unsigned long long)(sv / nv);
+    const unsigned long long t = tbase[v] + (unsigned long long)nx_st;
     const long long batch = p.perm[(size_t)i * p.B + (size_t)(t % (unsigned long long)p.B)];
     const int rows = min(TS, b - tl * TS);
-    const int slot = (int)(g & 1);
-    float* dst = xt + (size_t)slot * TS * XS;
+    const int slot = (int)(nx_g & 1);
+    float* dst = xt + (size_t)slot * 4 * QS;
     const float* src = p.X + ((size_t)i * p.H + (size_t)batch * b + (size_t)tl * TS) * D;
     if (lane == 0) mbar_expect_tx(bars + slot, (unsigned)rows * D * 4);
     __syncwarp();
-    for (int r = lane; r < rows; r += 32) bulk_g2s(dst + (size_t)r * XS, src + (size_t)r * D, D * 4, bars + slot);
+    if (lane < 4) {                                   // one copy per quarter of the tile
+      const int qrows = min(QR, rows - lane * QR);
+      if (qrows > 0) bulk_g2s(dst + (size_t)lane * QS, src + (size_t)lane * QR * D, (unsigned)qrows * D * 4, bars + slot);
+    }
+    ++nx_g;
+    if (++nx_tl == tiles) { nx_tl = 0; if (++nx_v == nv) { nx_v = 0; ++nx_st; } }
   };
-  if (wid == 0 && total_tiles > 0) issue_tile(0);
+  constexpr int ISSUER = WARPS - 1;               // the last warp has no row work in the merge phase
+  if (wid == ISSUER && total_tiles > 0) issue_next();
 
   int abort = 0;
   long long g = 0;
@@ -137,7 +148,7 @@ asgd_tiled_kernel(const Params p, const long long steps) {
           v4 = *reinterpret_cast<const float4*>(wglob + (size_t)a * D + 4 * j4);
           v4.x *= -2.f; v4.y *= -2.f; v4.z *= -2.f; v4.w *= -2.f;
         }
-        *reinterpret_cast<float4*>(wR + (size_t)a * XS + 4 * j4) = v4;
+        *reinterpret_cast<float4*>(wR + (size_t)a * WST + 4 * j4) = v4;
       }
       for (int e = tid; e < k * D; e += THREADS) S[e] = 0.f;
       for (int e = tid; e < KP; e += THREADS) cnt[e] = 0;
@@ -145,7 +156,7 @@ asgd_tiled_kernel(const Params p, const long long steps) {
       for (int a = wid; a < KP; a += WARPS) {
         float s = 0.f;
 #pragma unroll
-        for (int q = 0; q < DR; ++q) { const float u = wR[(size_t)a * XS + lane + 32 * q]; s = fmaf(u, u, s); }
+        for (int q = 0; q < DR; ++q) { const float u = wR[(size_t)a * WST + lane + 32 * q]; s = fmaf(u, u, s); }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         if (lane == 0) cn[a] = (a < k) ? 0.25f * s : INF;
@@ -163,11 +174,8 @@ asgd_tiled_kernel(const Params p, const long long steps) {
         const int slot = (int)(g & 1);
         const unsigned parity = (unsigned)((g >> 1) & 1);
         const int rows = min(TS, b - tl * TS);
-        const float* xb = xt + (size_t)slot * TS * XS;
-        if (wid == 0 && g + 1 < total_tiles) {
-          fence_proxy_async_smem();
-          issue_tile(g + 1);
-        }
+        const float* xb = xt + (size_t)slot * 4 * QS;
+        auto xrowp = [&](int r) { return xb + (size_t)(r / QR) * QS + (size_t)(r % QR) * XS; };   // tile row r
         if (tid == 0) flagged[0] = 0;
         if (!mbar_wait_bounded(bars + slot, parity)) abort = 1;
 
@@ -177,15 +185,15 @@ asgd_tiled_kernel(const Params p, const long long steps) {
         for (int m = 0; m < 4; ++m)
 #pragma unroll
           for (int c = 0; c < 4; ++c) acc[m][c] = 0.f;
-        const float* xrow = xb + (size_t)(wsi * 16 + sg) * XS;
-        const float* wrow = wR + (size_t)(wk * 32 + cg) * XS;
+        const float* xrow = xb + (size_t)sg * QS + (size_t)(wsi * 4) * XS;    // rows sg*QR + wsi*4 + m
+        const float* wrow = wR + (size_t)(wk * 32 + cg) * WST;
 #pragma unroll 2
         for (int j = 0; j < D; j += 4) {
           float4 xv[4], wv[4];
 #pragma unroll
-          for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xrow + (size_t)(4 * m) * XS + j);
+          for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xrow + (size_t)m * XS + j);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) wv[c] = *reinterpret_cast<const float4*>(wrow + (size_t)(8 * c) * XS + j);
+          for (int c = 0; c < 4; ++c) wv[c] = *reinterpret_cast<const float4*>(wrow + (size_t)(8 * c) * WST + j);
 #pragma unroll
           for (int m = 0; m < 4; ++m)
 #pragma unroll
@@ -206,7 +214,7 @@ asgd_tiled_kernel(const Params p, const long long steps) {
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             const float sc = acc[m][c] + cnv[c];
-            const float sp = __uint_as_float((__float_as_uint(sc) & ~T::INDEX_MASK) | (unsigned)(wk * 32 + 8 * c + cg));
+            const float sp = __uint_as_float((__float_as_uint(sc) & ~T::INDEX_MASK) | (unsigned)(8 * c + cg));
             s2 = fmaxf(s1, fminf(s2, sp));
             s1 = fminf(s1, sp);
           }
@@ -217,56 +225,95 @@ asgd_tiled_kernel(const Params p, const long long steps) {
             s2 = fminf(fmaxf(s1, o1), fminf(s2, o2));
             s1 = fminf(s1, o1);
           }
-          if (cg == 0) red[(size_t)wk * TS + wsi * 16 + 4 * m + sg] = make_float2(s1, s2);
+          if (cg == 0) red[(size_t)wk * TS + sg * QR + wsi * 4 + m] = make_float2(s1, s2);
         }
-        __syncthreads();                                         // (1) red complete
+        // the ring slot of the previous tile is free since that tile's last barrier: fetch the next tile now
+        if (wid == ISSUER && g + 1 < total_tiles) {
+          fence_proxy_async_smem();
+          issue_next();
+        }
+        // ---- ||x||^2 of every tile row: 8 threads per row, 4 dimensions at a time ----
+        for (int r = tid >> 3; r < TS; r += THREADS / 8) {
+          const int h = tid & 7;
+          float xx = 0.f;
+#pragma unroll
+          for (int q = 0; q < D / 32; ++q) {
+            const float4 u = *reinterpret_cast<const float4*>(xrowp(r) + 4 * h + 32 * q);
+            xx = fmaf(u.x, u.x, xx); xx = fmaf(u.y, u.y, xx); xx = fmaf(u.z, u.z, xx); xx = fmaf(u.w, u.w, xx);
+          }
+          xx += __shfl_xor_sync(0xffffffffu, xx, 1);
+          xx += __shfl_xor_sync(0xffffffffu, xx, 2);
+          xx += __shfl_xor_sync(0xffffffffu, xx, 4);
+          if (h == 0) x2s[r] = xx;
+        }
+        __syncthreads();                                         // (1) red, x2s complete
 
         // ---- one thread per tile row: merge over the centre blocks, decide or flag ----
         if (tid < TS) {
           int bst = -1;
           if (tid < rows) {
             float s1 = INF, s2 = INF;
+            int qwin = 0;
 #pragma unroll
             for (int q = 0; q < WK; ++q) {
               const float2 r = red[(size_t)q * TS + tid];
               s2 = fminf(fmaxf(s1, r.x), fminf(s2, r.y));
-              s1 = fminf(s1, r.x);
+              if (r.x < s1) { s1 = r.x; qwin = q; }             // equal packed scores of two blocks: second look below
             }
-            float xx = 0.f;
-            const float4* xr = reinterpret_cast<const float4*>(xb + (size_t)tid * XS);
-            for (int j4 = 0; j4 < D / 4; ++j4) {
-              const float4 u = xr[j4];
-              xx = fmaf(u.x, u.x, xx); xx = fmaf(u.y, u.y, xx); xx = fmaf(u.z, u.z, xx); xx = fmaf(u.w, u.w, xx);
-            }
-            bst = (int)(__float_as_uint(s1) & T::INDEX_MASK);
-            if (k > 1 && (s2 - s1) <= tau_scale * (misc[0] + xx)) flagged[1 + atomicAdd(flagged, 1)] = tid;
+            bst = qwin * 32 + (int)(__float_as_uint(s1) & T::INDEX_MASK);
+            if (k > 1 && (s2 - s1) <= tau_scale * (misc[0] + x2s[tid])) flagged[1 + atomicAdd(flagged, 1)] = tid;
           }
           best[tid] = bst;
         }
         __syncthreads();                                         // (2) best, flagged complete
 
-        // ---- rows too close for the expanded form: a warp per row, direct differences in fp64 ----
+        // ---- rows too close for the expanded form: a warp per row, lanes over centres, direct
+        //      differences in fp32; if that is still within rounding of a tie, in fp64 ----
         const int nflag = flagged[0];
         if (nflag > 0) {
           for (int f = wid; f < nflag; f += WARPS) {
             const int r = flagged[1 + f];
-            const float* xr = xb + (size_t)r * XS;
-            double bd = 1e300;
-            int bi = 0x7fffffff;
+            const float* xr = xrowp(r);
+            float fd1 = INF, fd2 = INF;
+            int fi = 0x7fffffff;
             for (int a = lane; a < k; a += 32) {
-              const float* wa = wR + (size_t)a * XS;
-              double s = 0.0;
+              const float* wa = wR + (size_t)a * WST;
+              float s = 0.f;
+#pragma unroll 4
               for (int j = 0; j < D; ++j) {
-                const double df = (double)xr[j] + 0.5 * (double)wa[j];     // -0.5 * (-2w) = w, exact
-                s = fma(df, df, s);
+                const float df = xr[j] + 0.5f * wa[j];                     // -0.5 * (-2w) = w, exact
+                s = fmaf(df, df, s);
               }
-              if (s < bd) { bd = s; bi = a; }                    // ascending a: the lowest index keeps a tie
+              if (s < fd1) { fd2 = fd1; fd1 = s; fi = a; } else if (s < fd2) { fd2 = s; }
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
-              const double od = __shfl_xor_sync(0xffffffffu, bd, o);
-              const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-              if (od < bd || (od == bd && oi < bi)) { bd = od; bi = oi; }
+              const float o1 = __shfl_xor_sync(0xffffffffu, fd1, o);
+              const float o2 = __shfl_xor_sync(0xffffffffu, fd2, o);
+              const int oi = __shfl_xor_sync(0xffffffffu, fi, o);
+              const bool take = (o1 < fd1) || (o1 == fd1 && oi < fi);
+              fd2 = fminf(take ? fd1 : o1, fminf(fd2, o2));
+              if (take) { fd1 = o1; fi = oi; }
+            }
+            int bi = fi;
+            if (fd2 - fd1 <= (float)(4 * D + 16) * 5.9604645e-8f * fd2) {
+              double bd = 1e300;
+              bi = 0x7fffffff;
+              for (int a = lane; a < k; a += 32) {
+                const float* wa = wR + (size_t)a * WST;
+                double s = 0.0;
+                for (int j = 0; j < D; ++j) {
+                  const double df = (double)xr[j] + 0.5 * (double)wa[j];
+                  s = fma(df, df, s);
+                }
+                if (s < bd) { bd = s; bi = a; }                  // ascending a: the lowest index keeps a tie
+              }
+#pragma unroll
+              for (int o = 16; o > 0; o >>= 1) {
+                const double od = __shfl_xor_sync(0xffffffffu, bd, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (od < bd || (od == bd && oi < bi)) { bd = od; bi = oi; }
+              }
             }
             if (lane == 0) best[r] = bi;
           }
@@ -297,8 +344,23 @@ asgd_tiled_kernel(const Params p, const long long steps) {
               while (m) {
                 const int r = 32 * h + __ffs(m) - 1;
                 m &= m - 1;
+                const float* xr = xrowp(r);
+                float u[DR];
 #pragma unroll
-                for (int q = 0; q < DR; ++q) sum[q] += xb[(size_t)r * XS + lane + 32 * q];
+                for (int q = 0; q < DR; ++q) u[q] = xr[lane + 32 * q];
+                if (m) {                                           // a second row in flight with the first
+                  const int r2 = 32 * h + __ffs(m) - 1;
+                  m &= m - 1;
+                  const float* xr2 = xrowp(r2);
+                  float u2[DR];
+#pragma unroll
+                  for (int q = 0; q < DR; ++q) u2[q] = xr2[lane + 32 * q];
+#pragma unroll
+                  for (int q = 0; q < DR; ++q) sum[q] = (sum[q] + u[q]) + u2[q];
+                } else {
+#pragma unroll
+                  for (int q = 0; q < DR; ++q) sum[q] += u[q];
+                }
               }
             }
 #pragma unroll
@@ -310,7 +372,15 @@ asgd_tiled_kernel(const Params p, const long long steps) {
       }
       if (abort) break;
 
-      step_tail<kDet>(p, i, t, wglob, S, cnt, nullptr, ts);
+      // the tail works on the state in shared memory: turn the -2w rows back into w (exact)
+      for (int e = tid; e < k * (D / 4); e += THREADS) {
+        float4* q4 = reinterpret_cast<float4*>(wR + (size_t)(e / (D / 4)) * WST + 4 * (e % (D / 4)));
+        float4 u = *q4;
+        u.x *= -0.5f; u.y *= -0.5f; u.z *= -0.5f; u.w *= -0.5f;
+        *q4 = u;
+      }
+      __syncthreads();
+      step_tail<kDet>(p, i, t, wR, WST, S, cnt, wglob, ts);
       __syncthreads();
     }
   }
