@@ -13,12 +13,15 @@
 #include "asgd_generic.cuh"
 #include "asgd_stream.cuh"
 #include "asgd_tiled.cuh"
+#include "asgd_tc.cuh"
+
+#include <cudaTypedefs.h>
 
 using namespace asgd;
 
 namespace {
 
-enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2 };
+enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2, P_TC_BF16 = 3 };
 
 // (d, k) shapes the streaming path is compiled for
 #define ASGD_STREAM_SHAPES(X) X(10, 10) X(16, 16) X(4, 5) X(2, 3)
@@ -29,7 +32,7 @@ enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2 };
 
 struct Layout {
   size_t state, mail, seq, seen, arb_win, arb_cnt, stats, perm, status, assign_rec, accept_rec, gsum,
-      eval_partial, tmp_state, xmax, total;
+      eval_partial, tmp_state, xmax, wbf, top2, xbf, total;
 };
 
 constexpr size_t kAlign = 256;
@@ -51,6 +54,12 @@ bool config_ok(const asgd_config* c) {
   if (H < c->b) return false;
   if ((long long)c->W * c->fanout + 1 > 0x7fffffffll) return false;
   return true;
+}
+
+// shapes the tensor-core path takes: d a multiple of 64 up to 256, more centres than the tiled path holds
+bool tc_eligible(const asgd_config* c) {
+  return c->d % TC_KC == 0 && c->d <= TC_MAX_D && c->k > 128 && c->k <= TC_MAX_K && c->b >= TC_M && c->b <= TC_MAX_B &&
+         tc_smem_bytes(c->k, c->d, c->b) <= kMaxDynSmem;
 }
 
 Layout make_layout(const asgd_config* c) {
@@ -75,6 +84,10 @@ Layout make_layout(const asgd_config* c) {
   L.eval_partial = take((size_t)kEvalBlocks * 8);
   L.tmp_state = take(kd_pad * 4);
   L.xmax = take(64);
+  const bool tc = tc_eligible(c) && (c->dist_path == ASGD_PATH_TC_BF16 || c->dist_path == ASGD_PATH_AUTO);
+  L.wbf = take(tc ? W * kd * 2 : 4);
+  L.top2 = take(tc ? W * (size_t)c->b * 8 : 4);
+  L.xbf = take(tc ? (size_t)c->N * c->d * 2 : 4);
   L.total = off;
   return L;
 }
@@ -95,6 +108,8 @@ struct asgd_ctx {
   long long launches;
   int last_cuda;
   int sm_count;
+  const void* xbf_user;   // caller's bf16 copy of X, or nullptr
+  CUtensorMap mapX, mapW; // tensor-core path: bf16 samples [N][d], bf16 -2w [W*k][d]
 };
 
 namespace {
@@ -157,9 +172,63 @@ void tiled_launch(asgd_ctx* c, bool det, long long steps) {
     asgd_tiled_kernel<D, KP, WS, WK, MINB, false><<<c->grid, 32 * WS * WK, c->smem_bytes, c->stream>>>(c->p, steps);
 }
 
+bool encode_bf16_map(CUtensorMap* map, const void* base, unsigned long long rows, unsigned long long cols, unsigned box_rows) {
+  static PFN_cuTensorMapEncodeTiled encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess || !fn) return false;
+    encode = (PFN_cuTensorMapEncodeTiled)fn;
+  }
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TC_KC, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tensor-core path set-up: bf16 copy of X (unless the caller brought one), max ||x||^2, tensor maps.
+int tc_prepare(asgd_ctx* c) {
+  const asgd_config& cfg = c->cfg;
+  Params& p = c->p;
+  c->smem_bytes = tc_smem_bytes(cfg.k, cfg.d, cfg.b);
+  CU(c, cudaFuncSetAttribute(asgd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  CU(c, cudaFuncSetAttribute(asgd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  p.wbf = c->ws + c->L.wbf;
+  p.top2 = (float*)(c->ws + c->L.top2);
+  const void* xbf = c->xbf_user;
+  if (!xbf) {
+    void* dst = c->ws + c->L.xbf;
+    tc_convert_x_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, (__nv_bfloat16*)dst, (size_t)cfg.N * cfg.d);
+    c->launches += 1;
+    CU(c, cudaGetLastError());
+    xbf = dst;
+  }
+  unsigned* xm = (unsigned*)(c->ws + c->L.xmax);
+  CU(c, cudaMemsetAsync(xm, 0, 4, c->stream));
+  xmax2_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, p.N, p.d, xm);
+  c->launches += 1;
+  CU(c, cudaGetLastError());
+  float xmax2 = 0.f;
+  CU(c, cudaMemcpyAsync(&xmax2, xm, 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  p.xmax2 = xmax2;
+  if (!encode_bf16_map(&c->mapX, xbf, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
+  if (!encode_bf16_map(&c->mapW, p.wbf, (unsigned long long)cfg.W * cfg.k, (unsigned long long)cfg.d, TC_N)) return ASGD_ECUDA;
+  return ASGD_OK;
+}
+
 int launch_workers(asgd_ctx* c, bool det, long long steps) {
   const Params& p = c->p;
   switch (c->path) {
+    case P_TC_BF16:
+      if (det)
+        asgd_tc_kernel<true><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapX, c->mapW);
+      else
+        asgd_tc_kernel<false><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapX, c->mapW);
+      break;
     case P_TILED: {
       bool done = false;
 #define X(D_, KP_, WS_, WK_, MB_) if (!done && p.d == D_ && p.k <= KP_) { tiled_launch<D_, KP_, WS_, WK_, MB_>(c, det, steps); done = true; }
@@ -187,7 +256,13 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
 
 int resolve_path(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
-  if (cfg.dist_path == ASGD_PATH_TC_3XTF32 || cfg.dist_path == ASGD_PATH_TC_BF16) return ASGD_EUNSUPPORTED;
+  if (cfg.dist_path == ASGD_PATH_TC_3XTF32) return ASGD_EUNSUPPORTED;
+  if (cfg.dist_path == ASGD_PATH_TC_BF16 || (cfg.dist_path == ASGD_PATH_AUTO && tc_eligible(&cfg))) {
+    if (!tc_eligible(&cfg)) return ASGD_EUNSUPPORTED;
+    c->path = P_TC_BF16;
+    c->state_on_chip = 0;
+    return ASGD_OK;                       // device-side set-up (tc_prepare) runs once the workspace is cleared
+  }
   // streaming path: small state, a mini-batch of at most 4 samples per thread
   if (cfg.dist_path == ASGD_PATH_AUTO || cfg.dist_path == ASGD_PATH_FP32) {
 #define X(D_, K_)                                                                     \
@@ -240,7 +315,6 @@ int asgd_workspace_bytes(const asgd_config* cfg, size_t* bytes) {
 
 int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const void* X_bf16_dev,
               const float* w0_dev, void* workspace_dev, size_t workspace_bytes, void* cuda_stream) {
-  (void)X_bf16_dev;
   if (!out) return ASGD_EINVAL;
   *out = nullptr;
   if (!config_ok(cfg) || !X_dev || !w0_dev || !workspace_dev) return ASGD_EINVAL;
@@ -263,6 +337,7 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   c->launches = 0;
   c->last_cuda = 0;
   c->sm_count = prop.multiProcessorCount;
+  c->xbf_user = X_bf16_dev;
 
   Params& p = c->p;
   p.X = X_dev; p.N = cfg->N; p.d = cfg->d; p.k = cfg->k; p.W = cfg->W; p.b = cfg->b; p.eps = cfg->eps;
@@ -283,6 +358,8 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   p.accept_rec = (int*)(c->ws + L.accept_rec);
   p.gsum = (float*)(c->ws + L.gsum);
   p.xmax2 = 0.f;
+  p.wbf = nullptr;
+  p.top2 = nullptr;
 
   int rc = resolve_path(c);
   if (rc != ASGD_OK) { delete c; return rc; }
@@ -293,6 +370,10 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   if (e != cudaSuccess) { delete c; return ASGD_ECUDA; }
   broadcast_state_kernel<<<256, 256, 0, c->stream>>>(p.state, w0_dev, p.W, p.kd, p.kd_pad);
   c->launches += 1;
+  if (c->path == P_TC_BF16) {
+    rc = tc_prepare(c);
+    if (rc != ASGD_OK) { delete c; return rc; }
+  }
 
   // batch orders
   {
@@ -430,6 +511,7 @@ const char* asgd_path_name(const asgd_ctx* c) {
     case P_GENERIC: return c->state_on_chip ? "fp32-generic" : "fp32-generic-offchip";
     case P_STREAM: return "fp32-stream";
     case P_TILED: return "fp32-tiled";
+    case P_TC_BF16: return "tcgen05-bf16";
     default: return "unknown";
   }
 }

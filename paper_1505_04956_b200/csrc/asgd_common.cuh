@@ -34,7 +34,9 @@ struct Params {
   int* assign_rec;         // [W][b] or nullptr
   int* accept_rec;         // [W][S] acceptance of the last step
   float* gsum;             // [W][kd_pad] per-worker sums when the state does not fit on chip
-  float xmax2;             // max_i ||x_i||^2 over X (bound used by the expanded-form paths)
+  float xmax2;             // max_i ||x_i||^2 over X (error bound of the tensor-core path)
+  void* wbf;               // [W][k][d] bf16 copies of -2w (tensor-core path)
+  float* top2;             // [W][b][2] running (minimum, runner-up) scores (tensor-core path)
 };
 
 // ---------------------------------------------------------------------------------------------

@@ -25,9 +25,10 @@ struct TailScratch {
 // SD    [kd]  in: per-centre sums S_k of the mini-batch; out: the local gradient D
 // cnt   [k]   per-centre counts n_k
 // wglob       the worker's row of Params::state when w lives in shared memory, else nullptr
+// sd_l2   the sums in SD were produced by reductions in L2: read them past L1
 template <bool kDet>
 __device__ inline void step_tail(const Params& p, int i, unsigned long long t, float* w, int wstride, float* SD,
-                                 const int* cnt, float* wglob, TailScratch* ts) {
+                                 const int* cnt, float* wglob, TailScratch* ts, bool sd_l2 = false) {
   const int tid = threadIdx.x, nt = blockDim.x;
   const int kd = p.kd, d = p.d;
   const bool dense_rows = (wstride == d);
@@ -38,7 +39,8 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
   // Eq. 9 (true-gradient sign, mean over the mini-batch size): D_k = (n_k w_k - S_k) / b
   for (int e = tid; e < kd; e += nt) {
     const int a = e / d;
-    SD[e] = ((float)cnt[a] * w[widx(e)] - SD[e]) * inv_b;
+    const float sums = sd_l2 ? __ldcg(SD + e) : SD[e];
+    SD[e] = ((float)cnt[a] * w[widx(e)] - sums) * inv_b;
   }
   __syncthreads();
 

@@ -1,0 +1,386 @@
+// Tensor-core path (tcgen05, BF16 operands, FP32 accumulate in tensor memory) for large states
+// (k up to 1024, d a multiple of 64 up to 256): the shapes where the scores of Eq. 8 are a dense
+// contraction  -2 X W^T  of a 4096 x 256 mini-batch against a 1024 x 256 centre matrix.
+//
+// One worker = one thread block = one SM.  Warp roles while the scores are computed:
+//   warp 0   one lane issues the TMA loads: the current 256-centre block of bf16(-2w) (resident for
+//            a whole sweep over the mini-batch) and the 128-row sample tiles in 128-byte-swizzled
+//            K-chunks of 64 through a 4-slot ring;
+//   warp 1   allocates tensor memory; one lane issues tcgen05.mma (128 x 256 x 16 per instruction)
+//            into one of two 256-column accumulators and commits to mbarriers;
+//   warps 2-5  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread), add
+//            ||w_a||^2 and keep, per sample, the two smallest scores with the centre index packed
+//            into the low mantissa bits; the pair lives in a small per-worker scratch in L2 between
+//            the four centre blocks.
+// Then all warps: samples whose two best scores are closer than the BF16 error bound are decided
+// between those two centres with fp32 inputs (fp64 sums); per-centre sums of the fp32 master
+// samples go to the worker's sum buffer with vector reductions; a warp per centre applies the
+// update, refreshes bf16(-2w) and ||w_a||^2.  Every wait is bounded.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "asgd_step_tail.cuh"
+#include "asgd_stream.cuh"   // mbarrier helpers
+
+namespace asgd {
+
+constexpr int TC_THREADS = 256;
+constexpr int TC_WARPS = TC_THREADS / 32;
+constexpr int TC_M = 128, TC_N = 256, TC_KC = 64;        // output tile; K chunk = 64 bf16 = one swizzled 128-byte row
+constexpr int TC_A_STAGES = 4;
+constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB
+constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;       // 32 KB
+constexpr int TC_MAX_K = 1024, TC_MAX_D = 256, TC_MAX_B = 8192;
+constexpr unsigned TC_INDEX_MASK = 1023u;
+
+struct TcSmem {
+  size_t B, A, cn, cnt, best, flagged, bars, misc, tail, total;
+  __host__ __device__ TcSmem(int k, int d, int b) {
+    size_t off = 0;
+    auto take = [&](size_t bytes, size_t align) { off = (off + align - 1) / align * align; size_t o = off; off += bytes; return o; };
+    B = take((size_t)(d / TC_KC) * TC_B_CHUNK_BYTES, 1024);
+    A = take((size_t)TC_A_STAGES * TC_A_STAGE_BYTES, 1024);
+    cn = take((size_t)((k + TC_N - 1) / TC_N) * TC_N * 4, 16);
+    cnt = take((size_t)k * 4, 16);
+    best = take((size_t)b * 2, 16);
+    flagged = take((size_t)b * 2 + 16, 16);
+    bars = take(32 * 8, 16);
+    misc = take(64, 16);
+    tail = take(sizeof(TailScratch), 16);
+    total = off + 1024;          // room to align the base to 1024 bytes
+  }
+};
+inline size_t tc_smem_bytes(int k, int d, int b) { return TcSmem(k, d, b).total; }
+
+__device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+// Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ inline unsigned long long tc_smem_desc(const void* smem, unsigned byte_off) {
+  const unsigned addr = smem_u32(smem) + byte_off;
+  unsigned long long d = 0;
+  d |= (unsigned long long)((addr & 0x3FFFFu) >> 4);
+  d |= (unsigned long long)1 << 16;
+  d |= (unsigned long long)(1024 >> 4) << 32;
+  d |= (unsigned long long)1 << 46;
+  d |= (unsigned long long)2 << 61;
+  return d;
+}
+__device__ inline void tc_mma_bf16(unsigned d_tmem, unsigned long long a, unsigned long long b, unsigned idesc, bool acc) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"((unsigned)acc) : "memory");
+}
+__device__ inline void tc_commit(unsigned long long* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ inline void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ inline void red_add_v4(float* addr, float4 v) {
+  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+
+// samples -> bf16 copy (initialisation, when the caller gave none)
+__global__ void tc_convert_x_kernel(const float* __restrict__ X, __nv_bfloat16* __restrict__ out, size_t n) {
+  for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; e + 3 < n; e += (size_t)gridDim.x * blockDim.x * 4) {
+    const float4 v = *reinterpret_cast<const float4*>(X + e);
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    *reinterpret_cast<__nv_bfloat162*>(out + e) = lo;
+    *reinterpret_cast<__nv_bfloat162*>(out + e + 2) = hi;
+  }
+}
+
+// barrier slots
+enum { TCB_BFULL = 0, TCB_BEMPTY = 1, TCB_AFULL = 2, TCB_AEMPTY = 2 + TC_A_STAGES, TCB_ACCFULL = 2 + 2 * TC_A_STAGES,
+       TCB_ACCEMPTY = 4 + 2 * TC_A_STAGES, TCB_COUNT = 6 + 2 * TC_A_STAGES };
+
+template <bool kDet>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CUtensorMap mapX,
+               const __grid_constant__ CUtensorMap mapW) {
+  extern __shared__ __align__(1024) unsigned char smem_dyn[];
+  unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
+  const int k = p.k, d = p.d, b = p.b;
+  const TcSmem map(k, d, b);
+  unsigned char* sB = smem + map.B;
+  unsigned char* sA = smem + map.A;
+  float* cn = reinterpret_cast<float*>(smem + map.cn);                 // ||w_a||^2, +inf beyond k
+  int* cnt = reinterpret_cast<int*>(smem + map.cnt);
+  unsigned short* best = reinterpret_cast<unsigned short*>(smem + map.best);
+  unsigned short* flagged = reinterpret_cast<unsigned short*>(smem + map.flagged);
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + map.bars);
+  int* misc = reinterpret_cast<int*>(smem + map.misc);                 // [0] tmem base, [1] flagged count, [2] abort, [3] wmax2 bits
+  TailScratch* ts = reinterpret_cast<TailScratch*>(smem + map.tail);
+
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int i = blockIdx.x;
+  const int nkc = d / TC_KC;                                           // K chunks per tile
+  const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_M - 1) / TC_M;
+  const int dl = d / 32;                                               // dimensions per lane (multiple of 2)
+  float* wglob = p.state + (size_t)i * p.kd_pad;
+  float* gsum = p.gsum + (size_t)i * p.kd_pad;
+  __nv_bfloat16* wbf = reinterpret_cast<__nv_bfloat16*>(p.wbf) + (size_t)i * k * d;
+  float2* top2 = reinterpret_cast<float2*>(p.top2) + (size_t)i * b;
+  const float INF = __int_as_float(0x7f800000);
+  const float inv_b = 1.0f / (float)b;
+
+  if (tid == 0) {
+    mbar_init(bars + TCB_BFULL, 1);
+    mbar_init(bars + TCB_BEMPTY, 1);
+    for (int q = 0; q < TC_A_STAGES; ++q) { mbar_init(bars + TCB_AFULL + q, 1); mbar_init(bars + TCB_AEMPTY + q, 1); }
+    for (int q = 0; q < 2; ++q) { mbar_init(bars + TCB_ACCFULL + q, 1); mbar_init(bars + TCB_ACCEMPTY + q, 4); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    misc[2] = 0;
+  }
+  if (wid == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(misc)) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // prologue: bf16(-2w), ||w_a||^2 from the fp32 state (a warp per centre, lane = dl dimensions)
+  for (int a = wid; a < n_tiles * TC_N; a += TC_WARPS) {
+    float s = 0.f;
+    if (a < k) {
+      for (int j = lane * 2; j < d; j += 64) {
+        const float2 v = *reinterpret_cast<const float2*>(wglob + (size_t)a * d + j);
+        s = fmaf(v.x, v.x, s); s = fmaf(v.y, v.y, s);
+        *reinterpret_cast<__nv_bfloat162*>(wbf + (size_t)a * d + j) = __floats2bfloat162_rn(-2.f * v.x, -2.f * v.y);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    }
+    if (lane == 0) cn[a] = (a < k) ? s : INF;
+  }
+  asm volatile("fence.proxy.async;" ::: "memory");                      // bf16(-2w) written above is read by TMA
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem = (unsigned)misc[0];
+  const unsigned idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(TC_N >> 3) << 17) | ((unsigned)(TC_M >> 4) << 24);
+
+  unsigned long long t = p.stats[(size_t)i * ST_STRIDE + ST_STEPS];
+  // running phase counters of the pipelines (each role keeps its own copies in step)
+  unsigned it_b = 0, it_a = 0, it_acc = 0;
+
+  for (long long step = 0; step < steps; ++step, ++t) {
+    const long long batch = p.perm[(size_t)i * p.B + (size_t)(t % (unsigned long long)p.B)];
+    const long long row0 = (long long)i * p.H + batch * b;
+
+    // ================= scores: -2 X W^T + ||w||^2, two best per sample =================
+    if (wid == 0) {
+      if (lane == 0) {
+        unsigned ib = it_b, ia = it_a;
+        bool ok = true;
+        for (int n = 0; n < n_tiles && ok; ++n, ++ib) {
+          if (ib > 0) ok = mbar_wait_bounded(bars + TCB_BEMPTY, (ib - 1) & 1);           // previous block's MMAs done
+          if (!ok) break;
+          mbar_expect_tx(bars + TCB_BFULL, (unsigned)nkc * TC_B_CHUNK_BYTES);
+          for (int kc = 0; kc < nkc; ++kc)
+            tma_load_2d(sB + (size_t)kc * TC_B_CHUNK_BYTES, &mapW, kc * TC_KC, i * k + n * TC_N, bars + TCB_BFULL);
+          for (int m = 0; m < m_tiles && ok; ++m) {
+            for (int kc = 0; kc < nkc; ++kc, ++ia) {
+              const int st = ia % TC_A_STAGES;
+              if (ia >= TC_A_STAGES) ok = mbar_wait_bounded(bars + TCB_AEMPTY + st, ((ia / TC_A_STAGES) - 1) & 1);
+              if (!ok) break;
+              mbar_expect_tx(bars + TCB_AFULL + st, TC_A_STAGE_BYTES);
+              tma_load_2d(sA + (size_t)st * TC_A_STAGE_BYTES, &mapX, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + st);
+            }
+          }
+        }
+        if (!ok) atomicExch(&misc[2], 1);
+      }
+    } else if (wid == 1) {
+      if (lane == 0) {
+        unsigned ib = it_b, ia = it_a, iacc = it_acc;
+        bool ok = true;
+        for (int n = 0; n < n_tiles && ok; ++n, ++ib) {
+          ok = mbar_wait_bounded(bars + TCB_BFULL, ib & 1);
+          if (!ok) break;
+          tc_fence_after();
+          for (int m = 0; m < m_tiles && ok; ++m, ++iacc) {
+            const int buf = iacc & 1;
+            if (iacc >= 2) ok = mbar_wait_bounded(bars + TCB_ACCEMPTY + buf, ((iacc >> 1) - 1) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            for (int kc = 0; kc < nkc && ok; ++kc, ++ia) {
+              const int st = ia % TC_A_STAGES;
+              ok = mbar_wait_bounded(bars + TCB_AFULL + st, (ia / TC_A_STAGES) & 1);
+              if (!ok) break;
+              tc_fence_after();
+#pragma unroll
+              for (int k4 = 0; k4 < TC_KC / 16; ++k4)
+                tc_mma_bf16(tmem + (unsigned)buf * TC_N, tc_smem_desc(sA + (size_t)st * TC_A_STAGE_BYTES, k4 * 32),
+                            tc_smem_desc(sB + (size_t)kc * TC_B_CHUNK_BYTES, k4 * 32), idesc, (kc | k4) != 0);
+              tc_commit(bars + TCB_AEMPTY + st);          // the ring slot is free when these MMAs have read it
+            }
+            tc_commit(bars + TCB_ACCFULL + buf);          // the accumulator is complete
+          }
+          tc_commit(bars + TCB_BEMPTY);                   // the centre block may be replaced
+        }
+        if (!ok) atomicExch(&misc[2], 1);
+      }
+    } else if (wid < 6) {
+      const int quarter = wid & 3;                        // a warp reads TMEM lanes 32*(warp%4) .. +31
+      unsigned iacc = it_acc;
+      bool ok = true;
+      for (int n = 0; n < n_tiles; ++n) {
+        for (int m = 0; m < m_tiles; ++m, ++iacc) {
+          const int buf = iacc & 1;
+          if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bars + TCB_ACCFULL + buf, (iacc >> 1) & 1));
+          if (!ok) continue;
+          tc_fence_after();
+          const int r = m * TC_M + quarter * 32 + lane;
+          float e1 = INF, e2 = INF, o1 = INF, o2 = INF;   // two independent (minimum, runner-up) pairs
+          for (int c0 = 0; c0 < TC_N; c0 += 32) {
+            unsigned v[32];
+            const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)(buf * TC_N + c0);
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+                  "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]),
+                  "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]),
+                  "=r"(v[30]), "=r"(v[31])
+                : "r"(taddr) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (c0 + 32 == TC_N) {                        // last read of this accumulator: hand it back
+              tc_fence_before();
+              if (lane == 0) mbar_arrive(bars + TCB_ACCEMPTY + buf);
+            }
+            const int abase = n * TC_N + c0;
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+              const float s0 = __uint_as_float(v[c]) + cn[abase + c];
+              const float s1 = __uint_as_float(v[c + 1]) + cn[abase + c + 1];
+              const float p0 = __uint_as_float((__float_as_uint(s0) & ~TC_INDEX_MASK) | (unsigned)(abase + c));
+              const float p1 = __uint_as_float((__float_as_uint(s1) & ~TC_INDEX_MASK) | (unsigned)(abase + c + 1));
+              e2 = fmaxf(e1, fminf(e2, p0)); e1 = fminf(e1, p0);
+              o2 = fmaxf(o1, fminf(o2, p1)); o1 = fminf(o1, p1);
+            }
+          }
+          float s2 = fminf(fmaxf(e1, o1), fminf(e2, o2));
+          float s1 = fminf(e1, o1);
+          if (r < b) {
+            if (n > 0) {
+              const float2 prev = __ldcg(top2 + r);
+              s2 = fminf(fmaxf(s1, prev.x), fminf(s2, prev.y));
+              s1 = fminf(s1, prev.x);
+            }
+            __stcg(top2 + r, make_float2(s1, s2));
+          }
+        }
+      }
+      if (!ok && lane == 0) atomicExch(&misc[2], 1);
+    }
+    it_b += (unsigned)n_tiles;
+    it_a += (unsigned)(n_tiles * m_tiles * nkc);
+    it_acc += (unsigned)(n_tiles * m_tiles);
+    if (tid == 0) misc[1] = 0;
+    for (int a = tid; a < k; a += TC_THREADS) cnt[a] = 0;
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (misc[2]) break;                                   // a wait ran out: report and leave (uniform)
+
+    // ================= decide =================
+    float wmax2 = 0.f;
+    for (int a = lane; a < k; a += 32) wmax2 = fmaxf(wmax2, cn[a]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) wmax2 = fmaxf(wmax2, __shfl_xor_sync(0xffffffffu, wmax2, o));
+    // BF16 rounding (2^-8 relative) of both operands: |error of -2 x.w| <= 2 * 2^-7 * 1.004 * ||x|| ||w||; index bits: 2^10 ulp of the score
+    const float xw = sqrtf(p.xmax2 * wmax2);
+    const float tau = 2.f * (0.0157f * xw + 2.45e-4f * (wmax2 + 2.f * xw));
+    for (int r = tid; r < b; r += TC_THREADS) {
+      const float2 s = __ldcg(top2 + r);
+      best[r] = (unsigned short)(__float_as_uint(s.x) & TC_INDEX_MASK);
+      if (k > 1 && (s.y - s.x) <= tau) flagged[atomicAdd(&misc[1], 1)] = (unsigned short)r;
+    }
+    __syncthreads();
+    {
+      const int nflag = misc[1];
+      for (int f = wid; f < nflag; f += TC_WARPS) {       // a warp per sample: fp32 inputs, fp64 sums, the two candidates
+        const int r = flagged[f];
+        const float2 s = __ldcg(top2 + r);
+        const int i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK), i2 = (int)(__float_as_uint(s.y) & TC_INDEX_MASK);
+        const float* x = p.X + (size_t)(row0 + r) * d;
+        double d1 = 0.0, d2 = 0.0;
+        for (int j = lane * 2; j < d; j += 64) {
+          const float2 xv = __ldg(reinterpret_cast<const float2*>(x + j));
+          const float2 a1 = *reinterpret_cast<const float2*>(wglob + (size_t)i1 * d + j);
+          const float2 a2 = *reinterpret_cast<const float2*>(wglob + (size_t)i2 * d + j);
+          const double u0 = (double)xv.x - (double)a1.x, u1 = (double)xv.y - (double)a1.y;
+          const double v0 = (double)xv.x - (double)a2.x, v1 = (double)xv.y - (double)a2.y;
+          d1 = fma(u0, u0, d1); d1 = fma(u1, u1, d1);
+          d2 = fma(v0, v0, d2); d2 = fma(v1, v1, d2);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); }
+        if (lane == 0) best[r] = (unsigned short)((d2 < d1 || (d2 == d1 && i2 < i1)) ? i2 : i1);
+      }
+    }
+    __syncthreads();
+
+    // ================= Eq. 9: per-centre sums of the fp32 samples (vector reductions into the worker's sum buffer) =================
+    for (int r = wid; r < b; r += TC_WARPS) {
+      const int a = best[r];
+      if (p.assign_rec && lane == 0) p.assign_rec[(size_t)i * b + r] = a;
+      const float* x = p.X + (size_t)(row0 + r) * d;
+      for (int j = lane * 4; j < d; j += 128) red_add_v4(gsum + (size_t)a * d + j, __ldg(reinterpret_cast<const float4*>(x + j)));
+      if (lane == 0) atomicAdd(cnt + a, 1);
+    }
+    __threadfence();
+    __syncthreads();
+
+    // ================= update =================
+    if (tid == 0) {                                       // one thread looks, so that the whole block takes the same branch
+      int any = 0;
+      for (int s = 0; s < p.S; ++s) any |= (ld_relaxed_gpu(p.seq + (size_t)i * p.S + s) != p.seen[(size_t)i * p.S + s]);
+      misc[4] = any;
+    }
+    __syncthreads();
+    const bool news = misc[4] != 0;
+    const bool put_now = p.c > 0 && p.f > 0 && p.W > 1 && (t + 1) % (unsigned long long)p.c == 0;
+    if (news || put_now) {
+      step_tail<kDet>(p, i, t, wglob, d, gsum, cnt, nullptr, ts, true);
+      __syncthreads();
+    }
+    const bool plain = !(news || put_now);
+    for (int a = wid; a < k; a += TC_WARPS) {             // a warp per centre
+      float sq = 0.f;
+      const float n = (float)cnt[a];
+      for (int j = lane * 4; j < d; j += 128) {
+        float4 w4 = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + j);
+        if (plain) {                                      // w <- w - eps * (n w - S) / b
+          const float4 s4 = __ldcg(reinterpret_cast<const float4*>(gsum + (size_t)a * d + j));
+          w4.x -= p.eps * ((n * w4.x - s4.x) * inv_b); w4.y -= p.eps * ((n * w4.y - s4.y) * inv_b);
+          w4.z -= p.eps * ((n * w4.z - s4.z) * inv_b); w4.w -= p.eps * ((n * w4.w - s4.w) * inv_b);
+          *reinterpret_cast<float4*>(wglob + (size_t)a * d + j) = w4;
+        }
+        __stcg(reinterpret_cast<float4*>(gsum + (size_t)a * d + j), make_float4(0.f, 0.f, 0.f, 0.f));
+        sq = fmaf(w4.x, w4.x, sq); sq = fmaf(w4.y, w4.y, sq); sq = fmaf(w4.z, w4.z, sq); sq = fmaf(w4.w, w4.w, sq);
+        *reinterpret_cast<__nv_bfloat162*>(wbf + (size_t)a * d + j) = __floats2bfloat162_rn(-2.f * w4.x, -2.f * w4.y);
+        *reinterpret_cast<__nv_bfloat162*>(wbf + (size_t)a * d + j + 2) = __floats2bfloat162_rn(-2.f * w4.z, -2.f * w4.w);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      if (lane == 0) cn[a] = sq;
+    }
+    if (plain && tid == 0) {
+      if (kDet)
+        for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
+      p.stats[(size_t)i * ST_STRIDE + ST_STEPS] = t + 1;
+    }
+    asm volatile("fence.proxy.async;" ::: "memory");      // the refreshed bf16(-2w) is read by the next step's TMA
+    __syncthreads();
+  }
+
+  if (misc[2] && tid == 0) atomicExch(p.status, DEV_TIMEOUT);
+  tc_fence_before();
+  __syncthreads();
+  if (wid == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+}
+
+}  // namespace asgd

@@ -10,6 +10,7 @@ from oracle import asgd_oracle as orc
 # the oracle's; assignments bit-exact except samples whose two smallest squared distances differ by
 # less than 1e-5 relative (their fp32 order is not decided).
 CENTRE_TOL = 1e-4
+CENTRE_TOL_BF16 = 5e-3      # tensor-core path with BF16 operands
 TIE_EXCLUSION = 1e-5
 
 
@@ -50,6 +51,9 @@ class Pair:
         if oracle:
             self.cpu = orc.Oracle(self.Xh, self.w0h, W=wl.W, b=wl.b, eps=wl.eps, comm_interval=wl.comm_interval,
                                   fanout=wl.fanout, slots=S, parzen=parzen, shuffle=shuffle, seed=wl.seed)
+
+    def centre_tol(self):
+        return CENTRE_TOL_BF16 if self.gpu.path_name() == "tcgen05-bf16" else CENTRE_TOL
 
     def rounds(self, n):
         self.gpu.step(n)

@@ -7,7 +7,7 @@ import torch
 
 import paper_1505_04956_b200 as pkg
 from oracle import asgd_oracle as orc
-from tests.gpu_util import CENTRE_TOL, PARITY_WORKLOADS, Pair, decided, scaled
+from tests.gpu_util import CENTRE_TOL, CENTRE_TOL_BF16, PARITY_WORKLOADS, Pair, decided, scaled
 
 pytestmark = pytest.mark.gpu
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
@@ -39,7 +39,7 @@ def test_trajectory_matches_oracle(name):
         pr.rounds(n)
         done += n
         pr.gpu.sync()
-        assert pr.max_rel_l2() < CENTRE_TOL, (name, done, pr.max_rel_l2())
+        assert pr.max_rel_l2() < pr.centre_tol(), (name, done, pr.max_rel_l2())
         for i in range(wl.W):
             tr = pr.cpu.last_step(i)
             acc = pr.gpu.get_accept(i)
@@ -72,16 +72,27 @@ def test_single_step_assignments_bit_exact(name):
     pr.rounds(1)
     pr.gpu.sync()
     got = pr.gpu.get_assign().cpu().numpy()
+    bf16 = pr.gpu.path_name() == "tcgen05-bf16"
     checked = 0
     for i in range(wl.W):
         tr = pr.cpu.last_step(i)
         ok = decided(tr["d1"], tr["d2"])
-        assert (got[i][ok] == tr["assign"][ok]).all(), (name, i)
+        if bf16:
+            # BF16 operands: a score is off by at most 2 * 2^-7 * 1.004 * ||x|| ||w|| (+ index bits); the kernel settles
+            # the two best exactly, so only samples with a third centre inside that bound may differ
+            w = pr.cpu.state(i).astype(np.float64)
+            xw = np.sqrt((pr.Xh.astype(np.float64) ** 2).sum(1).max() * (w ** 2).sum(1).max())
+            tau = 2 * (0.0157 * xw + 2.45e-4 * ((w ** 2).sum(1).max() + 2 * xw))
+            wrong = ok & (got[i] != tr["assign"])
+            assert wrong.mean() < 0.01, (name, i, wrong.mean())
+            assert ((tr["d2"] - tr["d1"])[wrong] <= tau).all()
+        else:
+            assert (got[i][ok] == tr["assign"][ok]).all(), (name, i)
+            if ok.all():
+                assert np.bincount(got[i], minlength=wl.k).tolist() == tr["counts"].tolist()
         checked += int(ok.sum())
-        if ok.all():
-            assert np.bincount(got[i], minlength=wl.k).tolist() == tr["counts"].tolist()
     assert checked >= 0.99 * wl.W * wl.b
-    assert pr.max_rel_l2() < CENTRE_TOL
+    assert pr.max_rel_l2() < pr.centre_tol()
     pr.close()
 
 
@@ -128,6 +139,9 @@ EDGE_CASES = {
     "tiled_32_many_workers": dict(N=700 * 12, d=32, k=8, W=700, b=4, comm_interval=1, fanout=1),
     "tiled_128_k128": dict(N=3 * 200 * 2, d=128, k=128, W=3, b=200, comm_interval=1, fanout=1),
     "tiled_128_k5_tiny_batch": dict(N=4 * 7 * 3, d=128, k=5, W=4, b=7, comm_interval=1, fanout=3),
+    # shapes of the tensor-core kernel: a centre block that is not full, one K chunk, a ragged last sample tile
+    "tc_d64_k300_ragged": dict(N=3 * 200 * 3 + 5, d=64, k=300, W=3, b=200, comm_interval=2, fanout=1),
+    "tc_d128_k129": dict(N=2 * 128 * 4, d=128, k=129, W=2, b=128, comm_interval=1, fanout=1),
     "general_10x10_big_batch": dict(N=2 * 700 * 3, d=10, k=10, W=2, b=700, comm_interval=2, fanout=1),
 }
 
@@ -142,7 +156,7 @@ def test_edge_cases(case, parzen):
     rounds = 2 * wl.B + 3
     pr.rounds(rounds)
     pr.gpu.sync()
-    assert pr.max_rel_l2() < CENTRE_TOL, (case, pr.max_rel_l2())
+    assert pr.max_rel_l2() < pr.centre_tol(), (case, pr.max_rel_l2())
     _compare_stats(pr, exact_accept=(parzen == 0))
     pr.close()
 
@@ -161,6 +175,16 @@ def test_specialised_and_general_kernels_agree():
         assert a.gpu.get_stats(i) == g.gpu.get_stats(i)
     a.close()
     g.close()
+
+
+def test_dense_shape_on_the_fp32_kernel_too():
+    wl, rounds = PARITY_WORKLOADS["dense"]
+    pr = Pair(wl, dist_path=pkg.PATH_FP32_GENERAL)
+    assert pr.gpu.path_name().startswith("fp32-generic")
+    pr.rounds(rounds)
+    pr.gpu.sync()
+    assert pr.max_rel_l2() < CENTRE_TOL
+    pr.close()
 
 
 def test_unshuffled_batches_and_many_slots():
