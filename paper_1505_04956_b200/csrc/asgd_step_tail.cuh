@@ -21,26 +21,54 @@ struct TailScratch {
   int m;
 };
 
+// V floats at a time (V = 4: 128-bit accesses).
+template <int V> struct TailVec { float v[V]; };
+template <int V> __device__ inline TailVec<V> tail_ld(const float* q) {
+  TailVec<V> r;
+  if (V == 4) { const float4 t = *reinterpret_cast<const float4*>(q); r.v[0] = t.x; r.v[V > 1 ? 1 : 0] = t.y; r.v[V > 2 ? 2 : 0] = t.z; r.v[V > 3 ? 3 : 0] = t.w; }
+  else r.v[0] = *q;
+  return r;
+}
+template <int V> __device__ inline TailVec<V> tail_ldcg(const float* q) {
+  TailVec<V> r;
+  if (V == 4) { const float4 t = __ldcg(reinterpret_cast<const float4*>(q)); r.v[0] = t.x; r.v[V > 1 ? 1 : 0] = t.y; r.v[V > 2 ? 2 : 0] = t.z; r.v[V > 3 ? 3 : 0] = t.w; }
+  else r.v[0] = __ldcg(q);
+  return r;
+}
+template <int V> __device__ inline void tail_st(float* q, const TailVec<V>& r) {
+  if (V == 4) *reinterpret_cast<float4*>(q) = make_float4(r.v[0], r.v[V > 1 ? 1 : 0], r.v[V > 2 ? 2 : 0], r.v[V > 3 ? 3 : 0]);
+  else *q = r.v[0];
+}
+
 // w     [k rows of d, row stride wstride]  this worker's state (shared or global memory), updated in place
 // SD    [kd]  in: per-centre sums S_k of the mini-batch; out: the local gradient D
 // cnt   [k]   per-centre counts n_k
 // wglob       the worker's row of Params::state when w lives in shared memory, else nullptr
-// sd_l2   the sums in SD were produced by reductions in L2: read them past L1
-template <bool kDet>
-__device__ inline void step_tail(const Params& p, int i, unsigned long long t, float* w, int wstride, float* SD,
-                                 const int* cnt, float* wglob, TailScratch* ts, bool sd_l2 = false) {
+// sd_l2       the sums in SD were produced by reductions in L2: read them past L1
+// V           elements per access; V = 4 needs d % 4 == 0 and 16-byte aligned w, SD, wglob rows
+template <bool kDet, int V>
+__device__ inline void step_tail_impl(const Params& p, int i, unsigned long long t, float* __restrict__ w, int wstride,
+                                      float* __restrict__ SD, const int* __restrict__ cnt, float* __restrict__ wglob,
+                                      TailScratch* ts, bool sd_l2) {
   const int tid = threadIdx.x, nt = blockDim.x;
   const int kd = p.kd, d = p.d;
+  const int nvec = kd / V;                                  // V divides d, so an access never straddles two centres
   const bool dense_rows = (wstride == d);
   auto widx = [&](int e) { return dense_rows ? e : (e / d) * wstride + (e % d); };
   const float inv_b = 1.0f / (float)p.b;
   const float eps = p.eps;
 
   // Eq. 9 (true-gradient sign, mean over the mini-batch size): D_k = (n_k w_k - S_k) / b
-  for (int e = tid; e < kd; e += nt) {
-    const int a = e / d;
-    const float sums = sd_l2 ? __ldcg(SD + e) : SD[e];
-    SD[e] = ((float)cnt[a] * w[widx(e)] - sums) * inv_b;
+#pragma unroll 2
+  for (int q = tid; q < nvec; q += nt) {
+    const int e = q * V;
+    const float n = (float)cnt[e / d];
+    const TailVec<V> sums = sd_l2 ? tail_ldcg<V>(SD + e) : tail_ld<V>(SD + e);
+    const TailVec<V> ww = tail_ld<V>(w + widx(e));
+    TailVec<V> D;
+#pragma unroll
+    for (int u = 0; u < V; ++u) D.v[u] = (n * ww.v[u] - sums.v[u]) * inv_b;
+    tail_st<V>(SD + e, D);
   }
   __syncthreads();
 
@@ -64,15 +92,21 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
     const bool fresh = ts->fresh[s] != 0;
     int acc = -1;
     if (fresh) {
-      const float* v = p.mail + si * (size_t)p.kd_pad;
+      const float* __restrict__ v = p.mail + si * (size_t)p.kd_pad;
       double dot = 0.0, dd = 0.0, nv = 0.0;
-      for (int e = tid; e < kd; e += nt) {
-        const float vv = __ldcg(v + e);
-        const float D = SD[e];
-        const float df = w[widx(e)] - vv;
-        dot += (double)D * (double)df;
-        dd += (double)D * (double)D;
-        nv += (double)vv * (double)vv;
+#pragma unroll 2
+      for (int q = tid; q < nvec; q += nt) {
+        const int e = q * V;
+        const TailVec<V> vv = tail_ldcg<V>(v + e);
+        const TailVec<V> D = tail_ld<V>(SD + e);
+        const TailVec<V> ww = tail_ld<V>(w + widx(e));
+#pragma unroll
+        for (int u = 0; u < V; ++u) {
+          const float df = ww.v[u] - vv.v[u];
+          dot += (double)D.v[u] * (double)df;
+          dd += (double)D.v[u] * (double)D.v[u];
+          nv += (double)vv.v[u] * (double)vv.v[u];
+        }
       }
       block_sum3(dot, dd, nv, ts->red);
       // Eq. 4 expanded: ||(w - eps D) - v||^2 < ||w - v||^2  <=>  2 <D, w - v> > eps ||D||^2
@@ -86,16 +120,29 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
 
   // Eq. 6: Dbar = w - (w + sum_s a_s v_s) / (1 + sum_s a_s) + D ;  w <- w - eps * Dbar
   const float inv_m1 = 1.0f / (float)(1 + m);
-  for (int e = tid; e < kd; e += nt) {
-    float sumv = 0.f;
+#pragma unroll 2
+  for (int q = tid; q < nvec; q += nt) {
+    const int e = q * V;
+    TailVec<V> sumv;
+#pragma unroll
+    for (int u = 0; u < V; ++u) sumv.v[u] = 0.f;
     for (int s = 0; s < p.S; ++s)
-      if (ts->accept[s] == 1) sumv += __ldcg(p.mail + ((size_t)i * p.S + s) * (size_t)p.kd_pad + e);
+      if (ts->accept[s] == 1) {
+        const TailVec<V> vv = tail_ldcg<V>(p.mail + ((size_t)i * p.S + s) * (size_t)p.kd_pad + e);
+#pragma unroll
+        for (int u = 0; u < V; ++u) sumv.v[u] += vv.v[u];
+      }
     const int we = widx(e);
-    const float ww = w[we];
-    const float Dbar = (ww - (ww + sumv) * inv_m1) + SD[e];
-    const float nw = ww - eps * Dbar;
-    w[we] = nw;
-    if (wglob) wglob[e] = nw;
+    const TailVec<V> ww = tail_ld<V>(w + we);
+    const TailVec<V> D = tail_ld<V>(SD + e);
+    TailVec<V> nw;
+#pragma unroll
+    for (int u = 0; u < V; ++u) {
+      const float Dbar = (ww.v[u] - (ww.v[u] + sumv.v[u]) * inv_m1) + D.v[u];
+      nw.v[u] = ww.v[u] - eps * Dbar;
+    }
+    tail_st<V>(w + we, nw);
+    if (wglob) tail_st<V>(wglob + e, nw);
   }
   __syncthreads();
 
@@ -121,7 +168,8 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
       for (int j = 0; j < p.f; ++j) {
         const size_t ri = (size_t)ts->peers[j] * p.S + ts->pslots[j];
         float* dst = p.mail + ri * (size_t)p.kd_pad;
-        for (int e = tid; e < kd; e += nt) dst[e] = w[widx(e)];
+#pragma unroll 2
+        for (int q = tid; q < nvec; q += nt) tail_st<V>(dst + q * V, tail_ld<V>(w + widx(q * V)));
         __syncthreads();
         if (tid == 0) red_release_gpu_inc(p.seq + ri);
       }
@@ -135,6 +183,15 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
     if (n_sent) atomicAdd(st + ST_SENT, n_sent);
     if (m) atomicAdd(st + ST_ACCEPT, (unsigned long long)m);
   }
+}
+
+// Picks 128-bit accesses when the layout allows it.
+template <bool kDet>
+__device__ inline void step_tail(const Params& p, int i, unsigned long long t, float* w, int wstride, float* SD,
+                                 const int* cnt, float* wglob, TailScratch* ts, bool sd_l2 = false) {
+  const bool vec = (p.d % 4 == 0) && (wstride % 4 == 0) && ((((size_t)w) | ((size_t)SD) | ((size_t)wglob)) & 15) == 0;
+  if (vec) step_tail_impl<kDet, 4>(p, i, t, w, wstride, SD, cnt, wglob, ts, sd_l2);
+  else step_tail_impl<kDet, 1>(p, i, t, w, wstride, SD, cnt, wglob, ts, sd_l2);
 }
 
 }  // namespace asgd

@@ -293,82 +293,197 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     // BF16 rounding (2^-8 relative) of both operands: |error of -2 x.w| <= 2 * 2^-7 * 1.004 * ||x|| ||w||; index bits: 2^10 ulp of the score
     const float xw = sqrtf(p.xmax2 * wmax2);
     const float tau = 2.f * (0.0157f * xw + 2.45e-4f * (wmax2 + 2.f * xw));
-    for (int r = tid; r < b; r += TC_THREADS) {
-      const float2 s = __ldcg(top2 + r);
-      best[r] = (unsigned short)(__float_as_uint(s.x) & TC_INDEX_MASK);
-      if (k > 1 && (s.y - s.x) <= tau) flagged[atomicAdd(&misc[1], 1)] = (unsigned short)r;
-    }
-    __syncthreads();
-    {
-      const int nflag = misc[1];
-      for (int f = wid; f < nflag; f += TC_WARPS) {       // a warp per sample: fp32 inputs, fp64 sums, the two candidates
-        const int r = flagged[f];
-        const float2 s = __ldcg(top2 + r);
-        const int i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK), i2 = (int)(__float_as_uint(s.y) & TC_INDEX_MASK);
-        const float* x = p.X + (size_t)(row0 + r) * d;
-        double d1 = 0.0, d2 = 0.0;
-        for (int j = lane * 2; j < d; j += 64) {
-          const float2 xv = __ldg(reinterpret_cast<const float2*>(x + j));
-          const float2 a1 = *reinterpret_cast<const float2*>(wglob + (size_t)i1 * d + j);
-          const float2 a2 = *reinterpret_cast<const float2*>(wglob + (size_t)i2 * d + j);
-          const double u0 = (double)xv.x - (double)a1.x, u1 = (double)xv.y - (double)a1.y;
-          const double v0 = (double)xv.x - (double)a2.x, v1 = (double)xv.y - (double)a2.y;
-          d1 = fma(u0, u0, d1); d1 = fma(u1, u1, d1);
-          d2 = fma(v0, v0, d2); d2 = fma(v1, v1, d2);
-        }
+    // Scratch for the rest of the step lives in the sample ring, which is idle until the next step's loads.
+    int* wcnt = reinterpret_cast<int*>(sA);                                   // [TC_WARPS][k] rows of a centre in a warp's row block
+    unsigned short* lrank = reinterpret_cast<unsigned short*>(sA + (size_t)TC_WARPS * k * 4);   // [b] rank of a row among its warp's rows of the centre
+    unsigned short* order = flagged;                                          // [b] rows grouped by centre, ascending inside a group
+    const int sub = lane >> 3, l8 = lane & 7;                                 // eight lanes share a row or a centre
+    const int nq = d / 32;
+
+    // ---- decide: a row whose two best scores are closer than the bound is settled between those two
+    //      centres with fp32 inputs and fp64 sums (lane l8 holds dimensions 4*l8 + 32*q) ----
+    for (int e = tid; e < TC_WARPS * k; e += TC_THREADS) wcnt[e] = 0;
+    for (int base = wid * 4; base < b; base += TC_WARPS * 4) {
+      const int r = base + sub;
+      const bool valid = r < b;
+      const float2 s = valid ? __ldcg(top2 + r) : make_float2(0.f, INF);
+      const int i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK), i2 = (int)(__float_as_uint(s.y) & TC_INDEX_MASK);
+      const bool flag = valid && k > 1 && (s.y - s.x) <= tau;
+      double d1 = 0.0, d2 = 0.0;
+      if (flag) {
+        const float* x = p.X + (size_t)(row0 + r) * d + 4 * l8;
+        const float* w1 = wglob + (size_t)i1 * d + 4 * l8;
+        const float* w2 = wglob + (size_t)i2 * d + 4 * l8;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) { d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); }
-        if (lane == 0) best[r] = (unsigned short)((d2 < d1 || (d2 == d1 && i2 < i1)) ? i2 : i1);
+        for (int q = 0; q < TC_MAX_D / 32; ++q) {
+          if (q < nq) {
+            const float4 xv = __ldg(reinterpret_cast<const float4*>(x + 32 * q));
+            const float4 a1 = *reinterpret_cast<const float4*>(w1 + 32 * q);
+            const float4 a2 = *reinterpret_cast<const float4*>(w2 + 32 * q);
+            double u;
+            u = (double)xv.x - (double)a1.x; d1 = fma(u, u, d1); u = (double)xv.y - (double)a1.y; d1 = fma(u, u, d1);
+            u = (double)xv.z - (double)a1.z; d1 = fma(u, u, d1); u = (double)xv.w - (double)a1.w; d1 = fma(u, u, d1);
+            u = (double)xv.x - (double)a2.x; d2 = fma(u, u, d2); u = (double)xv.y - (double)a2.y; d2 = fma(u, u, d2);
+            u = (double)xv.z - (double)a2.z; d2 = fma(u, u, d2); u = (double)xv.w - (double)a2.w; d2 = fma(u, u, d2);
+          }
+        }
+      }
+#pragma unroll
+      for (int o = 1; o < 8; o <<= 1) { d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); }
+      if (valid && l8 == 0) {
+        const int bst = (flag && (d2 < d1 || (d2 == d1 && i2 < i1))) ? i2 : i1;
+        best[r] = (unsigned short)bst;
+        if (p.assign_rec) p.assign_rec[(size_t)i * b + r] = bst;
       }
     }
     __syncthreads();
 
-    // ================= Eq. 9: per-centre sums of the fp32 samples (vector reductions into the worker's sum buffer) =================
-    for (int r = wid; r < b; r += TC_WARPS) {
-      const int a = best[r];
-      if (p.assign_rec && lane == 0) p.assign_rec[(size_t)i * b + r] = a;
-      const float* x = p.X + (size_t)(row0 + r) * d;
-      for (int j = lane * 4; j < d; j += 128) red_add_v4(gsum + (size_t)a * d + j, __ldg(reinterpret_cast<const float4*>(x + j)));
-      if (lane == 0) atomicAdd(cnt + a, 1);
+    // ---- rows grouped by centre, in row order (stable): ranks inside each warp's block of rows, then offsets ----
+    {
+      const int R = ((b + TC_WARPS - 1) / TC_WARPS + 31) / 32 * 32;           // rows per warp, whole chunks of 32
+      int* mine = wcnt + wid * k;
+      for (int r0 = wid * R; r0 < min(b, (wid + 1) * R); r0 += 32) {
+        const int r = r0 + lane;
+        const int a = (r < b) ? (int)best[r] : -1;
+        const unsigned grp = __match_any_sync(0xffffffffu, a);
+        const unsigned below = grp & ((1u << lane) - 1u);
+        const int lead = __ffs(grp) - 1;
+        int base = 0;
+        if (a >= 0 && below == 0) { base = mine[a]; mine[a] = base + __popc(grp); }
+        base = __shfl_sync(0xffffffffu, base, lead);
+        if (a >= 0) lrank[r] = (unsigned short)(base + __popc(below));
+        __syncwarp();
+      }
     }
-    __threadfence();
     __syncthreads();
-
-    // ================= update =================
+    // per centre: total count, then start = exclusive prefix over centres (block scan of k <= 1024 values)
+    {
+      int tot[4], run = 0;
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int a = tid * 4 + u;
+        int c = 0;
+        if (a < k)
+          for (int w8 = 0; w8 < TC_WARPS; ++w8) { const int v = wcnt[w8 * k + a]; wcnt[w8 * k + a] = c; c += v; }   // per-warp offsets
+        tot[u] = c;
+        run += c;
+      }
+      int incl = run;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += y; }
+      int* wsum = reinterpret_cast<int*>(ts->red);
+      if (lane == 31) wsum[wid] = incl;
+      __syncthreads();
+      int before = incl - run;
+      for (int w8 = 0; w8 < wid; ++w8) before += wsum[w8];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int a = tid * 4 + u;
+        if (a < k) { cnt[a] = tot[u]; reinterpret_cast<int*>(sB)[a] = before; }      // start[a] (the centre block is idle too)
+        before += tot[u];
+      }
+    }
+    __syncthreads();
+    {
+      const int* start = reinterpret_cast<const int*>(sB);
+      const int R = ((b + TC_WARPS - 1) / TC_WARPS + 31) / 32 * 32;
+      for (int r = tid; r < b; r += TC_THREADS) {
+        const int a = best[r];
+        order[start[a] + wcnt[(r / R) * k + a] + lrank[r]] = (unsigned short)r;
+      }
+    }
     if (tid == 0) {                                       // one thread looks, so that the whole block takes the same branch
       int any = 0;
       for (int s = 0; s < p.S; ++s) any |= (ld_relaxed_gpu(p.seq + (size_t)i * p.S + s) != p.seen[(size_t)i * p.S + s]);
       misc[4] = any;
     }
     __syncthreads();
-    const bool news = misc[4] != 0;
     const bool put_now = p.c > 0 && p.f > 0 && p.W > 1 && (t + 1) % (unsigned long long)p.c == 0;
-    if (news || put_now) {
-      step_tail<kDet>(p, i, t, wglob, d, gsum, cnt, nullptr, ts, true);
-      __syncthreads();
-    }
-    const bool plain = !(news || put_now);
-    for (int a = wid; a < k; a += TC_WARPS) {             // a warp per centre
+    const bool plain = !(misc[4] != 0 || put_now);
+
+    // ---- Eq. 9 and the update: eight lanes per centre add its rows (fp32 master, ascending row order);
+    //      plain step: w <- w - eps (n w - S) / b at once; otherwise S goes to the sum buffer for the general tail ----
+    auto refresh = [&](int a, const float4 (&w4)[TC_MAX_D / 32]) {           // bf16(-2w), ||w||^2 of one centre
       float sq = 0.f;
-      const float n = (float)cnt[a];
-      for (int j = lane * 4; j < d; j += 128) {
-        float4 w4 = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + j);
-        if (plain) {                                      // w <- w - eps * (n w - S) / b
-          const float4 s4 = __ldcg(reinterpret_cast<const float4*>(gsum + (size_t)a * d + j));
-          w4.x -= p.eps * ((n * w4.x - s4.x) * inv_b); w4.y -= p.eps * ((n * w4.y - s4.y) * inv_b);
-          w4.z -= p.eps * ((n * w4.z - s4.z) * inv_b); w4.w -= p.eps * ((n * w4.w - s4.w) * inv_b);
-          *reinterpret_cast<float4*>(wglob + (size_t)a * d + j) = w4;
-        }
-        __stcg(reinterpret_cast<float4*>(gsum + (size_t)a * d + j), make_float4(0.f, 0.f, 0.f, 0.f));
-        sq = fmaf(w4.x, w4.x, sq); sq = fmaf(w4.y, w4.y, sq); sq = fmaf(w4.z, w4.z, sq); sq = fmaf(w4.w, w4.w, sq);
-        *reinterpret_cast<__nv_bfloat162*>(wbf + (size_t)a * d + j) = __floats2bfloat162_rn(-2.f * w4.x, -2.f * w4.y);
-        *reinterpret_cast<__nv_bfloat162*>(wbf + (size_t)a * d + j + 2) = __floats2bfloat162_rn(-2.f * w4.z, -2.f * w4.w);
-      }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-      if (lane == 0) cn[a] = sq;
+      for (int q = 0; q < TC_MAX_D / 32; ++q) {
+        if (q < nq) {
+          sq = fmaf(w4[q].x, w4[q].x, sq); sq = fmaf(w4[q].y, w4[q].y, sq); sq = fmaf(w4[q].z, w4[q].z, sq); sq = fmaf(w4[q].w, w4[q].w, sq);
+          __nv_bfloat16* o = wbf + (size_t)a * d + 4 * l8 + 32 * q;
+          *reinterpret_cast<__nv_bfloat162*>(o) = __floats2bfloat162_rn(-2.f * w4[q].x, -2.f * w4[q].y);
+          *reinterpret_cast<__nv_bfloat162*>(o + 2) = __floats2bfloat162_rn(-2.f * w4[q].z, -2.f * w4[q].w);
+        }
+      }
+      return sq;
+    };
+    {
+      const int* start = reinterpret_cast<const int*>(sB);
+      for (int a0 = (wid * 4) ; a0 < k; a0 += TC_WARPS * 4) {
+        const int a = a0 + sub;
+        const bool on = a < k;
+        const int n = on ? cnt[a] : 0, p0 = on ? start[a] : 0;
+        float4 S4[TC_MAX_D / 32];
+#pragma unroll
+        for (int q = 0; q < TC_MAX_D / 32; ++q) S4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int e = 0; e < n; ++e) {
+          const float* x = p.X + (size_t)(row0 + order[p0 + e]) * d + 4 * l8;
+#pragma unroll
+          for (int q = 0; q < TC_MAX_D / 32; ++q) {
+            if (q < nq) {
+              const float4 v = __ldg(reinterpret_cast<const float4*>(x + 32 * q));
+              S4[q].x += v.x; S4[q].y += v.y; S4[q].z += v.z; S4[q].w += v.w;
+            }
+          }
+        }
+        float sq = 0.f;
+        if (on) {
+          if (plain) {
+            float4 w4[TC_MAX_D / 32];
+            const float fn = (float)n;
+#pragma unroll
+            for (int q = 0; q < TC_MAX_D / 32; ++q) {
+              if (q < nq) {
+                float* wp = wglob + (size_t)a * d + 4 * l8 + 32 * q;
+                float4 u = *reinterpret_cast<const float4*>(wp);
+                u.x -= p.eps * ((fn * u.x - S4[q].x) * inv_b); u.y -= p.eps * ((fn * u.y - S4[q].y) * inv_b);
+                u.z -= p.eps * ((fn * u.z - S4[q].z) * inv_b); u.w -= p.eps * ((fn * u.w - S4[q].w) * inv_b);
+                *reinterpret_cast<float4*>(wp) = u;
+                w4[q] = u;
+              }
+            }
+            sq = refresh(a, w4);
+          } else {
+#pragma unroll
+            for (int q = 0; q < TC_MAX_D / 32; ++q)
+              if (q < nq) *reinterpret_cast<float4*>(gsum + (size_t)a * d + 4 * l8 + 32 * q) = S4[q];
+          }
+        }
+        if (plain) {
+#pragma unroll
+          for (int o = 1; o < 8; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+          if (on && l8 == 0) cn[a] = sq;
+        }
+      }
     }
-    if (plain && tid == 0) {
+    if (!plain) {
+      __syncthreads();
+      step_tail<kDet>(p, i, t, wglob, d, gsum, cnt, nullptr, ts, false);
+      __syncthreads();
+      for (int a0 = wid * 4; a0 < k; a0 += TC_WARPS * 4) {
+        const int a = a0 + sub;
+        float sq = 0.f;
+        if (a < k) {
+          float4 w4[TC_MAX_D / 32];
+#pragma unroll
+          for (int q = 0; q < TC_MAX_D / 32; ++q)
+            if (q < nq) w4[q] = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q);
+          sq = refresh(a, w4);
+        }
+#pragma unroll
+        for (int o = 1; o < 8; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        if (a < k && l8 == 0) cn[a] = sq;
+      }
+    } else if (tid == 0) {
       if (kDet)
         for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
       p.stats[(size_t)i * ST_STRIDE + ST_STEPS] = t + 1;
