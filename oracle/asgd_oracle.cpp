@@ -247,6 +247,16 @@ extern "C" {
 uint64_t oracle_sm64(uint64_t x) { return sm64(x); }
 uint64_t oracle_draw(uint64_t seed, uint64_t tag, uint64_t a, uint64_t b, uint64_t c) { return draw(seed, tag, a, b, c); }
 
+// Batch order of one worker without building a whole oracle (same draws as make_perm).
+void oracle_batch_order(uint64_t seed, int32_t shuffle, int32_t worker, int64_t B, int32_t* out) {
+  Config c{};
+  c.seed = seed;
+  c.shuffle = shuffle;
+  std::vector<int32_t> perm;
+  make_perm(c, B, worker, perm);
+  std::memcpy(out, perm.data(), sizeof(int32_t) * (size_t)B);
+}
+
 void* oracle_create(int64_t N, int32_t d, int32_t k, int32_t W, int32_t b, float eps,
                     int32_t comm_interval, int32_t fanout, int32_t slots, int32_t parzen,
                     int32_t shuffle, uint64_t seed, const float* X, const float* w0) {

@@ -35,6 +35,7 @@ def lib():
         L.oracle_sm64.argtypes = [u64]
         L.oracle_draw.restype = u64
         L.oracle_draw.argtypes = [u64] * 5
+        L.oracle_batch_order.argtypes = [u64, i32, i32, i64, vp]
         L.oracle_create.restype = vp
         L.oracle_create.argtypes = [i64, i32, i32, i32, i32, f32, i32, i32, i32, i32, i32, u64, vp, vp]
         L.oracle_destroy.argtypes = [vp]
@@ -76,6 +77,13 @@ def sm64(x: int) -> int:
 
 def draw(seed: int, tag: int, a: int, b: int, c: int) -> int:
     return lib().oracle_draw(seed, tag, a, b, c)
+
+
+def batch_order(seed: int, worker: int, B: int, shuffle: int = 1):
+    """The worker's seeded order of its B mini-batches (Algorithm 5: shuffle, then draw in turn)."""
+    out = np.empty(B, np.int32)
+    lib().oracle_batch_order(int(seed), int(shuffle), int(worker), int(B), _p(out))
+    return out
 
 
 def assign(X, w):
