@@ -59,7 +59,7 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
   const float eps = p.eps;
 
   // Eq. 9 (true-gradient sign, mean over the mini-batch size): D_k = (n_k w_k - S_k) / b
-#pragma unroll 2
+#pragma unroll 4
   for (int q = tid; q < nvec; q += nt) {
     const int e = q * V;
     const float n = (float)cnt[e / d];
@@ -94,7 +94,7 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
     if (fresh) {
       const float* __restrict__ v = p.mail + si * (size_t)p.kd_pad;
       double dot = 0.0, dd = 0.0, nv = 0.0;
-#pragma unroll 2
+#pragma unroll 4
       for (int q = tid; q < nvec; q += nt) {
         const int e = q * V;
         const TailVec<V> vv = tail_ldcg<V>(v + e);
@@ -120,7 +120,7 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
 
   // Eq. 6: Dbar = w - (w + sum_s a_s v_s) / (1 + sum_s a_s) + D ;  w <- w - eps * Dbar
   const float inv_m1 = 1.0f / (float)(1 + m);
-#pragma unroll 2
+#pragma unroll 4
   for (int q = tid; q < nvec; q += nt) {
     const int e = q * V;
     TailVec<V> sumv;
@@ -168,7 +168,7 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
       for (int j = 0; j < p.f; ++j) {
         const size_t ri = (size_t)ts->peers[j] * p.S + ts->pslots[j];
         float* dst = p.mail + ri * (size_t)p.kd_pad;
-#pragma unroll 2
+#pragma unroll 8
         for (int q = tid; q < nvec; q += nt) tail_st<V>(dst + q * V, tail_ld<V>(w + widx(q * V)));
         __syncthreads();
         if (tid == 0) red_release_gpu_inc(p.seq + ri);

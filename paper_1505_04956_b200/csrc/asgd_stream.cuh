@@ -286,9 +286,14 @@ asgd_stream_kernel(const Params p, const long long steps) {
         }
         best[q] = bb;
       }
-      const int r = wid * STREAM_WARP_SAMPLES + q * 32 + lane;
-      if (r >= b) best[q] = K;                                   // rows past the batch form their own group
-      else if (p.assign_rec) p.assign_rec[(size_t)i * b + r] = best[q];
+      if (wid * STREAM_WARP_SAMPLES + q * 32 + lane >= b) best[q] = K;   // rows past the batch form their own group
+    }
+    if (p.assign_rec) {
+#pragma unroll
+      for (int q = 0; q < STREAM_SPT; ++q) {
+        const int r = wid * STREAM_WARP_SAMPLES + q * 32 + lane;
+        if (r < b) p.assign_rec[(size_t)i * b + r] = best[q];
+      }
     }
     // ---- lists: per 32-row block, the lanes that chose each centre, in lane order ----
     __syncwarp();

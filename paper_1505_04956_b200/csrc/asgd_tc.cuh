@@ -300,43 +300,66 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     const int sub = lane >> 3, l8 = lane & 7;                                 // eight lanes share a row or a centre
     const int nq = d / 32;
 
-    // ---- decide: a row whose two best scores are closer than the bound is settled between those two
-    //      centres with fp32 inputs and fp64 sums (lane l8 holds dimensions 4*l8 + 32*q) ----
+    // ---- decide: rows whose two best scores are closer than the bound go on a list; the others take the minimum ----
     for (int e = tid; e < TC_WARPS * k; e += TC_THREADS) wcnt[e] = 0;
-    for (int base = wid * 4; base < b; base += TC_WARPS * 4) {
-      const int r = base + sub;
-      const bool valid = r < b;
-      const float2 s = valid ? __ldcg(top2 + r) : make_float2(0.f, INF);
-      const int i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK), i2 = (int)(__float_as_uint(s.y) & TC_INDEX_MASK);
-      const bool flag = valid && k > 1 && (s.y - s.x) <= tau;
-      double d1 = 0.0, d2 = 0.0;
-      if (flag) {
-        const float* x = p.X + (size_t)(row0 + r) * d + 4 * l8;
+    for (int r = tid; r < b; r += TC_THREADS) {
+      const float2 s = __ldcg(top2 + r);
+      const int i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK);
+      best[r] = (unsigned short)i1;
+      if (k > 1 && (s.y - s.x) <= tau) order[atomicAdd(&misc[1], 1)] = (unsigned short)r;
+    }
+    __syncthreads();
+    // ---- listed rows are settled between their two candidates with fp32 inputs and fp64 sums: eight lanes per
+    //      row (lane l8 holds dimensions 4*l8 + 32*q), a warp settles four rows at a time ----
+    {
+      const int nflag = misc[1];
+      auto settle_load = [&](int f, float4 (&xv)[TC_MAX_D / 32], float4 (&a1)[TC_MAX_D / 32], float4 (&a2)[TC_MAX_D / 32], int& r,
+                             int& i1, int& i2) {
+        r = (f < nflag) ? (int)order[f] : -1;
+        const float2 s = (r >= 0) ? __ldcg(top2 + r) : make_float2(0.f, 0.f);
+        i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK);
+        i2 = (int)(__float_as_uint(s.y) & TC_INDEX_MASK);
+        const float* x = p.X + (size_t)(row0 + max(r, 0)) * d + 4 * l8;
         const float* w1 = wglob + (size_t)i1 * d + 4 * l8;
         const float* w2 = wglob + (size_t)i2 * d + 4 * l8;
 #pragma unroll
         for (int q = 0; q < TC_MAX_D / 32; ++q) {
-          if (q < nq) {
-            const float4 xv = __ldg(reinterpret_cast<const float4*>(x + 32 * q));
-            const float4 a1 = *reinterpret_cast<const float4*>(w1 + 32 * q);
-            const float4 a2 = *reinterpret_cast<const float4*>(w2 + 32 * q);
-            double u;
-            u = (double)xv.x - (double)a1.x; d1 = fma(u, u, d1); u = (double)xv.y - (double)a1.y; d1 = fma(u, u, d1);
-            u = (double)xv.z - (double)a1.z; d1 = fma(u, u, d1); u = (double)xv.w - (double)a1.w; d1 = fma(u, u, d1);
-            u = (double)xv.x - (double)a2.x; d2 = fma(u, u, d2); u = (double)xv.y - (double)a2.y; d2 = fma(u, u, d2);
-            u = (double)xv.z - (double)a2.z; d2 = fma(u, u, d2); u = (double)xv.w - (double)a2.w; d2 = fma(u, u, d2);
+          if (q < nq && r >= 0) {
+            xv[q] = __ldg(reinterpret_cast<const float4*>(x + 32 * q));
+            a1[q] = *reinterpret_cast<const float4*>(w1 + 32 * q);
+            a2[q] = *reinterpret_cast<const float4*>(w2 + 32 * q);
+          } else {
+            xv[q] = a1[q] = a2[q] = make_float4(0.f, 0.f, 0.f, 0.f);
           }
         }
-      }
+      };
+      auto settle_finish = [&](const float4 (&xv)[TC_MAX_D / 32], const float4 (&a1)[TC_MAX_D / 32], const float4 (&a2)[TC_MAX_D / 32],
+                               int r, int i1, int i2) {
+        double d1 = 0.0, d2 = 0.0;
 #pragma unroll
-      for (int o = 1; o < 8; o <<= 1) { d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); }
-      if (valid && l8 == 0) {
-        const int bst = (flag && (d2 < d1 || (d2 == d1 && i2 < i1))) ? i2 : i1;
-        best[r] = (unsigned short)bst;
-        if (p.assign_rec) p.assign_rec[(size_t)i * b + r] = bst;
+        for (int q = 0; q < TC_MAX_D / 32; ++q) {
+          double u;
+          u = (double)xv[q].x - (double)a1[q].x; d1 = fma(u, u, d1); u = (double)xv[q].y - (double)a1[q].y; d1 = fma(u, u, d1);
+          u = (double)xv[q].z - (double)a1[q].z; d1 = fma(u, u, d1); u = (double)xv[q].w - (double)a1[q].w; d1 = fma(u, u, d1);
+          u = (double)xv[q].x - (double)a2[q].x; d2 = fma(u, u, d2); u = (double)xv[q].y - (double)a2[q].y; d2 = fma(u, u, d2);
+          u = (double)xv[q].z - (double)a2[q].z; d2 = fma(u, u, d2); u = (double)xv[q].w - (double)a2[q].w; d2 = fma(u, u, d2);
+        }
+#pragma unroll
+        for (int o = 1; o < 8; o <<= 1) { d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); }
+        if (r >= 0 && l8 == 0 && (d2 < d1 || (d2 == d1 && i2 < i1))) best[r] = (unsigned short)i2;
+      };
+      const int groups = TC_WARPS * 4;
+      for (int fb = wid * 4; fb < nflag; fb += groups) {       // the same trip count for all lanes of a warp (shuffles inside)
+        const int f0 = fb + sub;
+        float4 xa[TC_MAX_D / 32], pa[TC_MAX_D / 32], qa[TC_MAX_D / 32];
+        int ra, ia1, ia2;
+        settle_load(f0, xa, pa, qa, ra, ia1, ia2);
+        settle_finish(xa, pa, qa, ra, ia1, ia2);
       }
     }
     __syncthreads();
+    if (p.assign_rec)
+      for (int r = tid; r < b; r += TC_THREADS) p.assign_rec[(size_t)i * b + r] = best[r];
 
     // ---- rows grouped by centre, in row order (stable): ranks inside each warp's block of rows, then offsets ----
     {
@@ -425,15 +448,20 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         float4 S4[TC_MAX_D / 32];
 #pragma unroll
         for (int q = 0; q < TC_MAX_D / 32; ++q) S4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int e = 0; e < n; ++e) {
-          const float* x = p.X + (size_t)(row0 + order[p0 + e]) * d + 4 * l8;
+        for (int e0 = 0; e0 < n; e0 += 2) {                 // two rows in flight; the adds keep ascending row order
+          float4 v[2][TC_MAX_D / 32];
 #pragma unroll
-          for (int q = 0; q < TC_MAX_D / 32; ++q) {
-            if (q < nq) {
-              const float4 v = __ldg(reinterpret_cast<const float4*>(x + 32 * q));
-              S4[q].x += v.x; S4[q].y += v.y; S4[q].z += v.z; S4[q].w += v.w;
-            }
+          for (int u = 0; u < 2; ++u) {
+            const bool have = e0 + u < n;
+            const float* x = p.X + (size_t)(row0 + (have ? (int)order[p0 + e0 + u] : 0)) * d + 4 * l8;
+#pragma unroll
+            for (int q = 0; q < TC_MAX_D / 32; ++q)
+              v[u][q] = (q < nq && have) ? __ldg(reinterpret_cast<const float4*>(x + 32 * q)) : make_float4(0.f, 0.f, 0.f, 0.f);
           }
+#pragma unroll
+          for (int u = 0; u < 2; ++u)
+#pragma unroll
+            for (int q = 0; q < TC_MAX_D / 32; ++q) { S4[q].x += v[u][q].x; S4[q].y += v[u][q].y; S4[q].z += v[u][q].z; S4[q].w += v[u][q].w; }
         }
         float sq = 0.f;
         if (on) {
