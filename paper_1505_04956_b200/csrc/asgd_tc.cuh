@@ -3,19 +3,17 @@
 // contraction  -2 X W^T  of a 4096 x 256 mini-batch against a 1024 x 256 centre matrix.
 //
 // One worker = one thread block = one SM.  Warp roles while the scores are computed:
-//   warp 0   one lane issues the TMA loads: the current 256-centre block of bf16(-2w) (resident for
-//            a whole sweep over the mini-batch) and the 128-row sample tiles in 128-byte-swizzled
-//            K-chunks of 64 through a 4-slot ring;
+//   warp 0   one lane issues the TMA loads: a 128-row sample tile in 128-byte-swizzled K-chunks of 64,
+//            resident while all centre blocks pass, and 256-centre blocks of bf16(-2w) through a
+//            4-slot ring (they come from L2: all workers' bf16 states fit there);
 //   warp 1   allocates tensor memory; one lane issues tcgen05.mma (128 x 256 x 16 per instruction)
-//            into one of two 256-column accumulators and commits to mbarriers;
-//   warps 2-5  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread), add
+//            into one of two 256-column accumulator stages and commits to mbarriers;
+//   warps 4-7  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread), add
 //            ||w_a||^2 and keep, per sample, the two smallest scores with the centre index packed
-//            into the low mantissa bits; the pair lives in a small per-worker scratch in L2 between
-//            the four centre blocks.
+//            into the low mantissa bits, carried in registers over the centre blocks.
 // Then all warps: samples whose two best scores are closer than the BF16 error bound are decided
-// between those two centres with fp32 inputs (fp64 sums); per-centre sums of the fp32 master
-// samples go to the worker's sum buffer with vector reductions; a warp per centre applies the
-// update, refreshes bf16(-2w) and ||w_a||^2.  Every wait is bounded.
+// between those two centres with fp32 inputs (fp64 sums); rows are grouped by centre and each centre's
+// sum of fp32 master samples, update, bf16(-2w) and ||w_a||^2 come from one pass.  Every wait is bounded.
 #pragma once
 
 #include <cuda.h>
@@ -28,9 +26,11 @@ namespace asgd {
 
 constexpr int TC_THREADS = 256;
 constexpr int TC_WARPS = TC_THREADS / 32;
-constexpr int TC_M = 128, TC_N = 256, TC_KC = 64;        // output tile; K chunk = 64 bf16 = one swizzled 128-byte row
-constexpr int TC_A_STAGES = 4;
-constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB
+constexpr int TC_M = 128, TC_N = 256, TC_KC = 64;        // one MMA's output tile; K chunk = 64 bf16 = one swizzled 128-byte row
+constexpr int TC_MH = 1;                                  // 128-row parts of the resident sample tile (TC_MH * TC_N <= 256 accumulator columns per stage)
+constexpr int TC_A_STAGES = 4;                            // K chunks of the resident sample tile (d <= 256)
+constexpr int TC_B_STAGES = 4;                            // ring of centre-block chunks
+constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB per part
 constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;       // 32 KB
 constexpr int TC_MAX_K = 1024, TC_MAX_D = 256, TC_MAX_B = 8192;
 constexpr unsigned TC_INDEX_MASK = 1023u;
@@ -40,8 +40,8 @@ struct TcSmem {
   __host__ __device__ TcSmem(int k, int d, int b) {
     size_t off = 0;
     auto take = [&](size_t bytes, size_t align) { off = (off + align - 1) / align * align; size_t o = off; off += bytes; return o; };
-    B = take((size_t)(d / TC_KC) * TC_B_CHUNK_BYTES, 1024);
-    A = take((size_t)TC_A_STAGES * TC_A_STAGE_BYTES, 1024);
+    A = take((size_t)TC_A_STAGES * TC_MH * TC_A_STAGE_BYTES, 1024);   // [K chunk][part]
+    B = take((size_t)TC_B_STAGES * TC_B_CHUNK_BYTES, 1024);
     cn = take((size_t)((k + TC_N - 1) / TC_N) * TC_N * 4, 16);
     cnt = take((size_t)k * 4, 16);
     best = take((size_t)b * 2, 16);
@@ -96,8 +96,8 @@ __global__ void tc_convert_x_kernel(const float* __restrict__ X, __nv_bfloat16* 
 }
 
 // barrier slots
-enum { TCB_BFULL = 0, TCB_BEMPTY = 1, TCB_AFULL = 2, TCB_AEMPTY = 2 + TC_A_STAGES, TCB_ACCFULL = 2 + 2 * TC_A_STAGES,
-       TCB_ACCEMPTY = 4 + 2 * TC_A_STAGES, TCB_COUNT = 6 + 2 * TC_A_STAGES };
+enum { TCB_BFULL = 0, TCB_BEMPTY = TC_B_STAGES, TCB_AFULL = 2 * TC_B_STAGES, TCB_AEMPTY = 2 * TC_B_STAGES + TC_A_STAGES,
+       TCB_ACCFULL = 2 * TC_B_STAGES + 2 * TC_A_STAGES, TCB_ACCEMPTY = TCB_ACCFULL + 2, TCB_COUNT = TCB_ACCFULL + 4 };
 
 template <bool kDet>
 __global__ void __launch_bounds__(TC_THREADS, 1)
@@ -120,18 +120,17 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int i = blockIdx.x;
   const int nkc = d / TC_KC;                                           // K chunks per tile
-  const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_M - 1) / TC_M;
+  const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_MH * TC_M - 1) / (TC_MH * TC_M);
   const int dl = d / 32;                                               // dimensions per lane (multiple of 2)
   float* wglob = p.state + (size_t)i * p.kd_pad;
   float* gsum = p.gsum + (size_t)i * p.kd_pad;
   __nv_bfloat16* wbf = reinterpret_cast<__nv_bfloat16*>(p.wbf) + (size_t)i * k * d;
-  float2* top2 = reinterpret_cast<float2*>(p.top2) + (size_t)i * b;
+  float2* top2 = reinterpret_cast<float2*>(p.top2) + (size_t)i * b;        // per row: (minimum, runner-up)
   const float INF = __int_as_float(0x7f800000);
   const float inv_b = 1.0f / (float)b;
 
   if (tid == 0) {
-    mbar_init(bars + TCB_BFULL, 1);
-    mbar_init(bars + TCB_BEMPTY, 1);
+    for (int q = 0; q < TC_B_STAGES; ++q) { mbar_init(bars + TCB_BFULL + q, 1); mbar_init(bars + TCB_BEMPTY + q, 1); }
     for (int q = 0; q < TC_A_STAGES; ++q) { mbar_init(bars + TCB_AFULL + q, 1); mbar_init(bars + TCB_AEMPTY + q, 1); }
     for (int q = 0; q < 2; ++q) { mbar_init(bars + TCB_ACCFULL + q, 1); mbar_init(bars + TCB_ACCEMPTY + q, 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -164,30 +163,36 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
 
   unsigned long long t = p.stats[(size_t)i * ST_STRIDE + ST_STEPS];
   // running phase counters of the pipelines (each role keeps its own copies in step)
-  unsigned it_b = 0, it_a = 0, it_acc = 0;
+  unsigned it_m = 0, it_bc = 0, it_acc = 0;
 
   for (long long step = 0; step < steps; ++step, ++t) {
     const long long batch = p.perm[(size_t)i * p.B + (size_t)(t % (unsigned long long)p.B)];
     const long long row0 = (long long)i * p.H + batch * b;
 
     // ================= scores: -2 X W^T + ||w||^2, two best per sample =================
+    // A sample tile (TC_MH parts of 128 rows, nkc K-chunks each) stays in shared memory while the centre blocks stream
+    // past it through a 4-slot ring (the bf16 states of all workers fit in L2; the samples are read from HBM once).
     if (wid == 0) {
       if (lane == 0) {
-        unsigned ib = it_b, ia = it_a;
+        unsigned um = it_m, ibc = it_bc;
         bool ok = true;
-        for (int n = 0; n < n_tiles && ok; ++n, ++ib) {
-          if (ib > 0) ok = mbar_wait_bounded(bars + TCB_BEMPTY, (ib - 1) & 1);           // previous block's MMAs done
-          if (!ok) break;
-          mbar_expect_tx(bars + TCB_BFULL, (unsigned)nkc * TC_B_CHUNK_BYTES);
-          for (int kc = 0; kc < nkc; ++kc)
-            tma_load_2d(sB + (size_t)kc * TC_B_CHUNK_BYTES, &mapW, kc * TC_KC, i * k + n * TC_N, bars + TCB_BFULL);
-          for (int m = 0; m < m_tiles && ok; ++m) {
-            for (int kc = 0; kc < nkc; ++kc, ++ia) {
-              const int st = ia % TC_A_STAGES;
-              if (ia >= TC_A_STAGES) ok = mbar_wait_bounded(bars + TCB_AEMPTY + st, ((ia / TC_A_STAGES) - 1) & 1);
+        for (int m = 0; m < m_tiles && ok; ++m, ++um) {
+          const int halves = min(TC_MH, (b - m * TC_MH * TC_M + TC_M - 1) / TC_M);
+          for (int kc = 0; kc < nkc && ok; ++kc) {
+            if (um > 0) ok = mbar_wait_bounded(bars + TCB_AEMPTY + kc, (um - 1) & 1);     // last use of the chunk by the previous tile
+            if (!ok) break;
+            mbar_expect_tx(bars + TCB_AFULL + kc, (unsigned)(halves * TC_A_STAGE_BYTES));
+            for (int h = 0; h < halves; ++h)
+              tma_load_2d(sA + (size_t)(kc * TC_MH + h) * TC_A_STAGE_BYTES, &mapX, kc * TC_KC,
+                          (int)(row0 + (long long)(m * TC_MH + h) * TC_M), bars + TCB_AFULL + kc);
+          }
+          for (int n = 0; n < n_tiles && ok; ++n) {
+            for (int kc = 0; kc < nkc; ++kc, ++ibc) {
+              const int st = ibc % TC_B_STAGES;
+              if (ibc >= TC_B_STAGES) ok = mbar_wait_bounded(bars + TCB_BEMPTY + st, ((ibc / TC_B_STAGES) - 1) & 1);
               if (!ok) break;
-              mbar_expect_tx(bars + TCB_AFULL + st, TC_A_STAGE_BYTES);
-              tma_load_2d(sA + (size_t)st * TC_A_STAGE_BYTES, &mapX, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + st);
+              mbar_expect_tx(bars + TCB_BFULL + st, TC_B_CHUNK_BYTES);
+              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, kc * TC_KC, i * k + n * TC_N, bars + TCB_BFULL + st);
             }
           }
         }
@@ -195,88 +200,103 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       }
     } else if (wid == 1) {
       if (lane == 0) {
-        unsigned ib = it_b, ia = it_a, iacc = it_acc;
+        unsigned um = it_m, ibc = it_bc, iacc = it_acc;
         bool ok = true;
-        for (int n = 0; n < n_tiles && ok; ++n, ++ib) {
-          ok = mbar_wait_bounded(bars + TCB_BFULL, ib & 1);
-          if (!ok) break;
-          tc_fence_after();
-          for (int m = 0; m < m_tiles && ok; ++m, ++iacc) {
+        for (int m = 0; m < m_tiles && ok; ++m, ++um) {
+          const int halves = min(TC_MH, (b - m * TC_MH * TC_M + TC_M - 1) / TC_M);
+          for (int n = 0; n < n_tiles && ok; ++n, ++iacc) {
             const int buf = iacc & 1;
             if (iacc >= 2) ok = mbar_wait_bounded(bars + TCB_ACCEMPTY + buf, ((iacc >> 1) - 1) & 1);
             if (!ok) break;
             tc_fence_after();
-            for (int kc = 0; kc < nkc && ok; ++kc, ++ia) {
-              const int st = ia % TC_A_STAGES;
-              ok = mbar_wait_bounded(bars + TCB_AFULL + st, (ia / TC_A_STAGES) & 1);
+            for (int kc = 0; kc < nkc && ok; ++kc, ++ibc) {
+              const int st = ibc % TC_B_STAGES;
+              if (n == 0) ok = mbar_wait_bounded(bars + TCB_AFULL + kc, um & 1);
+              if (ok) ok = mbar_wait_bounded(bars + TCB_BFULL + st, (ibc / TC_B_STAGES) & 1);
               if (!ok) break;
               tc_fence_after();
+              for (int h = 0; h < halves; ++h) {
 #pragma unroll
-              for (int k4 = 0; k4 < TC_KC / 16; ++k4)
-                tc_mma_bf16(tmem + (unsigned)buf * TC_N, tc_smem_desc(sA + (size_t)st * TC_A_STAGE_BYTES, k4 * 32),
-                            tc_smem_desc(sB + (size_t)kc * TC_B_CHUNK_BYTES, k4 * 32), idesc, (kc | k4) != 0);
-              tc_commit(bars + TCB_AEMPTY + st);          // the ring slot is free when these MMAs have read it
+                for (int k4 = 0; k4 < TC_KC / 16; ++k4)
+                  tc_mma_bf16(tmem + (unsigned)((buf * TC_MH + h) * TC_N), tc_smem_desc(sA + (size_t)(kc * TC_MH + h) * TC_A_STAGE_BYTES, k4 * 32),
+                              tc_smem_desc(sB + (size_t)st * TC_B_CHUNK_BYTES, k4 * 32), idesc, (kc | k4) != 0);
+              }
+              tc_commit(bars + TCB_BEMPTY + st);                        // the ring slot is free when these MMAs have read it
+              if (n == n_tiles - 1) tc_commit(bars + TCB_AEMPTY + kc);  // and so is the sample chunk after its last centre block
             }
-            tc_commit(bars + TCB_ACCFULL + buf);          // the accumulator is complete
+            tc_commit(bars + TCB_ACCFULL + buf);                        // the accumulator stage is complete
           }
-          tc_commit(bars + TCB_BEMPTY);                   // the centre block may be replaced
         }
         if (!ok) atomicExch(&misc[2], 1);
       }
-    } else if (wid < 6) {
-      const int quarter = wid & 3;                        // a warp reads TMEM lanes 32*(warp%4) .. +31
+    } else if (wid >= 4) {
+      // four warps read the accumulators: warp q of them owns TMEM lanes 32q .. 32q+31, i.e. one row of each part per thread
+      const int quarter = wid & 3;
       unsigned iacc = it_acc;
       bool ok = true;
-      for (int n = 0; n < n_tiles; ++n) {
-        for (int m = 0; m < m_tiles; ++m, ++iacc) {
+      for (int m = 0; m < m_tiles; ++m) {
+        const int r0 = m * TC_MH * TC_M + quarter * 32 + lane;     // the thread's row of part 0; part h is h * TC_M further
+        float m1[TC_MH][2], m2[TC_MH][2];                           // per row two independent (minimum, runner-up) pairs, kept over the centre blocks
+#pragma unroll
+        for (int h = 0; h < TC_MH; ++h) { m1[h][0] = m1[h][1] = INF; m2[h][0] = m2[h][1] = INF; }
+        for (int n = 0; n < n_tiles; ++n, ++iacc) {
           const int buf = iacc & 1;
           if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bars + TCB_ACCFULL + buf, (iacc >> 1) & 1));
           if (!ok) continue;
           tc_fence_after();
-          const int r = m * TC_M + quarter * 32 + lane;
-          float e1 = INF, e2 = INF, o1 = INF, o2 = INF;   // two independent (minimum, runner-up) pairs
+#pragma unroll 1
           for (int c0 = 0; c0 < TC_N; c0 += 32) {
-            unsigned v[32];
-            const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)(buf * TC_N + c0);
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
-                  "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]),
-                  "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]),
-                  "=r"(v[30]), "=r"(v[31])
-                : "r"(taddr) : "memory");
+            unsigned v[TC_MH][32];
+#pragma unroll
+            for (int h = 0; h < TC_MH; ++h) {
+              const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)((buf * TC_MH + h) * TC_N + c0);
+              asm volatile(
+                  "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                  : "=r"(v[h][0]), "=r"(v[h][1]), "=r"(v[h][2]), "=r"(v[h][3]), "=r"(v[h][4]), "=r"(v[h][5]), "=r"(v[h][6]), "=r"(v[h][7]),
+                    "=r"(v[h][8]), "=r"(v[h][9]), "=r"(v[h][10]), "=r"(v[h][11]), "=r"(v[h][12]), "=r"(v[h][13]), "=r"(v[h][14]), "=r"(v[h][15]),
+                    "=r"(v[h][16]), "=r"(v[h][17]), "=r"(v[h][18]), "=r"(v[h][19]), "=r"(v[h][20]), "=r"(v[h][21]), "=r"(v[h][22]), "=r"(v[h][23]),
+                    "=r"(v[h][24]), "=r"(v[h][25]), "=r"(v[h][26]), "=r"(v[h][27]), "=r"(v[h][28]), "=r"(v[h][29]), "=r"(v[h][30]), "=r"(v[h][31])
+                  : "r"(taddr) : "memory");
+            }
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (c0 + 32 == TC_N) {                        // last read of this accumulator: hand it back
+            if (c0 + 32 == TC_N) {                        // last read of this accumulator stage: hand it back
               tc_fence_before();
               if (lane == 0) mbar_arrive(bars + TCB_ACCEMPTY + buf);
             }
             const int abase = n * TC_N + c0;
+            const unsigned hi_or_base = ~TC_INDEX_MASK | (unsigned)abase;   // abase is a multiple of 32: its bits and a column's do not meet
 #pragma unroll
-            for (int c = 0; c < 32; c += 2) {
-              const float s0 = __uint_as_float(v[c]) + cn[abase + c];
-              const float s1 = __uint_as_float(v[c + 1]) + cn[abase + c + 1];
-              const float p0 = __uint_as_float((__float_as_uint(s0) & ~TC_INDEX_MASK) | (unsigned)(abase + c));
-              const float p1 = __uint_as_float((__float_as_uint(s1) & ~TC_INDEX_MASK) | (unsigned)(abase + c + 1));
-              e2 = fmaxf(e1, fminf(e2, p0)); e1 = fminf(e1, p0);
-              o2 = fmaxf(o1, fminf(o2, p1)); o1 = fminf(o1, p1);
+            for (int c = 0; c < 32; c += 4) {
+              const float4 cn4 = *reinterpret_cast<const float4*>(cn + abase + c);
+              const float cv[4] = {cn4.x, cn4.y, cn4.z, cn4.w};
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+#pragma unroll
+                for (int h = 0; h < TC_MH; ++h) {
+                  const float sc = __uint_as_float(v[h][c + u]) + cv[u];
+                  // one logic op: the score's high bits, the block's and the column's index bits below them
+                  // (where both masks are set take the score, elsewhere the OR of the two index words)
+                  unsigned spb;
+                  asm("lop3.b32 %0, %1, %2, %3, 0xE6;" : "=r"(spb) : "r"(__float_as_uint(sc)), "r"(hi_or_base), "r"(~TC_INDEX_MASK | (unsigned)(c + u)));
+                  const float sp = __uint_as_float(spb);
+                  m2[h][u & 1] = fmaxf(m1[h][u & 1], fminf(m2[h][u & 1], sp));
+                  m1[h][u & 1] = fminf(m1[h][u & 1], sp);
+                }
+              }
             }
           }
-          float s2 = fminf(fmaxf(e1, o1), fminf(e2, o2));
-          float s1 = fminf(e1, o1);
-          if (r < b) {
-            if (n > 0) {
-              const float2 prev = __ldcg(top2 + r);
-              s2 = fminf(fmaxf(s1, prev.x), fminf(s2, prev.y));
-              s1 = fminf(s1, prev.x);
-            }
-            __stcg(top2 + r, make_float2(s1, s2));
-          }
+        }
+#pragma unroll
+        for (int h = 0; h < TC_MH; ++h) {
+          const int r = r0 + h * TC_M;
+          if (ok && r < b)
+            __stcg(top2 + r, make_float2(fminf(m1[h][0], m1[h][1]), fminf(fmaxf(m1[h][0], m1[h][1]), fminf(m2[h][0], m2[h][1]))));
         }
       }
       if (!ok && lane == 0) atomicExch(&misc[2], 1);
     }
-    it_b += (unsigned)n_tiles;
-    it_a += (unsigned)(n_tiles * m_tiles * nkc);
+    it_m += (unsigned)m_tiles;
+    it_bc += (unsigned)(m_tiles * n_tiles * nkc);
     it_acc += (unsigned)(n_tiles * m_tiles);
     if (tid == 0) misc[1] = 0;
     for (int a = tid; a < k; a += TC_THREADS) cnt[a] = 0;
