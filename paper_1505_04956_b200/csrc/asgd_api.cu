@@ -190,6 +190,22 @@ bool encode_bf16_map(CUtensorMap* map, const void* base, unsigned long long rows
 }
 
 // Tensor-core path set-up: bf16 copy of X (unless the caller brought one), max ||x||^2, tensor maps.
+// max_i ||x_i||^2 into Params::xmax2 (one pass over the samples at initialisation): the rounding bounds of the
+// streaming and tensor-core paths use it.
+int compute_xmax2(asgd_ctx* c) {
+  Params& p = c->p;
+  unsigned* xm = (unsigned*)(c->ws + c->L.xmax);
+  CU(c, cudaMemsetAsync(xm, 0, 4, c->stream));
+  xmax2_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, p.N, p.d, xm);
+  c->launches += 1;
+  CU(c, cudaGetLastError());
+  float xmax2 = 0.f;
+  CU(c, cudaMemcpyAsync(&xmax2, xm, 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  p.xmax2 = xmax2;
+  return ASGD_OK;
+}
+
 int tc_prepare(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
   Params& p = c->p;
@@ -206,15 +222,7 @@ int tc_prepare(asgd_ctx* c) {
     CU(c, cudaGetLastError());
     xbf = dst;
   }
-  unsigned* xm = (unsigned*)(c->ws + c->L.xmax);
-  CU(c, cudaMemsetAsync(xm, 0, 4, c->stream));
-  xmax2_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, p.N, p.d, xm);
-  c->launches += 1;
-  CU(c, cudaGetLastError());
-  float xmax2 = 0.f;
-  CU(c, cudaMemcpyAsync(&xmax2, xm, 4, cudaMemcpyDeviceToHost, c->stream));
-  CU(c, cudaStreamSynchronize(c->stream));
-  p.xmax2 = xmax2;
+  { const int rc = compute_xmax2(c); if (rc != ASGD_OK) return rc; }
   if (!encode_bf16_map(&c->mapX, xbf, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
   if (!encode_bf16_map(&c->mapW, p.wbf, (unsigned long long)cfg.W * cfg.k, (unsigned long long)cfg.d, TC_N)) return ASGD_ECUDA;
   return ASGD_OK;
@@ -372,6 +380,9 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   c->launches += 1;
   if (c->path == P_TC_BF16) {
     rc = tc_prepare(c);
+    if (rc != ASGD_OK) { delete c; return rc; }
+  } else if (c->path == P_STREAM) {
+    rc = compute_xmax2(c);
     if (rc != ASGD_OK) { delete c; return rc; }
   }
 

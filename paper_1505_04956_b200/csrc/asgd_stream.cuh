@@ -11,10 +11,12 @@
 // whose two best scores are closer than the rounding bound of this form is decided again in the
 // direct difference form.
 //
-// Per-centre sums (Eq. 9): for each of its four 32-row blocks a warp lists the lanes that chose each
-// centre (rank inside the block from a match, so a list is in row order); then lane (block, centre)
-// adds the listed rows from the shared-memory tile.  Every sum has a fixed order, so a step is
-// reproducible.  The plain local step needs two block-wide barriers.
+// Per-centre sums (Eq. 9): each warp files its 128 rows under the centres they chose (rank inside a
+// 32-row block from a match, so a warp's list of a centre is in row order; entries are byte offsets
+// into the tile, the unused tail of a list points at a row of zeros kept behind the tile).  Then one
+// thread per (half of the warps, centre, dimension pair) adds the listed rows from the shared-memory
+// tile.  Every sum has a fixed order, so a step is reproducible.  The plain local step needs three
+// block-wide barriers.
 #pragma once
 
 #include "asgd_step_tail.cuh"
@@ -27,7 +29,8 @@ constexpr int STREAM_STAGES = 2;
 constexpr int STREAM_SPT = 4;                          // samples per thread = 32-row blocks per warp
 constexpr int STREAM_MAX_B = STREAM_THREADS * STREAM_SPT;
 constexpr int STREAM_WARP_SAMPLES = 32 * STREAM_SPT;
-constexpr int STREAM_PARTS = STREAM_WARPS * STREAM_SPT;   // partial sums per centre
+constexpr int STREAM_PARTS = 2;                        // partial sums per centre: one per half of the warps
+constexpr int STREAM_SEG = STREAM_WARP_SAMPLES;        // capacity of a warp's list of one centre
 constexpr unsigned STREAM_WAIT_LIMIT = 1u << 22;       // bounded mbarrier wait (iterations of try_wait)
 
 __device__ inline unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -69,31 +72,36 @@ struct StreamLayout {
   static constexpr int INDEX_BITS = (K <= 2) ? 1 : (K <= 4) ? 2 : (K <= 8) ? 3 : 4;
   static constexpr unsigned INDEX_MASK = (1u << INDEX_BITS) - 1u;
   static constexpr int CPW = 32 / D;                // centres a warp updates at a time
-  static constexpr int LISTS = STREAM_SPT * K;      // lists per warp: (32-row block, centre)
+  static constexpr int ROWB = D * 4;                // bytes per sample
+  static constexpr int ZR_EXTRA = (16 + ROWB - 1) / ROWB;   // rows between the batch's last row and the row of zeros (a copy may overrun by < 16 bytes)
+  static constexpr int CWS = (K + 1 + 3) / 4 * 4;   // a warp's list lengths, one spare counter for rows past the batch
 };
 
 // Shared-memory map of the streaming kernel (byte offsets, every region 16-byte aligned).
 template <int D, int K>
 struct StreamSmem {
   using L = StreamLayout<D, K>;
-  size_t ring, bars, flags, zero, tail, wneg2, cnorm, w, sd, sw, cw, cnt, seen, lists, total;
+  size_t ring, bars, flags, tail, wneg2, cnorm, w, sd, sw, cw, cnt, seen, lists, total;
+  // a ring slot: the batch (source rounded out to 16-byte bounds), then a row of zeros wherever the batch starts in the slot
+  __host__ __device__ static size_t slot_bytes(int b) {
+    return ((size_t)(b + L::ZR_EXTRA) * L::ROWB + 16 + L::ROWB + 127) / 128 * 128;
+  }
   __host__ __device__ explicit StreamSmem(int b) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) / 16 * 16; return o; };
-    ring = take(STREAM_STAGES * (((size_t)b * D * 4 + 32 + 127) / 128 * 128));
+    ring = take(STREAM_STAGES * slot_bytes(b));
     bars = take(64);
     flags = take(64);
-    zero = take(64);                                            // a row of zeros
     tail = take(sizeof(TailScratch));
     wneg2 = take((size_t)K * L::DP * 4);
     cnorm = take((size_t)K * 8);                                // (||w_a||^2, 0) pairs
     w = take((size_t)K * D * 4);
     sd = take((size_t)K * D * 4);
     sw = take((size_t)STREAM_PARTS * K * D * 4);                // partial sums
-    cw = take((size_t)STREAM_WARPS * L::LISTS * 4);             // list lengths
+    cw = take((size_t)STREAM_WARPS * L::CWS * 4);               // list lengths
     cnt = take((size_t)K * 4);
     seen = take((size_t)MAX_SLOTS * 4);
-    lists = take((size_t)STREAM_WARPS * L::LISTS * 32);         // u8 lane numbers
+    lists = take((size_t)STREAM_WARPS * K * STREAM_SEG * 2);    // u16 byte offsets of rows in the tile
     total = (off + 127) / 128 * 128;
   }
 };
@@ -104,15 +112,15 @@ template <int D, int K, bool kDet>
 __global__ void __launch_bounds__(STREAM_THREADS, 4)
 asgd_stream_kernel(const Params p, const long long steps) {
   using L = StreamLayout<D, K>;
-  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, LISTS = L::LISTS;
+  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, ROWB = L::ROWB, CWS = L::CWS;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int b = p.b;
-  const unsigned slot_bytes = ((unsigned)b * D * 4 + 32 + 127) / 128 * 128;
+  const unsigned slot_bytes = (unsigned)StreamSmem<D, K>::slot_bytes(b);
+  const unsigned zr_off = (unsigned)(b + L::ZR_EXTRA) * ROWB;              // from a batch's first row to the row of zeros
   const StreamSmem<D, K> map(b);
   unsigned char* ring = smem_raw + map.ring;
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + map.bars);   // [STAGES]
   int* flags = reinterpret_cast<int*>(smem_raw + map.flags);                               // [0] a buffer has news
-  const float* zero_row = reinterpret_cast<const float*>(smem_raw + map.zero);
   TailScratch* ts = reinterpret_cast<TailScratch*>(smem_raw + map.tail);
   float* wneg2 = reinterpret_cast<float*>(smem_raw + map.wneg2);
   float2* cnorm = reinterpret_cast<float2*>(smem_raw + map.cnorm);
@@ -122,7 +130,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
   int* Cw = reinterpret_cast<int*>(smem_raw + map.cw);
   int* cnt = reinterpret_cast<int*>(smem_raw + map.cnt);
   unsigned* seen_s = reinterpret_cast<unsigned*>(smem_raw + map.seen);
-  unsigned char* lists = smem_raw + map.lists;
+  unsigned short* lists = reinterpret_cast<unsigned short*>(smem_raw + map.lists);
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int i = blockIdx.x;
@@ -135,7 +143,8 @@ asgd_stream_kernel(const Params p, const long long steps) {
 
   // state on chip: w, -2w (padded rows), (||w_a||^2, 0)
   for (int e = tid; e < K * DP; e += STREAM_THREADS) wneg2[e] = 0.f;
-  if (tid < 16) reinterpret_cast<float*>(smem_raw + map.zero)[tid] = 0.f;
+  for (int e = tid; e < STREAM_STAGES * (4 + D); e += STREAM_THREADS)       // the zeros behind each slot's batch, never overwritten
+    reinterpret_cast<float*>(ring + (size_t)(e / (4 + D)) * slot_bytes + zr_off)[e % (4 + D)] = 0.f;
   __syncthreads();
   for (int e = tid; e < KD; e += STREAM_THREADS) {
     const float v = wglob[e];
@@ -192,8 +201,9 @@ asgd_stream_kernel(const Params p, const long long steps) {
   __syncthreads();
 
   const float tau_scale = (float)(4 * D + 72) * 5.9604645e-8f;
-  int* myCw = Cw + wid * LISTS;
-  unsigned char* myLists = lists + (size_t)wid * (LISTS * 32);
+  const float xmax2 = p.xmax2;                                              // max ||x||^2 over the samples
+  int* myCw = Cw + wid * CWS;
+  unsigned short* myLists = lists + (size_t)wid * (K * STREAM_SEG);
   int abort = 0;
   for (long long step = 0; step < steps; ++step, ++t) {
     const int slot = (int)(step & 1);
@@ -208,7 +218,13 @@ asgd_stream_kernel(const Params p, const long long steps) {
     if (tid < p.S) my_seq = ld_relaxed_gpu(p.seq + (size_t)i * p.S + tid);
     const int pos2 = next_pos(pos1);
     const int batch_nn = myperm[pos2];
-    for (int e = lane; e < LISTS; e += 32) myCw[e] = 0;
+    {
+      // this warp's lists: every entry points at the row of zeros, lengths zero
+      const unsigned zz = zr_off | (zr_off << 16);
+      uint4* dst = reinterpret_cast<uint4*>(myLists);
+      for (int e = lane; e < K * STREAM_SEG / 8; e += 32) dst[e] = make_uint4(zz, zz, zz, zz);
+      for (int e = lane; e <= K; e += 32) myCw[e] = 0;
+    }
 
     unsigned head, bytes;
     const unsigned char* src = tile_src(batch_cur, head, bytes);
@@ -226,17 +242,12 @@ asgd_stream_kernel(const Params p, const long long steps) {
 
     // ---- Eq. 8: scores of this thread's samples against every centre ----
     float2 xv[STREAM_SPT][D2];
-    float x2[STREAM_SPT];
 #pragma unroll
     for (int q = 0; q < STREAM_SPT; ++q) {
       const int r = min(wid * STREAM_WARP_SAMPLES + q * 32 + lane, b - 1);   // rows past the batch re-read its last row
       const float2* xrow = reinterpret_cast<const float2*>(xs + (size_t)r * D);
 #pragma unroll
       for (int jp = 0; jp < D2; ++jp) xv[q][jp] = xrow[jp];
-      float2 n2 = __fmul2_rn(xv[q][0], xv[q][0]);
-#pragma unroll
-      for (int jp = 1; jp < D2; ++jp) n2 = __ffma2_rn(xv[q][jp], xv[q][jp], n2);
-      x2[q] = n2.x + n2.y;
     }
     float s1[STREAM_SPT], s2[STREAM_SPT];
 #pragma unroll
@@ -270,21 +281,26 @@ asgd_stream_kernel(const Params p, const long long steps) {
 #pragma unroll
     for (int q = 0; q < STREAM_SPT; ++q) {
       best[q] = (int)(__float_as_uint(s1[q]) & L::INDEX_MASK);
-      if (K > 1 && (s2[q] - s1[q]) <= tau_scale * (wmax2 + x2[q])) {
-        float bd = __int_as_float(0x7f800000);
-        int bb = 0;
-        for (int a = 0; a < K; ++a) {
-          float acc = 0.f;
+      if (K > 1 && (s2[q] - s1[q]) <= tau_scale * (wmax2 + xmax2)) {       // cheap test with the global bound on ||x||^2 first
+        float2 n2 = __fmul2_rn(xv[q][0], xv[q][0]);
 #pragma unroll
-          for (int jp = 0; jp < D2; ++jp) {
-            const float d0 = xv[q][jp].x + 0.5f * wneg2[a * DP + 2 * jp];        // -0.5 * (-2w) = w, exact
-            const float d1 = xv[q][jp].y + 0.5f * wneg2[a * DP + 2 * jp + 1];
-            acc = fmaf(d0, d0, acc);
-            acc = fmaf(d1, d1, acc);
+        for (int jp = 1; jp < D2; ++jp) n2 = __ffma2_rn(xv[q][jp], xv[q][jp], n2);
+        if ((s2[q] - s1[q]) <= tau_scale * (wmax2 + (n2.x + n2.y))) {
+          float bd = __int_as_float(0x7f800000);
+          int bb = 0;
+          for (int a = 0; a < K; ++a) {
+            float acc = 0.f;
+#pragma unroll
+            for (int jp = 0; jp < D2; ++jp) {
+              const float d0 = xv[q][jp].x + 0.5f * wneg2[a * DP + 2 * jp];        // -0.5 * (-2w) = w, exact
+              const float d1 = xv[q][jp].y + 0.5f * wneg2[a * DP + 2 * jp + 1];
+              acc = fmaf(d0, d0, acc);
+              acc = fmaf(d1, d1, acc);
+            }
+            if (acc < bd) { bd = acc; bb = a; }          // strict "<": the lowest index keeps a tie
           }
-          if (acc < bd) { bd = acc; bb = a; }          // strict "<": the lowest index keeps a tie
+          best[q] = bb;
         }
-        best[q] = bb;
       }
       if (wid * STREAM_WARP_SAMPLES + q * 32 + lane >= b) best[q] = K;   // rows past the batch form their own group
     }
@@ -295,49 +311,50 @@ asgd_stream_kernel(const Params p, const long long steps) {
         if (r < b) p.assign_rec[(size_t)i * b + r] = best[q];
       }
     }
-    // ---- lists: per 32-row block, the lanes that chose each centre, in lane order ----
+    // ---- lists: this warp's rows under the centres they chose, in row order ----
     __syncwarp();
 #pragma unroll
     for (int q = 0; q < STREAM_SPT; ++q) {
       const unsigned grp = __match_any_sync(0xffffffffu, best[q]);
       const unsigned below = grp & ((1u << lane) - 1u);
-      if (best[q] < K) {
-        myLists[(q * K + best[q]) * 32 + __popc(below)] = (unsigned char)lane;
-        if (below == 0) myCw[q * K + best[q]] = __popc(grp);
-      }
+      const int base = myCw[best[q]];                                      // rows past the batch count into the spare counter
+      __syncwarp();
+      if (best[q] < K) myLists[best[q] * STREAM_SEG + base + __popc(below)] = (unsigned short)((wid * STREAM_WARP_SAMPLES + q * 32 + lane) * ROWB);
+      if (below == 0) myCw[best[q]] = base + __popc(grp);
+      __syncwarp();
     }
     if (tid < p.S && my_seq != seen_s[tid]) flags[0] = 1;
-    __syncwarp();
 
-    // ---- Eq. 9: lane (block, centre) adds its list's rows; up to 8 independent row loads at a time ----
-    for (int l = lane; l < LISTS; l += 32) {
-      const int q = l / K, a = l % K;
-      const int n = myCw[l];
-      const float* blk = wblk + (size_t)q * 32 * D;
-      const uint2* ent = reinterpret_cast<const uint2*>(myLists + l * 32);
-      float2 acc[D2];
+    // ---- barrier B1: every warp's lists are complete ----
+    if (__syncthreads_or(abort)) { abort = 1; break; }
+
+    // ---- Eq. 9: thread (half, centre, dimension pair) adds the rows listed by its half of the warps ----
+    {
+      constexpr int ITEMS = STREAM_PARTS * K * D2, WPP = STREAM_WARPS / STREAM_PARTS;
+      for (int item = tid; item < ITEMS; item += STREAM_THREADS) {
+        const int h = item / (K * D2), rem = item - h * (K * D2), a = rem / D2, jp = rem - a * D2;
+        const unsigned char* xb = reinterpret_cast<const unsigned char*>(xs) + jp * 8;
+        auto row = [&](unsigned off) { return *reinterpret_cast<const float2*>(xb + off); };
+        float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
 #pragma unroll
-      for (int jp = 0; jp < D2; ++jp) acc[jp] = make_float2(0.f, 0.f);
-      const int nmax = (int)__reduce_max_sync(__activemask(), (unsigned)n);
-      for (int e0 = 0; e0 < nmax; e0 += 8) {
-        const uint2 pk = ent[e0 >> 3];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const unsigned word = (u < 4) ? pk.x : pk.y;
-          const int li = (int)((word >> (8 * (u & 3))) & 0xffu);
-          const float2* row = reinterpret_cast<const float2*>((e0 + u < n) ? blk + li * D : zero_row);
-#pragma unroll
-          for (int jp = 0; jp < D2; ++jp) acc[jp] = __fadd2_rn(acc[jp], row[jp]);
+        for (int ww = 0; ww < WPP; ++ww) {
+          const int wsrc = h * WPP + ww;
+          const int n = Cw[wsrc * CWS + a];
+          const uint4* seg = reinterpret_cast<const uint4*>(lists + (size_t)(wsrc * K + a) * STREAM_SEG);
+          for (int e0 = 0; e0 < n; e0 += 8) {                              // a list's tail points at the row of zeros
+            const uint4 pk = seg[e0 >> 3];
+            acc0 = __fadd2_rn(acc0, row(pk.x & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.x >> 16));
+            acc0 = __fadd2_rn(acc0, row(pk.y & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.y >> 16));
+            acc0 = __fadd2_rn(acc0, row(pk.z & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.z >> 16));
+            acc0 = __fadd2_rn(acc0, row(pk.w & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.w >> 16));
+          }
         }
+        *reinterpret_cast<float2*>(Sw + (size_t)(h * K + a) * D + 2 * jp) = __fadd2_rn(acc0, acc1);
       }
-      float2* out = reinterpret_cast<float2*>(Sw + (size_t)((wid * STREAM_SPT + q) * K + a) * D);
-#pragma unroll
-      for (int jp = 0; jp < D2; ++jp) out[jp] = acc[jp];
-      if (n) atomicAdd(cnt + a, n);
     }
 
-    // ---- barrier B: partial sums and counts complete, the ring slot is free again ----
-    if (__syncthreads_or(abort)) { abort = 1; break; }
+    // ---- barrier B2: partial sums complete, the ring slot is free again ----
+    __syncthreads();
 
     const bool put_now = (to_put == 1);
     if (flags[0] != 0 || put_now) {
@@ -345,8 +362,14 @@ asgd_stream_kernel(const Params p, const long long steps) {
       for (int e = tid; e < KD; e += STREAM_THREADS) {
         float ssum = 0.f;
 #pragma unroll
-        for (int q = 0; q < STREAM_PARTS; ++q) ssum += Sw[(size_t)(q * K + e / D) * D + (e % D)];
+        for (int q = 0; q < STREAM_PARTS; ++q) ssum += Sw[(size_t)q * KD + e];
         SD[e] = ssum;
+      }
+      if (tid < K) {
+        int n = 0;
+#pragma unroll
+        for (int q = 0; q < STREAM_WARPS; ++q) n += Cw[q * CWS + tid];
+        cnt[tid] = n;
       }
       __syncthreads();
       step_tail<kDet>(p, i, t, w, D, SD, cnt, wglob, ts);
@@ -368,7 +391,9 @@ asgd_stream_kernel(const Params p, const long long steps) {
         const bool on = (lane < L::CPW * D) && (a < K);
         float sq = 0.f;
         if (on) {
-          const int n = cnt[a];
+          int n = 0;
+#pragma unroll
+          for (int q = 0; q < STREAM_WARPS; ++q) n += Cw[q * CWS + a];
           float ssum = 0.f;
 #pragma unroll
           for (int q = 0; q < STREAM_PARTS; ++q) ssum += Sw[(size_t)(q * K + a) * D + j];
@@ -386,7 +411,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
           if (j + o < D) sq += up;
         }
         __syncwarp();
-        if (on && j == 0) { cnorm[a] = make_float2(sq, 0.f); cnt[a] = 0; }
+        if (on && j == 0) cnorm[a] = make_float2(sq, 0.f);
       }
       if (tid == 0) {
         if (kDet)
