@@ -40,6 +40,45 @@ template <int V> __device__ inline void tail_st(float* q, const TailVec<V>& r) {
   else *q = r.v[0];
 }
 
+// The send line of Algorithm 5: after step t, when (t + 1) is a multiple of the interval, w_{t+1} goes to f random
+// workers != i.  Called by all threads of the block with w complete and visible (a barrier before); returns the
+// number of messages sent.  Free-running: every thread stores part of the payload, a barrier, then one release
+// increment of the buffer's sequence number.  Synchronous rounds: the put is only announced; the delivery kernel
+// copies the payload of the highest announcing (sender, j) once every worker has finished the round.
+template <bool kDet, int V>
+__device__ inline unsigned long long step_send(const Params& p, int i, unsigned long long t, const float* __restrict__ w,
+                                               int wstride, TailScratch* ts) {
+  if (!(p.c > 0 && p.f > 0 && p.W > 1 && (t + 1) % (unsigned long long)p.c == 0)) return 0;
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int d = p.d, nvec = p.kd / V;
+  const bool dense_rows = (wstride == d);
+  auto widx = [&](int e) { return dense_rows ? e : (e / d) * wstride + (e % d); };
+  if (tid == 0) {
+    for (int j = 0; j < p.f; ++j) {
+      ts->peers[j] = sched_peer(p, i, t, j, ts->peers);
+      ts->pslots[j] = sched_slot(p, i, t, j);
+    }
+  }
+  __syncthreads();
+  if (kDet) {
+    if (tid < p.f) {
+      const size_t ri = (size_t)ts->peers[tid] * p.S + ts->pslots[tid];
+      atomicMax(p.arb_win + ri, (unsigned)(i * p.f + tid + 1));
+      atomicAdd(p.arb_cnt + ri, 1u);
+    }
+  } else {
+    for (int j = 0; j < p.f; ++j) {
+      const size_t ri = (size_t)ts->peers[j] * p.S + ts->pslots[j];
+      float* dst = p.mail + ri * (size_t)p.kd_pad;
+#pragma unroll 8
+      for (int q = tid; q < nvec; q += nt) tail_st<V>(dst + q * V, tail_ld<V>(w + widx(q * V)));
+      __syncthreads();
+      if (tid == 0) red_release_gpu_inc(p.seq + ri);
+    }
+  }
+  return (unsigned long long)p.f;
+}
+
 // w     [k rows of d, row stride wstride]  this worker's state (shared or global memory), updated in place
 // SD    [kd]  in: per-centre sums S_k of the mini-batch; out: the local gradient D
 // cnt   [k]   per-centre counts n_k
@@ -147,35 +186,7 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
   __syncthreads();
 
   // send w_{t+1} to f random workers != i
-  unsigned long long n_sent = 0;
-  if (p.c > 0 && p.f > 0 && p.W > 1 && (t + 1) % (unsigned long long)p.c == 0) {
-    if (tid == 0) {
-      for (int j = 0; j < p.f; ++j) {
-        ts->peers[j] = sched_peer(p, i, t, j, ts->peers);
-        ts->pslots[j] = sched_slot(p, i, t, j);
-      }
-    }
-    __syncthreads();
-    if (kDet) {
-      // synchronous rounds: only announce the put; the delivery kernel copies the payload of the
-      // highest announcing (sender, j) once every worker has finished the round
-      if (tid < p.f) {
-        const size_t ri = (size_t)ts->peers[tid] * p.S + ts->pslots[tid];
-        atomicMax(p.arb_win + ri, (unsigned)(i * p.f + tid + 1));
-        atomicAdd(p.arb_cnt + ri, 1u);
-      }
-    } else {
-      for (int j = 0; j < p.f; ++j) {
-        const size_t ri = (size_t)ts->peers[j] * p.S + ts->pslots[j];
-        float* dst = p.mail + ri * (size_t)p.kd_pad;
-#pragma unroll 8
-        for (int q = tid; q < nvec; q += nt) tail_st<V>(dst + q * V, tail_ld<V>(w + widx(q * V)));
-        __syncthreads();
-        if (tid == 0) red_release_gpu_inc(p.seq + ri);
-      }
-    }
-    n_sent = (unsigned long long)p.f;
-  }
+  const unsigned long long n_sent = step_send<kDet, V>(p, i, t, w, wstride, ts);
 
   if (tid == 0) {
     unsigned long long* st = p.stats + (size_t)i * ST_STRIDE;
@@ -192,6 +203,14 @@ __device__ inline void step_tail(const Params& p, int i, unsigned long long t, f
   const bool vec = (p.d % 4 == 0) && (wstride % 4 == 0) && ((((size_t)w) | ((size_t)SD) | ((size_t)wglob)) & 15) == 0;
   if (vec) step_tail_impl<kDet, 4>(p, i, t, w, wstride, SD, cnt, wglob, ts, sd_l2);
   else step_tail_impl<kDet, 1>(p, i, t, w, wstride, SD, cnt, wglob, ts, sd_l2);
+}
+
+// The send alone, for paths that fuse the plain local update into their own passes.
+template <bool kDet>
+__device__ inline unsigned long long step_send_any(const Params& p, int i, unsigned long long t, const float* w, int wstride,
+                                                   TailScratch* ts) {
+  const bool vec = (p.d % 4 == 0) && (wstride % 4 == 0) && (((size_t)w) & 15) == 0;
+  return vec ? step_send<kDet, 4>(p, i, t, w, wstride, ts) : step_send<kDet, 1>(p, i, t, w, wstride, ts);
 }
 
 }  // namespace asgd

@@ -357,8 +357,8 @@ asgd_stream_kernel(const Params p, const long long steps) {
     __syncthreads();
 
     const bool put_now = (to_put == 1);
-    if (flags[0] != 0 || put_now) {
-      // a message is waiting or a put is due: totals into SD, then the general tail handles both
+    if (flags[0] != 0) {
+      // a message is waiting: totals into SD, then the general tail (which also sends when a put is due)
       for (int e = tid; e < KD; e += STREAM_THREADS) {
         float ssum = 0.f;
 #pragma unroll
@@ -413,10 +413,17 @@ asgd_stream_kernel(const Params p, const long long steps) {
         __syncwarp();
         if (on && j == 0) cnorm[a] = make_float2(sq, 0.f);
       }
+      unsigned long long n_sent = 0;
+      if (put_now) {
+        __syncthreads();                                 // the new w is complete
+        n_sent = step_send_any<kDet>(p, i, t, w, D, ts);
+      }
       if (tid == 0) {
         if (kDet)
           for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
-        p.stats[(size_t)i * ST_STRIDE + ST_STEPS] = t + 1;
+        unsigned long long* st = p.stats + (size_t)i * ST_STRIDE;
+        st[ST_STEPS] = t + 1;
+        if (n_sent) atomicAdd(st + ST_SENT, n_sent);
       }
     }
     batch_cur = batch_nxt;

@@ -442,7 +442,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     }
     __syncthreads();
     const bool put_now = p.c > 0 && p.f > 0 && p.W > 1 && (t + 1) % (unsigned long long)p.c == 0;
-    const bool plain = !(misc[4] != 0 || put_now);
+    const bool plain = (misc[4] == 0);                    // no message waiting: the fused update below, then the send if one is due
 
     // ---- Eq. 9 and the update: eight lanes per centre add its rows (fp32 master, ascending row order);
     //      plain step: w <- w - eps (n w - S) / b at once; otherwise S goes to the sum buffer for the general tail ----
@@ -531,10 +531,19 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         for (int o = 1; o < 8; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
         if (a < k && l8 == 0) cn[a] = sq;
       }
-    } else if (tid == 0) {
-      if (kDet)
-        for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
-      p.stats[(size_t)i * ST_STRIDE + ST_STEPS] = t + 1;
+    } else {
+      unsigned long long n_sent = 0;
+      if (put_now) {
+        __syncthreads();                                  // every centre's new w is in place
+        n_sent = step_send_any<kDet>(p, i, t, wglob, d, ts);
+      }
+      if (tid == 0) {
+        if (kDet)
+          for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
+        unsigned long long* st = p.stats + (size_t)i * ST_STRIDE;
+        st[ST_STEPS] = t + 1;
+        if (n_sent) atomicAdd(st + ST_SENT, n_sent);
+      }
     }
     asm volatile("fence.proxy.async;" ::: "memory");      // the refreshed bf16(-2w) is read by the next step's TMA
     __syncthreads();
