@@ -18,6 +18,8 @@
 //   lambda (buffer non-empty)   -- Eq. 3
 //   merged step                 -- Eq. 6 / Eq. 7, then  w <- w - eps * Dbar  (Algorithm 5)
 //   send                        -- Algorithm 5 "send w_{t+1} to random node != i"
+//   partial (per-centre) puts   -- Section 4.4: a message carries some of the centre rows, lambda and
+//                                  delta are then taken row by row (the reading is stated at worker_step_rows)
 //
 // Parity status: every function here is pinned by the CPU tests (brute force, closed forms,
 // special cases, invariants).  The free-running asynchronous mode of the CUDA library has no
@@ -49,7 +51,7 @@ inline uint64_t sm64(uint64_t x) {
 }
 
 // Stream tags: one independent stream per kind of draw.
-constexpr uint64_t TAG_PERM = 1, TAG_PEER = 2, TAG_SLOT = 3;
+constexpr uint64_t TAG_PERM = 1, TAG_PEER = 2, TAG_SLOT = 3, TAG_ROWS = 4;
 
 // h(seed, tag, a, b, c): chain of four SplitMix64 outputs, each keyed by the next coordinate.
 inline uint64_t draw(uint64_t seed, uint64_t tag, uint64_t a, uint64_t b, uint64_t c) {
@@ -66,10 +68,12 @@ struct Config {
   float eps;
   int32_t comm_interval, fanout, slots, parzen, shuffle;
   uint64_t seed;
+  int32_t partial_rows = 0;   // 0: a put carries the whole state; m >= 1: m centre rows (Section 4.4)
 };
 
 struct Slot {
   std::vector<float> v;   // last payload written into this receive buffer
+  std::vector<uint8_t> has;  // per centre row: 1 if the last message carried it (all 1 for whole-state messages)
   uint64_t seq = 0;       // number of messages ever written into it
   uint64_t seen = 0;      // value of seq when the owner last looked
 };
@@ -86,7 +90,9 @@ struct Worker {
   std::vector<double> d1, d2;      // b: smallest and second smallest squared distance
   std::vector<int64_t> counts;     // k
   std::vector<int32_t> acc;        // S: acceptance a_s of the last step (-1 = slot had nothing new)
-  std::vector<double> lhs, rhs;    // S: both sides of Eq. 4
+  std::vector<double> lhs, rhs;    // S: both sides of Eq. 4 (whole-state messages)
+  std::vector<int32_t> row_acc;    // S*k: per-row acceptance of the last step in per-centre mode (-1 = row not in a new message)
+  std::vector<double> row_lhs, row_rhs;   // S*k: both sides of Eq. 4 per row
 };
 
 struct Oracle {
@@ -141,6 +147,8 @@ inline void nearest(const float* x, const float* w, int k, int d, int32_t& best,
   }
 }
 
+void worker_step_rows(const Oracle& o, Worker& me, const std::vector<double>& D);
+
 // One externally-modified mini-batch step of one worker (Algorithm 5, the "update" line).
 void worker_step(const Oracle& o, Worker& me, int32_t i) {
   const Config& c = o.c;
@@ -172,6 +180,8 @@ void worker_step(const Oracle& o, Worker& me, int32_t i) {
       size_t e = (size_t)kk * d + j;
       D[e] = ((double)me.counts[kk] * (double)me.w[e] - S[e]) / (double)b;
     }
+
+  if (c.partial_rows > 0) { worker_step_rows(o, me, D); return; }
 
   // receive buffers: lambda (Eq. 3) and delta (Eq. 4)
   const int Sn = c.slots;
@@ -212,6 +222,70 @@ void worker_step(const Oracle& o, Worker& me, int32_t i) {
   }
 }
 
+// The same step when messages carry single centre rows (Section 4.4: "for K-Means we partition along the
+// individual cluster centers of the states").  The paper gives no formulas for this case; the reading
+// taken here applies Eq. 3, Eq. 4 and Eq. 6 to each centre row k on its own:
+//   lambda_{s,k} = 1 if buffer s holds a new message that carries row k and that row is not all zero,
+//   delta_{s,k}  = [ ||(w_k - eps D_k) - v_{s,k}||^2 < ||w_k - v_{s,k}||^2 ],
+//   Dbar_k = w_k - (w_k + sum_s a_{s,k} v_{s,k}) / (1 + sum_s a_{s,k}) + D_k,   a = lambda * delta.
+// A message counts as accepted ("good") when at least one of its rows was.
+void worker_step_rows(const Oracle& o, Worker& me, const std::vector<double>& D) {
+  const Config& c = o.c;
+  const int k = c.k, d = c.d, Sn = c.slots;
+  const size_t kd = (size_t)k * d;
+  const double eps = (double)c.eps;
+  me.acc.assign(Sn, -1); me.lhs.assign(Sn, 0.0); me.rhs.assign(Sn, 0.0);
+  me.row_acc.assign((size_t)Sn * k, -1); me.row_lhs.assign((size_t)Sn * k, 0.0); me.row_rhs.assign((size_t)Sn * k, 0.0);
+  std::vector<double> sumv(kd, 0.0);
+  std::vector<int> mrow(k, 0);
+  for (int s = 0; s < Sn; ++s) {
+    Slot& sl = me.mail[s];
+    if (sl.seq == sl.seen) continue;
+    me.received += 1;
+    me.overwritten += (sl.seq - sl.seen - 1);
+    sl.seen = sl.seq;
+    int good_rows = 0;
+    for (int kk = 0; kk < k; ++kk) {
+      if (!sl.has[kk]) continue;
+      double nv = 0.0, lhs = 0.0, rhs = 0.0;
+      for (int j = 0; j < d; ++j) {
+        size_t e = (size_t)kk * d + j;
+        double v = (double)sl.v[e], w = (double)me.w[e];
+        nv += v * v;
+        double a = (w - eps * D[e]) - v, r = w - v;
+        lhs += a * a; rhs += r * r;
+      }
+      int lambda = (nv > 0.0) ? 1 : 0;
+      int delta = c.parzen ? ((lhs < rhs) ? 1 : 0) : 1;
+      int a_sk = lambda * delta;
+      me.row_acc[(size_t)s * k + kk] = a_sk;
+      me.row_lhs[(size_t)s * k + kk] = lhs; me.row_rhs[(size_t)s * k + kk] = rhs;
+      if (a_sk) {
+        mrow[kk] += 1; good_rows += 1;
+        for (int j = 0; j < d; ++j) sumv[(size_t)kk * d + j] += (double)sl.v[(size_t)kk * d + j];
+      }
+    }
+    me.acc[s] = good_rows;
+    if (good_rows > 0) me.accepted += 1;
+  }
+  me.w_next.resize(kd);
+  for (int kk = 0; kk < k; ++kk)
+    for (int j = 0; j < d; ++j) {
+      size_t e = (size_t)kk * d + j;
+      double w = (double)me.w[e];
+      double Dbar = w - (w + sumv[e]) / (double)(1 + mrow[kk]) + D[e];
+      me.w_next[e] = (float)(w - eps * Dbar);
+    }
+}
+
+// Rows of the j-th message of worker i's put after step t in per-centre mode: m consecutive rows
+// (cyclically) from a drawn first row.
+void put_rows(const Config& c, int32_t i, uint64_t t, int32_t j, std::vector<uint8_t>& has) {
+  has.assign(c.k, 0);
+  const int32_t r0 = (int32_t)(draw(c.seed, TAG_ROWS, (uint64_t)i, t, (uint64_t)j) % (uint64_t)c.k);
+  for (int32_t q = 0; q < c.partial_rows; ++q) has[(r0 + q) % c.k] = 1;
+}
+
 // One synchronous round: every worker steps once from the states and buffers it had at the start
 // of the round; afterwards the round's puts are delivered, senders in ascending order, whole
 // messages at a time (so a later sender into the same buffer wins).
@@ -231,7 +305,14 @@ void round_once(Oracle& o) {
       recipients(c, i, t, peers.data(), slots.data());
       for (int j = 0; j < c.fanout; ++j) {
         Slot& sl = o.wk[peers[j]].mail[slots[j]];
-        sl.v = me.w_next;
+        if (c.partial_rows > 0) {
+          put_rows(c, i, t, j, sl.has);
+          for (int kk = 0; kk < c.k; ++kk)
+            if (sl.has[kk]) std::memcpy(sl.v.data() + (size_t)kk * c.d, me.w_next.data() + (size_t)kk * c.d, sizeof(float) * c.d);
+        } else {
+          sl.v = me.w_next;
+          sl.has.assign(c.k, 1);
+        }
         sl.seq += 1;
         me.sent += 1;
       }
@@ -274,7 +355,7 @@ void* oracle_create(int64_t N, int32_t d, int32_t k, int32_t W, int32_t b, float
     w.w.assign(w0, w0 + kd);
     w.w_next.assign(kd, 0.f);
     w.mail.resize(slots);
-    for (auto& s : w.mail) s.v.assign(kd, 0.f);
+    for (auto& s : w.mail) { s.v.assign(kd, 0.f); s.has.assign(k, 0); }
     make_perm(o->c, o->B, i, w.perm);
   }
   return o;
@@ -310,7 +391,43 @@ void oracle_put(void* h, int32_t worker, int32_t slot, const float* payload) {
   Oracle* o = (Oracle*)h;
   Slot& s = o->wk[worker].mail[slot];
   s.v.assign(payload, payload + (size_t)o->c.k * o->c.d);
+  s.has.assign(o->c.k, 1);
   s.seq += 1;
+}
+// Per-centre mode: m >= 1 rows per message (0 = whole-state messages).  Set before the first round.
+int oracle_set_partial_rows(void* h, int32_t m) {
+  Oracle* o = (Oracle*)h;
+  if (m < 0 || m > o->c.k) return -1;
+  o->c.partial_rows = m;
+  return 0;
+}
+// A put from outside that carries only the rows flagged in has[k].
+void oracle_put_rows(void* h, int32_t worker, int32_t slot, const float* payload, const uint8_t* has) {
+  Oracle* o = (Oracle*)h;
+  Slot& s = o->wk[worker].mail[slot];
+  s.v.assign(payload, payload + (size_t)o->c.k * o->c.d);
+  s.has.assign(has, has + o->c.k);
+  s.seq += 1;
+}
+// Rows of the j-th message of worker i's put after step t (flags, k of them).
+void oracle_put_row_flags(void* h, int32_t i, uint64_t t, int32_t j, uint8_t* out) {
+  Oracle* o = (Oracle*)h;
+  std::vector<uint8_t> has;
+  put_rows(o->c, i, t, j, has);
+  std::memcpy(out, has.data(), (size_t)o->c.k);
+}
+// Per-row trace of the last step in per-centre mode: acc[S*k] (-1 = row not in a new message), lhs, rhs.
+void oracle_last_step_rows(void* h, int32_t worker, int32_t* acc, double* lhs, double* rhs) {
+  Worker& w = ((Oracle*)h)->wk[worker];
+  if (w.row_acc.empty()) return;
+  if (acc) std::memcpy(acc, w.row_acc.data(), sizeof(int32_t) * w.row_acc.size());
+  if (lhs) std::memcpy(lhs, w.row_lhs.data(), sizeof(double) * w.row_lhs.size());
+  if (rhs) std::memcpy(rhs, w.row_rhs.data(), sizeof(double) * w.row_rhs.size());
+}
+// has[k] flags of a receive buffer's last message.
+void oracle_get_mail_rows(void* h, int32_t worker, int32_t slot, uint8_t* out) {
+  Oracle* o = (Oracle*)h;
+  std::memcpy(out, o->wk[worker].mail[slot].has.data(), (size_t)o->c.k);
 }
 // Content and counters of a receive buffer: out[k*d], seq_seen[2] = {seq, seen}.
 void oracle_get_mail(void* h, int32_t worker, int32_t slot, float* out, uint64_t* seq_seen) {

@@ -58,6 +58,12 @@ def lib():
         L.oracle_eval.argtypes = [vp, i64, i32, vp, i32, C.c_int]
         L.oracle_eval.restype = C.c_double
         L.oracle_max_threads.restype = C.c_int
+        L.oracle_set_partial_rows.argtypes = [vp, i32]
+        L.oracle_set_partial_rows.restype = C.c_int
+        L.oracle_put_rows.argtypes = [vp, i32, i32, vp, vp]
+        L.oracle_put_row_flags.argtypes = [vp, i32, u64, i32, vp]
+        L.oracle_last_step_rows.argtypes = [vp, i32, vp, vp, vp]
+        L.oracle_get_mail_rows.argtypes = [vp, i32, i32, vp]
         _lib = L
     return _lib
 
@@ -114,7 +120,7 @@ class Oracle:
     """Deterministic, round-synchronous ASGD over W workers on the host."""
 
     def __init__(self, X, w0, *, W, b, eps, comm_interval=0, fanout=0, slots=None, parzen=1,
-                 shuffle=1, seed=0, threads=1):
+                 shuffle=1, seed=0, threads=1, partial_rows=0):
         self.X = _f32(X)
         w0 = _f32(w0)
         self.N, self.d = self.X.shape
@@ -128,6 +134,9 @@ class Oracle:
         if not self._h:
             raise ValueError("oracle_create rejected the configuration")
         self.threads = lib().oracle_set_threads(self._h, int(threads))
+        self.partial_rows = int(partial_rows)
+        if lib().oracle_set_partial_rows(self._h, self.partial_rows) != 0:
+            raise ValueError("partial_rows must lie in 0..k")
         self.H = int(lib().oracle_shard_rows(self._h))
         self.B = int(lib().oracle_batches_per_pass(self._h))
 
@@ -197,3 +206,31 @@ class Oracle:
         rhs = np.empty(self.S, np.float64)
         lib().oracle_last_step(self._h, worker, _p(a), _p(d1), _p(d2), _p(cnt), _p(acc), _p(lhs), _p(rhs))
         return dict(assign=a, d1=d1, d2=d2, counts=cnt, accept=acc, lhs=lhs, rhs=rhs)
+
+    # ---- per-centre messages (Section 4.4) ----
+    def put_rows(self, worker: int, slot: int, payload, has):
+        """External put that carries only the centre rows flagged in has[k]."""
+        v = _f32(payload)
+        assert v.shape == (self.k, self.d)
+        hs = np.ascontiguousarray(np.asarray(has, dtype=np.uint8))
+        assert hs.shape == (self.k,)
+        lib().oracle_put_rows(self._h, worker, slot, _p(v), _p(hs))
+
+    def put_row_flags(self, worker: int, t: int, j: int):
+        """Rows (k flags) of the j-th message of the put worker makes after its step t."""
+        out = np.zeros(self.k, np.uint8)
+        lib().oracle_put_row_flags(self._h, worker, int(t), int(j), _p(out))
+        return out
+
+    def mail_rows(self, worker: int, slot: int):
+        out = np.zeros(self.k, np.uint8)
+        lib().oracle_get_mail_rows(self._h, worker, slot, _p(out))
+        return out
+
+    def last_step_rows(self, worker: int):
+        """Per-row trace of the last step in per-centre mode: accept[S, k] (-1 = row not in a new message), lhs, rhs."""
+        acc = np.full((self.S, self.k), -1, np.int32)
+        lhs = np.zeros((self.S, self.k), np.float64)
+        rhs = np.zeros((self.S, self.k), np.float64)
+        lib().oracle_last_step_rows(self._h, worker, _p(acc), _p(lhs), _p(rhs))
+        return dict(accept=acc, lhs=lhs, rhs=rhs)

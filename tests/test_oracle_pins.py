@@ -389,3 +389,124 @@ def test_communication_pulls_workers_together():
             assert spread(o) < s0
         else:
             assert spread(o) == pytest.approx(s0)
+
+
+# ---------------------------------------------------------------------------------------------
+# Per-centre messages (Section 4.4): a put carries some of the centre rows; lambda, delta and the
+# merge are taken row by row.
+# ---------------------------------------------------------------------------------------------
+def test_partial_rows_1d_hand_cases():
+    for line in open(os.path.join(GOLD, "partial_rows_1d_cases.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = [float(s) for s in line.split()]
+        w0, w1, x0, x1, eps, v0, v1 = f[:7]
+        has = [int(f[7]), int(f[8])]
+        parzen, a0, a1 = int(f[9]), int(f[10]), int(f[11])
+        want = f[12:14]
+        batch = np.array([[x0], [x1], [x0], [x1]], np.float32)
+        X = np.vstack([batch, batch])
+        o = orc.Oracle(X, np.array([[w0], [w1]], np.float32), W=2, b=4, eps=eps, comm_interval=0, fanout=1,
+                       parzen=parzen, shuffle=0, partial_rows=1)
+        o.put_rows(0, 0, np.array([[v0], [v1]], np.float32), has)
+        o.rounds(1)
+        tr = o.last_step_rows(0)
+        got = [int(tr["accept"][0, r]) if has[r] else 0 for r in range(2)]
+        assert got == [a0, a1], line
+        for r in range(2):
+            if not has[r]:
+                assert tr["accept"][0, r] == -1, line          # the row was not in the message
+        assert np.allclose(o.state(0)[:, 0], want, atol=1e-6), line
+        # the worker that got nothing takes the plain local step on both rows
+        plain = [w0 - eps * (w0 - x0) / 2, w1 - eps * (w1 - x1) / 2]
+        assert np.allclose(o.state(1)[:, 0], plain, atol=1e-6), line
+        st = o.stats(0)
+        assert st["received"] == 1 and st["accepted"] == int(a0 + a1 > 0), line
+        assert o.last_step(0)["accept"][0] == a0 + a1, line      # accepted rows of the message
+
+
+def test_partial_rows_single_centre_equals_whole_state_messages():
+    # with k = 1 a row is the whole state: both modes must give the same trajectory bit for bit
+    rng = np.random.default_rng(3)
+    X = (rng.normal(size=(6000, 3)) + np.array([4.0, -2.0, 1.0])).astype(np.float32)
+    w0 = np.array([[0.5, 0.5, 0.5]], np.float32)
+    kw = dict(W=6, b=40, eps=0.2, comm_interval=2, fanout=2, slots=2, seed=11)
+    a = orc.Oracle(X, w0, **kw)
+    c = orc.Oracle(X, w0, partial_rows=1, **kw)
+    a.rounds(25)
+    c.rounds(25)
+    assert np.array_equal(a.states(), c.states())
+    sa, sc = [a.stats(i) for i in range(6)], [c.stats(i) for i in range(6)]
+    assert sa == sc and sum(s["accepted"] for s in sa) > 0
+
+
+def test_partial_rows_rows_outside_the_message_take_the_plain_step():
+    # closed form per row: a row the message does not carry moves exactly as with no communication,
+    # a carried row follows Eq. 6 with its own delta (checked in the inner-product form of Eq. 4)
+    eps = 0.3
+    rng = np.random.default_rng(21)
+    seen_accept = seen_reject = 0
+    for trial in range(30):
+        X, w, D = _known_gradient_problem(seed=trial, k=3, d=4, b=30)
+        v = (w + rng.normal(size=w.shape) * eps * np.abs(D).max()).astype(np.float32)
+        has = np.zeros(3, np.uint8)
+        has[rng.choice(3, size=int(rng.integers(1, 3)), replace=False)] = 1
+        Xd = np.vstack([X, X])
+        o = orc.Oracle(Xd, w, W=2, b=X.shape[0], eps=eps, shuffle=0, comm_interval=0, fanout=1, partial_rows=2)
+        o.put_rows(0, 0, v, has)
+        o.rounds(1)
+        tr = o.last_step_rows(0)
+        wd, vd = w.astype(np.float64), v.astype(np.float64)
+        e = float(np.float32(eps))
+        got = o.state(0).astype(np.float64)
+        for r in range(3):
+            plain = wd[r] - e * D[r]
+            if not has[r]:
+                assert tr["accept"][0, r] == -1
+                assert np.allclose(got[r], plain, rtol=0, atol=1e-6)
+                continue
+            margin = 2 * (D[r] * (wd[r] - vd[r])).sum() - e * (D[r] ** 2).sum()
+            if abs(margin) < 1e-9:
+                continue
+            acc = int(margin > 0)
+            assert tr["accept"][0, r] == acc
+            merged = wd[r] - e * (acc * (wd[r] - (wd[r] + vd[r]) / 2) + D[r])
+            assert np.allclose(got[r], merged, rtol=0, atol=1e-6)
+            seen_accept += acc
+            seen_reject += 1 - acc
+    assert seen_accept >= 5 and seen_reject >= 5
+
+
+def test_partial_rows_schedule_and_delivery():
+    k, d, W, m = 7, 2, 5, 3
+    rng = np.random.default_rng(5)
+    X = rng.normal(size=(5 * 40, d)).astype(np.float32)
+    w0 = X[:k].copy()
+    o = orc.Oracle(X, w0, W=W, b=8, eps=0.1, comm_interval=1, fanout=2, slots=3, seed=77, partial_rows=m)
+    firsts = []
+    for t in range(300):
+        for i in range(W):
+            for j in range(2):
+                fl = o.put_row_flags(i, t, j)
+                assert fl.sum() == m
+                r0 = [r for r in range(k) if fl[r] and not fl[(r - 1) % k]]
+                assert len(r0) == 1                       # one cyclic run of m consecutive rows
+                assert all(fl[(r0[0] + q) % k] for q in range(m))
+                firsts.append(r0[0])
+    cnt = np.bincount(firsts, minlength=k)
+    expect = len(firsts) / k
+    assert ((cnt - expect) ** 2 / expect).sum() < 30.0     # chi-square, 6 degrees of freedom (p ~ 1e-5 at 30)
+    # delivery: after one round a buffer holds the carried rows of the LAST sender's new state, flags of that message
+    o.rounds(1)
+    writers = {}
+    for i in range(W):
+        peers, slots = o.recipients(i, 0)
+        for j in range(2):
+            writers[(int(peers[j]), int(slots[j]))] = (i, j)        # ascending sender order: the last one stays
+    assert writers
+    for (r, s), (i, j) in writers.items():
+        payload, seq, seen = o.mail(r, s)
+        fl = o.put_row_flags(i, 0, j)
+        assert np.array_equal(o.mail_rows(r, s), fl)
+        assert np.array_equal(payload[fl == 1], o.state(i)[fl == 1])
+        assert seq >= 1 and seen == 0
