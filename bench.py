@@ -98,11 +98,11 @@ class ClockSampler:
         return out
 
 
-def algorithmic_bytes_per_pass(wl, steps):
-    """One read of every used sample (d*4 B) plus the put payloads (k*d*4 B per recipient per put)."""
+def algorithmic_bytes_per_pass(wl, steps, partial_rows=0):
+    """One read of every used sample (d*4 B) plus the put payloads (rows*d*4 B per recipient per put)."""
     sample_bytes = wl.W * steps * wl.b * wl.d * 4
     puts = wl.W * wl.fanout * (steps // wl.comm_interval if wl.comm_interval > 0 else 0)
-    return sample_bytes + puts * wl.k * wl.d * 4
+    return sample_bytes + puts * (partial_rows if partial_rows > 0 else wl.k) * wl.d * 4
 
 
 def cpu_baseline(wl, sample_rows, threads=None, min_seconds=0.0):
@@ -177,6 +177,11 @@ def main():
     ap.add_argument("--reference-rows", type=int, default=1 << 23)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    # points of the worker / communication sweep and the ablations (the defaults are the workload's own values)
+    ap.add_argument("--workers", type=int, default=0, help="W")
+    ap.add_argument("--comm-interval", type=int, default=-1, help="c; 0 = silent (no puts)")
+    ap.add_argument("--no-parzen", action="store_true", help="accept every non-empty message (Eq. 3 without Eq. 4)")
+    ap.add_argument("--partial-rows", type=int, default=0, help="centre rows per message (Section 4.4); 0 = whole state")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -194,12 +199,17 @@ def main():
     wl = inputs.WORKLOADS[args.workload]
     if args.rows:
         wl = wl.scaled(N=args.rows)
+    if args.workers:
+        wl = wl.scaled(W=args.workers)
+    if args.comm_interval >= 0:
+        wl = wl.scaled(comm_interval=args.comm_interval)
     # each rank owns an independent group of W workers on its own seeded shard (no cross-GPU exchange)
     wl_rank = wl.scaled(seed=dist.shard_seed(wl.seed, rank, world))
     X, _ = inputs.make_samples(wl_rank, device=dev)
     w0 = inputs.initial_centres(wl_rank, X)
     cfg = pkg.make_config(N=wl.N, d=wl.d, k=wl.k, W=wl.W, b=wl.b, eps=wl.eps, comm_interval=wl.comm_interval,
-                          fanout=wl.fanout, seed=wl_rank.seed)
+                          fanout=wl.fanout, seed=wl_rank.seed, parzen=0 if args.no_parzen else 1,
+                          partial_rows=args.partial_rows)
     ctx = pkg.Asgd(cfg, X, w0)
     steps = wl.B                                   # one pass
     samples_per_pass = wl.W * steps * wl.b
@@ -226,11 +236,17 @@ def main():
     total_ms = dist.max_over_ranks(ev[0].elapsed_time(ev[-1]))
     value = world * samples_per_pass * args.steps / (total_ms * 1e-3)
     E_final = ctx.eval(0)
+    E_mean = ctx.eval(-1)
+    msgs = {"sent": 0, "received": 0, "accepted": 0, "overwritten": 0}
+    for i in range(wl.W):
+        st = ctx.get_stats(i)
+        for key in msgs:
+            msgs[key] += st[key]
 
     # roofline of the dominant kernel (the persistent worker kernel: one launch per bench step)
     peak, peak_kind = measured_peaks()
     launch_ms = statistics.mean(per_launch_ms)
-    bytes_per_launch = algorithmic_bytes_per_pass(wl, steps)
+    bytes_per_launch = algorithmic_bytes_per_pass(wl, steps, args.partial_rows)
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
     traffic = None
     with open(os.path.join(ROOT, "paper_1505_04956_b200", "csrc", "asgd_stream.cuh"), "rb") as f:
@@ -293,11 +309,12 @@ def main():
             "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "k": wl.k, "W": wl.W, "b": wl.b, "eps": wl.eps,
-                       "comm_interval": wl.comm_interval, "fanout": wl.fanout, "mode": "free-running",
+                       "comm_interval": wl.comm_interval, "fanout": wl.fanout, "parzen": 0 if args.no_parzen else 1,
+                       "partial_rows": args.partial_rows, "mode": "free-running",
                        "steps_per_worker_per_bench_step": steps, "parallelism": "dp%d" % world,
                        "l2": "inputs larger than L2 (%.2f GB per pass)" % (bytes_per_launch / 1e9)},
             "roofline": roofline_alu or roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "quantization_error_worker0": E_final,
+            "quantization_error_worker0": E_final, "quantization_error_mean_state": E_mean, "messages": msgs, "messages_over_passes": args.warmup + args.steps,
         }
         print(json.dumps(line), flush=True)
     dist.shutdown()

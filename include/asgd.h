@@ -70,7 +70,7 @@ typedef struct asgd_config {
   int32_t dist_path;     /* ASGD_PATH_*                                                       */
   int32_t shuffle;       /* 1 = seeded permutation of each worker's batch order, 0 = in order */
   int32_t record_assign; /* 1 = keep the last step's assignments for asgd_get_assign()        */
-  int32_t reserved;      /* must be 0                                                         */
+  int32_t partial_rows;  /* 0 = a put carries the whole state; m in 1..k = m centre rows      */
   uint64_t seed;         /* batch order, recipients, buffer choice                            */
 } asgd_config;
 
@@ -115,6 +115,23 @@ int asgd_get_state(asgd_ctx *ctx, int32_t worker, float *out_dev);
 int asgd_set_state(asgd_ctx *ctx, int32_t worker, const float *w_dev /* DEVICE [k*d] */);
 /* A put from outside: write a whole message into receive buffer `slot` of `worker`. */
 int asgd_put(asgd_ctx *ctx, int32_t worker, int32_t slot, const float *payload_dev /* DEVICE [k*d] */);
+
+/* Per-centre messages (Section 4.4: updates are partitioned "along the individual cluster centers"),
+ * cfg.partial_rows = m >= 1.  The paper states no formulas for them; the library applies Eq. 3, Eq. 4
+ * and Eq. 6 to each centre row on its own: a put after step t carries the m consecutive rows (cyclic)
+ * that start at row h(seed, 4, i, t, j) mod k of the sender's new state; for every new message that
+ * carries row a, lambda is "the row is not all zero", delta compares ||(w_a - eps D_a) - v_a|| with
+ * ||w_a - v_a||, and row a is merged with its own count of accepted rows.  A message counts as accepted
+ * when at least one of its rows was.  asgd_put then writes a message that carries every row.
+ *
+ * asgd_put_rows: a put from outside carrying rows [first_row, first_row + n_rows) (cyclic) of
+ * payload_dev (DEVICE [k*d]; other rows are not read).  ASGD_EINVAL unless cfg.partial_rows >= 1. */
+int asgd_put_rows(asgd_ctx *ctx, int32_t worker, int32_t slot, const float *payload_dev, int32_t first_row,
+                  int32_t n_rows);
+/* Per-row acceptance of the last step of `worker` in per-centre mode: out_host[S*k], entry [s*k + a] is
+ * -1 when buffer s held no new message carrying row a, else 0 (rejected) or 1 (accepted).  Synchronises.
+ * asgd_get_accept then gives the number of accepted rows per buffer (-1 nothing new). */
+int asgd_get_accept_rows(asgd_ctx *ctx, int32_t worker, int32_t *out_host /* HOST [S*k] */);
 
 /* Eq. 8: E(w) of the given worker's state (-1 = mean state) over all N rows.  Synchronises. */
 int asgd_eval(asgd_ctx *ctx, int32_t worker, double *E_host /* HOST out */);

@@ -16,7 +16,7 @@ PATH_AUTO, PATH_FP32, PATH_TC_3XTF32, PATH_TC_BF16, PATH_FP32_GENERAL = 0, 1, 2,
 
 EXPORTS = (
     "asgd_workspace_bytes", "asgd_init", "asgd_step", "asgd_run", "asgd_get_state", "asgd_set_state",
-    "asgd_put", "asgd_eval", "asgd_get_stats", "asgd_get_assign", "asgd_get_accept", "asgd_sync",
+    "asgd_put", "asgd_put_rows", "asgd_get_accept_rows", "asgd_eval", "asgd_get_stats", "asgd_get_assign", "asgd_get_accept", "asgd_sync",
     "asgd_launch_count", "asgd_path_name", "asgd_last_cuda_error", "asgd_strerror", "asgd_destroy",
     "asgd_fit_host_bytes", "asgd_fit_host", "asgd_eval_noalloc",
 )
@@ -28,7 +28,7 @@ class AsgdConfig(C.Structure):
         ("N", C.c_int64), ("d", C.c_int32), ("k", C.c_int32), ("W", C.c_int32), ("b", C.c_int32),
         ("eps", C.c_float), ("comm_interval", C.c_int32), ("fanout", C.c_int32), ("slots", C.c_int32),
         ("parzen", C.c_int32), ("dist_path", C.c_int32), ("shuffle", C.c_int32),
-        ("record_assign", C.c_int32), ("reserved", C.c_int32), ("seed", C.c_uint64),
+        ("record_assign", C.c_int32), ("partial_rows", C.c_int32), ("seed", C.c_uint64),
     ]
 
 
@@ -62,6 +62,8 @@ def load():
     L.asgd_get_state.argtypes = [vp, i32, vp]
     L.asgd_set_state.argtypes = [vp, i32, vp]
     L.asgd_put.argtypes = [vp, i32, i32, vp]
+    L.asgd_put_rows.argtypes = [vp, i32, i32, vp, i32, i32]
+    L.asgd_get_accept_rows.argtypes = [vp, i32, C.POINTER(C.c_int32)]
     L.asgd_eval.argtypes = [vp, i32, C.POINTER(C.c_double)]
     L.asgd_get_stats.argtypes = [vp, i32, C.POINTER(C.c_uint64)]
     L.asgd_get_assign.argtypes = [vp, vp]
@@ -88,10 +90,10 @@ def strerror(status: int) -> str:
 
 
 def make_config(*, N, d, k, W, b, eps, comm_interval=0, fanout=0, slots=None, parzen=1,
-                dist_path=PATH_AUTO, shuffle=1, record_assign=0, seed=0) -> AsgdConfig:
+                dist_path=PATH_AUTO, shuffle=1, record_assign=0, seed=0, partial_rows=0) -> AsgdConfig:
     return AsgdConfig(int(N), int(d), int(k), int(W), int(b), float(eps), int(comm_interval), int(fanout),
                       int(slots) if slots else max(1, int(fanout)), int(parzen), int(dist_path), int(shuffle),
-                      int(record_assign), 0, int(seed))
+                      int(record_assign), int(partial_rows), int(seed))
 
 
 def asgd_workspace_bytes(cfg: AsgdConfig) -> int:
@@ -184,6 +186,17 @@ class Asgd:
     def put(self, worker: int, slot: int, payload):
         assert payload.is_cuda and payload.is_contiguous() and payload.numel() == self.k * self.d
         self._chk(self._L.asgd_put(self._h, int(worker), int(slot), C.c_void_p(payload.data_ptr())), "asgd_put")
+
+    def put_rows(self, worker: int, slot: int, payload, first_row: int, n_rows: int):
+        assert payload.is_cuda and payload.is_contiguous() and payload.numel() == self.k * self.d
+        self._chk(self._L.asgd_put_rows(self._h, int(worker), int(slot), C.c_void_p(payload.data_ptr()), int(first_row),
+                                        int(n_rows)), "asgd_put_rows")
+
+    def get_accept_rows(self, worker: int):
+        """[S][k] per-row acceptance of the worker's last step in per-centre mode (-1, 0, 1)."""
+        out = (C.c_int32 * (self.S * self.k))()
+        self._chk(self._L.asgd_get_accept_rows(self._h, int(worker), out), "asgd_get_accept_rows")
+        return [[int(out[s * self.k + a]) for a in range(self.k)] for s in range(self.S)]
 
     def eval(self, worker: int = 0) -> float:
         e = C.c_double(0.0)

@@ -31,7 +31,7 @@ enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2, P_TC_BF16 = 3 };
 #define ASGD_TILED_SHAPES(X) X(32, 64, 4, 2, 2) X(128, 128, 4, 4, 1)
 
 struct Layout {
-  size_t state, mail, seq, seen, arb_win, arb_cnt, stats, perm, status, assign_rec, accept_rec, gsum,
+  size_t state, mail, seq, seen, arb_win, arb_cnt, mail_rows, rowacc, rowin, stats, perm, status, assign_rec, accept_rec, gsum,
       eval_partial, tmp_state, xmax, wbf, top2, xbf, total;
 };
 
@@ -47,7 +47,7 @@ bool config_ok(const asgd_config* c) {
   if (!(c->eps > 0.f)) return false;
   if (c->comm_interval < 0 || c->fanout < 0 || c->fanout > c->W - 1 || c->fanout > MAX_FANOUT) return false;
   if (c->slots < 1 || c->slots > MAX_SLOTS) return false;
-  if (c->reserved != 0) return false;
+  if (c->partial_rows < 0 || c->partial_rows > c->k) return false;
   if (c->dist_path < ASGD_PATH_AUTO || c->dist_path > ASGD_PATH_FP32_GENERAL) return false;
   if ((long long)c->k * c->d > (1ll << 28)) return false;
   const long long H = c->N / c->W;
@@ -75,6 +75,9 @@ Layout make_layout(const asgd_config* c) {
   L.seen = take(W * S * 4);
   L.arb_win = take(W * S * 4);
   L.arb_cnt = take(W * S * 4);
+  L.mail_rows = take(W * S * 8);
+  L.rowacc = take(c->partial_rows > 0 ? W * (size_t)c->k * 4 : 4);
+  L.rowin = take(c->partial_rows > 0 ? W * (size_t)c->k * 4 : 4);
   L.stats = take(W * ST_STRIDE * 8);
   L.perm = take(W * B * 4);
   L.status = take(64);
@@ -364,6 +367,10 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   p.status = (int*)(c->ws + L.status);
   p.assign_rec = cfg->record_assign ? (int*)(c->ws + L.assign_rec) : nullptr;
   p.accept_rec = (int*)(c->ws + L.accept_rec);
+  p.rows_m = cfg->partial_rows;
+  p.mail_rows = (int2*)(c->ws + L.mail_rows);
+  p.rowacc = (unsigned*)(c->ws + L.rowacc);
+  p.rowin = (unsigned*)(c->ws + L.rowin);
   p.gsum = (float*)(c->ws + L.gsum);
   p.xmax2 = 0.f;
   p.wbf = nullptr;
@@ -448,7 +455,20 @@ int asgd_put(asgd_ctx* c, int32_t worker, int32_t slot, const float* payload_dev
   if (!c || !payload_dev || worker < 0 || worker >= c->p.W || slot < 0 || slot >= c->p.S) return ASGD_EINVAL;
   const Params& p = c->p;
   const size_t ri = (size_t)worker * p.S + slot;
+  if (p.rows_m > 0) return asgd_put_rows(c, worker, slot, payload_dev, 0, p.k);      // a whole message carries every row
   external_put_kernel<<<1, 256, 0, c->stream>>>(p.mail + ri * (size_t)p.kd_pad, payload_dev, p.seq + ri, p.kd);
+  c->launches += 1;
+  CU(c, cudaGetLastError());
+  return ASGD_OK;
+}
+
+int asgd_put_rows(asgd_ctx* c, int32_t worker, int32_t slot, const float* payload_dev, int32_t first_row, int32_t n_rows) {
+  if (!c || !payload_dev || worker < 0 || worker >= c->p.W || slot < 0 || slot >= c->p.S) return ASGD_EINVAL;
+  const Params& p = c->p;
+  if (p.rows_m <= 0 || first_row < 0 || first_row >= p.k || n_rows < 1 || n_rows > p.k) return ASGD_EINVAL;
+  const size_t ri = (size_t)worker * p.S + slot;
+  external_put_rows_kernel<<<1, 256, 0, c->stream>>>(p.mail + ri * (size_t)p.kd_pad, payload_dev, p.seq + ri, p.mail_rows + ri,
+                                                     p.k, p.d, first_row, n_rows);
   c->launches += 1;
   CU(c, cudaGetLastError());
   return ASGD_OK;
@@ -502,6 +522,21 @@ int asgd_get_accept(asgd_ctx* c, int32_t worker, int32_t* out_host) {
   if (!c || !out_host || worker < 0 || worker >= c->p.W) return ASGD_EINVAL;
   CU(c, cudaMemcpyAsync(out_host, c->p.accept_rec + (size_t)worker * c->p.S, (size_t)c->p.S * 4, cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
+  return ASGD_OK;
+}
+
+int asgd_get_accept_rows(asgd_ctx* c, int32_t worker, int32_t* out_host) {
+  if (!c || !out_host || worker < 0 || worker >= c->p.W) return ASGD_EINVAL;
+  const Params& p = c->p;
+  if (p.rows_m <= 0) return ASGD_EINVAL;
+  std::vector<unsigned> acc, in;
+  try { acc.resize(p.k); in.resize(p.k); } catch (...) { return ASGD_ENOMEM; }
+  CU(c, cudaMemcpyAsync(acc.data(), p.rowacc + (size_t)worker * p.k, (size_t)p.k * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaMemcpyAsync(in.data(), p.rowin + (size_t)worker * p.k, (size_t)p.k * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU(c, cudaStreamSynchronize(c->stream));
+  for (int s = 0; s < p.S; ++s)
+    for (int a = 0; a < p.k; ++a)
+      out_host[(size_t)s * p.k + a] = ((in[a] >> s) & 1u) ? (int32_t)((acc[a] >> s) & 1u) : -1;
   return ASGD_OK;
 }
 

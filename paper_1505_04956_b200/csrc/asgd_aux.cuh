@@ -23,9 +23,25 @@ __global__ void deliver_kernel(const Params p) {
   const unsigned win = p.arb_win[ri];
   if (win == 0) return;
   const int sender = (int)((win - 1u) / (unsigned)p.f);
-  const float4* src = reinterpret_cast<const float4*>(p.state + (size_t)sender * p.kd_pad);
-  float4* dst = reinterpret_cast<float4*>(p.mail + ri * (size_t)p.kd_pad);
-  for (int e = threadIdx.x; e < p.kd_pad / 4; e += blockDim.x) dst[e] = src[e];
+  if (p.rows_m > 0) {
+    // per-centre message: the rows the sender drew for this message of the step it has just finished
+    const int j = (int)((win - 1u) % (unsigned)p.f);
+    const unsigned long long t = p.stats[(size_t)sender * ST_STRIDE + ST_STEPS] - 1ull;
+    const int r0 = sched_first_row(p, sender, t, j);
+    const float* src = p.state + (size_t)sender * p.kd_pad;
+    float* dst = p.mail + ri * (size_t)p.kd_pad;
+    for (int q = threadIdx.x; q < p.rows_m * p.d; q += blockDim.x) {
+      int a = r0 + q / p.d;
+      if (a >= p.k) a -= p.k;
+      const int e = a * p.d + q % p.d;
+      dst[e] = src[e];
+    }
+    if (threadIdx.x == 0) p.mail_rows[ri] = make_int2(r0, p.rows_m);
+  } else {
+    const float4* src = reinterpret_cast<const float4*>(p.state + (size_t)sender * p.kd_pad);
+    float4* dst = reinterpret_cast<float4*>(p.mail + ri * (size_t)p.kd_pad);
+    for (int e = threadIdx.x; e < p.kd_pad / 4; e += blockDim.x) dst[e] = src[e];
+  }
   __syncthreads();
   if (threadIdx.x == 0) {
     p.seq[ri] += p.arb_cnt[ri];
@@ -39,6 +55,16 @@ __global__ void external_put_kernel(float* dst, const float* src, unsigned* seq,
   for (int e = threadIdx.x; e < kd; e += blockDim.x) dst[e] = src[e];
   __syncthreads();
   if (threadIdx.x == 0) red_release_gpu_inc(seq);
+}
+// The same for a per-centre message: rows [r0, r0 + m) cyclically, their description, then the sequence number.
+__global__ void external_put_rows_kernel(float* dst, const float* src, unsigned* seq, int2* rows, int k, int d, int r0, int m) {
+  for (int q = threadIdx.x; q < m * d; q += blockDim.x) {
+    int a = r0 + q / d;
+    if (a >= k) a -= k;
+    dst[a * d + q % d] = src[a * d + q % d];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) { *rows = make_int2(r0, m); red_release_gpu_inc(seq); }
 }
 
 // Aggregation variant of Section 4.3: out = (1/W) sum_i w^i, summed in ascending worker order.

@@ -37,6 +37,10 @@ struct Params {
   float xmax2;             // max_i ||x_i||^2 over X (error bound of the tensor-core path)
   void* wbf;               // [W][k][d] bf16 copies of -2w (tensor-core path)
   float* top2;             // [W][b][2] running (minimum, runner-up) scores (tensor-core path)
+  int rows_m;              // per-centre messages (Section 4.4): centre rows per message, 0 = whole-state messages
+  int2* mail_rows;         // [W][S] (first row, number of rows) of the buffer's last message (per-centre mode)
+  unsigned* rowacc;        // [W][k] bit s: row accepted from buffer s in the worker's last step (per-centre mode)
+  unsigned* rowin;         // [W][k] bit s: buffer s held a new message carrying the row
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -48,7 +52,7 @@ __host__ __device__ inline unsigned long long splitmix_first(unsigned long long 
   z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
   return z ^ (z >> 31);
 }
-enum : unsigned long long { TAG_PERM = 1, TAG_PEER = 2, TAG_SLOT = 3 };
+enum : unsigned long long { TAG_PERM = 1, TAG_PEER = 2, TAG_SLOT = 3, TAG_ROWS = 4 };
 __host__ __device__ inline unsigned long long sched_draw(unsigned long long seed, unsigned long long tag,
                                                          unsigned long long a, unsigned long long b,
                                                          unsigned long long c) {
@@ -74,6 +78,17 @@ __device__ inline int sched_peer(const Params& p, int i, unsigned long long t, i
 __device__ inline int sched_slot(const Params& p, int i, unsigned long long t, int j) {
   return (int)(sched_draw(p.seed, TAG_SLOT, (unsigned long long)i, t, (unsigned long long)j) %
                (unsigned long long)p.S);
+}
+// Per-centre messages: first of the rows_m consecutive (cyclic) centre rows of the j-th message.
+__device__ inline int sched_first_row(const Params& p, int i, unsigned long long t, int j) {
+  return (int)(sched_draw(p.seed, TAG_ROWS, (unsigned long long)i, t, (unsigned long long)j) %
+               (unsigned long long)p.k);
+}
+// Is row a among the m rows that start (cyclically) at r0?
+__device__ inline bool row_in_run(int a, int r0, int m, int k) {
+  int off = a - r0;
+  if (off < 0) off += k;
+  return off < m;
 }
 
 // ---------------------------------------------------------------------------------------------

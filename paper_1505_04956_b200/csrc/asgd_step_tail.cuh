@@ -1,6 +1,7 @@
 // Second half of a worker's step, shared by every distance path: local gradient (Eq. 9), receive
 // buffers with lambda (Eq. 3) and the Parzen test (Eq. 4), merged update (Eq. 6 / Eq. 7 and the
-// update line of Algorithm 5), and the send line of Algorithm 5.
+// update line of Algorithm 5), and the send line of Algorithm 5.  With per-centre messages
+// (Section 4.4, Params::rows_m > 0) lambda, delta and the merge are taken centre row by centre row.
 #pragma once
 
 #include "asgd_common.cuh"
@@ -66,6 +67,25 @@ __device__ inline unsigned long long step_send(const Params& p, int i, unsigned 
       atomicMax(p.arb_win + ri, (unsigned)(i * p.f + tid + 1));
       atomicAdd(p.arb_cnt + ri, 1u);
     }
+  } else if (p.rows_m > 0) {
+    // per-centre message: rows_m consecutive (cyclic) rows, then their description, then the release
+    for (int j = 0; j < p.f; ++j) {
+      const size_t ri = (size_t)ts->peers[j] * p.S + ts->pslots[j];
+      float* dst = p.mail + ri * (size_t)p.kd_pad;
+      const int r0 = sched_first_row(p, i, t, j);
+      const int per_row = d / V;
+      for (int q = tid; q < p.rows_m * per_row; q += nt) {
+        int a = r0 + q / per_row;
+        if (a >= p.k) a -= p.k;
+        const int e = a * d + (q % per_row) * V;
+        tail_st<V>(dst + e, tail_ld<V>(w + widx(e)));
+      }
+      __syncthreads();
+      if (tid == 0) {
+        p.mail_rows[ri] = make_int2(r0, p.rows_m);
+        red_release_gpu_inc(p.seq + ri);
+      }
+    }
   } else {
     for (int j = 0; j < p.f; ++j) {
       const size_t ri = (size_t)ts->peers[j] * p.S + ts->pslots[j];
@@ -126,47 +146,96 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
     }
   }
   __syncthreads();
-  for (int s = 0; s < p.S; ++s) {
-    const size_t si = (size_t)i * p.S + s;
-    const bool fresh = ts->fresh[s] != 0;
-    int acc = -1;
-    if (fresh) {
-      const float* __restrict__ v = p.mail + si * (size_t)p.kd_pad;
-      double dot = 0.0, dd = 0.0, nv = 0.0;
+  const bool by_rows = p.rows_m > 0;
+  unsigned whole_bits = 0;                                   // whole-state messages: buffers accepted in this step
+  unsigned* rowacc = by_rows ? p.rowacc + (size_t)i * p.k : nullptr;
+  if (!by_rows) {
+    for (int s = 0; s < p.S; ++s) {
+      const size_t si = (size_t)i * p.S + s;
+      const bool fresh = ts->fresh[s] != 0;
+      int acc = -1;
+      if (fresh) {
+        const float* __restrict__ v = p.mail + si * (size_t)p.kd_pad;
+        double dot = 0.0, dd = 0.0, nv = 0.0;
 #pragma unroll 4
-      for (int q = tid; q < nvec; q += nt) {
-        const int e = q * V;
-        const TailVec<V> vv = tail_ldcg<V>(v + e);
-        const TailVec<V> D = tail_ld<V>(SD + e);
-        const TailVec<V> ww = tail_ld<V>(w + widx(e));
+        for (int q = tid; q < nvec; q += nt) {
+          const int e = q * V;
+          const TailVec<V> vv = tail_ldcg<V>(v + e);
+          const TailVec<V> D = tail_ld<V>(SD + e);
+          const TailVec<V> ww = tail_ld<V>(w + widx(e));
 #pragma unroll
-        for (int u = 0; u < V; ++u) {
-          const float df = ww.v[u] - vv.v[u];
-          dot += (double)D.v[u] * (double)df;
-          dd += (double)D.v[u] * (double)D.v[u];
-          nv += (double)vv.v[u] * (double)vv.v[u];
+          for (int u = 0; u < V; ++u) {
+            const float df = ww.v[u] - vv.v[u];
+            dot += (double)D.v[u] * (double)df;
+            dd += (double)D.v[u] * (double)D.v[u];
+            nv += (double)vv.v[u] * (double)vv.v[u];
+          }
+        }
+        block_sum3(dot, dd, nv, ts->red);
+        // Eq. 4 expanded: ||(w - eps D) - v||^2 < ||w - v||^2  <=>  2 <D, w - v> > eps ||D||^2
+        const bool delta = p.parzen ? (2.0 * dot > (double)eps * dd) : true;
+        acc = (nv > 0.0 && delta) ? 1 : 0;   // lambda * delta
+        m += acc;
+        if (acc) whole_bits |= 1u << s;
+      }
+      if (tid == 0) { ts->accept[s] = acc; p.accept_rec[si] = acc; }
+      __syncthreads();
+    }
+  } else {
+    // Section 4.4: a warp per centre row; for every buffer with a new message that carries the row, the
+    // row's own lambda and delta (fp64 sums over its d entries, fixed lane order)
+    if (tid < p.S) ts->accept[tid] = ts->fresh[tid] ? 0 : -1;          // becomes the number of accepted rows
+    __syncthreads();
+    unsigned* rowin = p.rowin + (size_t)i * p.k;
+    const int lane = tid & 31, wrp = tid >> 5, nw = nt >> 5;
+    for (int a = wrp; a < p.k; a += nw) {
+      unsigned bits = 0, inbits = 0;
+      for (int s = 0; s < p.S; ++s) {
+        if (!ts->fresh[s]) continue;
+        const size_t si = (size_t)i * p.S + s;
+        const int2 run = __ldcg(p.mail_rows + si);
+        if (!row_in_run(a, run.x, run.y, p.k)) continue;
+        inbits |= 1u << s;
+        const float* __restrict__ v = p.mail + si * (size_t)p.kd_pad + (size_t)a * d;
+        double dot = 0.0, dd = 0.0, nv = 0.0;
+        for (int j = lane; j < d; j += 32) {
+          const float vv = __ldcg(v + j), D = SD[a * d + j], ww = w[widx(a * d + j)];
+          const float df = ww - vv;
+          dot += (double)D * (double)df;
+          dd += (double)D * (double)D;
+          nv += (double)vv * (double)vv;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          dot += __shfl_xor_sync(0xffffffffu, dot, o);
+          dd += __shfl_xor_sync(0xffffffffu, dd, o);
+          nv += __shfl_xor_sync(0xffffffffu, nv, o);
+        }
+        const bool delta = p.parzen ? (2.0 * dot > (double)eps * dd) : true;
+        if (nv > 0.0 && delta) {
+          bits |= 1u << s;
+          if (lane == 0) atomicAdd(&ts->accept[s], 1);
         }
       }
-      block_sum3(dot, dd, nv, ts->red);
-      // Eq. 4 expanded: ||(w - eps D) - v||^2 < ||w - v||^2  <=>  2 <D, w - v> > eps ||D||^2
-      const bool delta = p.parzen ? (2.0 * dot > (double)eps * dd) : true;
-      acc = (nv > 0.0 && delta) ? 1 : 0;   // lambda * delta
-      m += acc;
+      if (lane == 0) { rowacc[a] = bits; rowin[a] = inbits; }
     }
-    if (tid == 0) { ts->accept[s] = acc; p.accept_rec[si] = acc; }
     __syncthreads();
+    for (int s = 0; s < p.S; ++s) m += (ts->accept[s] > 0);           // messages with at least one accepted row
+    if (tid < p.S) p.accept_rec[(size_t)i * p.S + tid] = ts->accept[tid];
   }
 
-  // Eq. 6: Dbar = w - (w + sum_s a_s v_s) / (1 + sum_s a_s) + D ;  w <- w - eps * Dbar
-  const float inv_m1 = 1.0f / (float)(1 + m);
+  // Eq. 6: Dbar = w - (w + sum_s a_s v_s) / (1 + sum_s a_s) + D ;  w <- w - eps * Dbar   (a_s per row in per-centre mode)
+  const float inv_m1_whole = 1.0f / (float)(1 + m);
 #pragma unroll 4
   for (int q = tid; q < nvec; q += nt) {
     const int e = q * V;
+    const unsigned bits = by_rows ? rowacc[e / d] : whole_bits;
+    const float inv_m1 = by_rows ? 1.0f / (float)(1 + __popc(bits)) : inv_m1_whole;
     TailVec<V> sumv;
 #pragma unroll
     for (int u = 0; u < V; ++u) sumv.v[u] = 0.f;
     for (int s = 0; s < p.S; ++s)
-      if (ts->accept[s] == 1) {
+      if (bits & (1u << s)) {
         const TailVec<V> vv = tail_ldcg<V>(p.mail + ((size_t)i * p.S + s) * (size_t)p.kd_pad + e);
 #pragma unroll
         for (int u = 0; u < V; ++u) sumv.v[u] += vv.v[u];

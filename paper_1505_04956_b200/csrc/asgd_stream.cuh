@@ -238,7 +238,6 @@ asgd_stream_kernel(const Params p, const long long steps) {
       __syncthreads();
     }
     const float* xs = reinterpret_cast<const float*>(tile + head);
-    const float* wblk = xs + (size_t)wid * STREAM_WARP_SAMPLES * D;      // this warp's 128 rows
 
     // ---- Eq. 8: scores of this thread's samples against every centre ----
     float2 xv[STREAM_SPT][D2];
@@ -418,6 +417,8 @@ asgd_stream_kernel(const Params p, const long long steps) {
         __syncthreads();                                 // the new w is complete
         n_sent = step_send_any<kDet>(p, i, t, w, D, ts);
       }
+      if (kDet && p.rows_m > 0)                            // per-row record of a step that looked at no message
+        for (int a = tid; a < p.k; a += STREAM_THREADS) p.rowin[(size_t)i * p.k + a] = 0;
       if (tid == 0) {
         if (kDet)
           for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;

@@ -121,7 +121,6 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   const int i = blockIdx.x;
   const int nkc = d / TC_KC;                                           // K chunks per tile
   const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_MH * TC_M - 1) / (TC_MH * TC_M);
-  const int dl = d / 32;                                               // dimensions per lane (multiple of 2)
   float* wglob = p.state + (size_t)i * p.kd_pad;
   float* gsum = p.gsum + (size_t)i * p.kd_pad;
   __nv_bfloat16* wbf = reinterpret_cast<__nv_bfloat16*>(p.wbf) + (size_t)i * k * d;
@@ -537,6 +536,8 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         __syncthreads();                                  // every centre's new w is in place
         n_sent = step_send_any<kDet>(p, i, t, wglob, d, ts);
       }
+      if (kDet && p.rows_m > 0)                            // per-row record of a step that looked at no message
+        for (int a = tid; a < p.k; a += TC_THREADS) p.rowin[(size_t)i * p.k + a] = 0;
       if (tid == 0) {
         if (kDet)
           for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;

@@ -32,7 +32,7 @@ class Pair:
     """The CUDA context and the oracle on identical inputs."""
 
     def __init__(self, wl, *, parzen=1, slots=None, shuffle=1, record_assign=1, dist_path=pkg.PATH_AUTO,
-                 X=None, w0=None, oracle=True, device="cuda"):
+                 X=None, w0=None, oracle=True, device="cuda", partial_rows=0):
         self.wl = wl
         if X is None:
             Xh, _ = inputs.make_samples(wl, device="cpu")
@@ -45,12 +45,14 @@ class Pair:
         self.S = S
         self.cfg = pkg.make_config(N=Xh.shape[0], d=wl.d, k=wl.k, W=wl.W, b=wl.b, eps=wl.eps,
                                    comm_interval=wl.comm_interval, fanout=wl.fanout, slots=S, parzen=parzen,
-                                   shuffle=shuffle, record_assign=record_assign, seed=wl.seed, dist_path=dist_path)
+                                   shuffle=shuffle, record_assign=record_assign, seed=wl.seed, dist_path=dist_path,
+                                   partial_rows=partial_rows)
         self.gpu = pkg.Asgd(self.cfg, self.X, self.w0)
         self.cpu = None
         if oracle:
             self.cpu = orc.Oracle(self.Xh, self.w0h, W=wl.W, b=wl.b, eps=wl.eps, comm_interval=wl.comm_interval,
-                                  fanout=wl.fanout, slots=S, parzen=parzen, shuffle=shuffle, seed=wl.seed)
+                                  fanout=wl.fanout, slots=S, parzen=parzen, shuffle=shuffle, seed=wl.seed,
+                                  partial_rows=partial_rows)
 
     def centre_tol(self):
         return CENTRE_TOL_BF16 if self.gpu.path_name() == "tcgen05-bf16" else CENTRE_TOL
