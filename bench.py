@@ -205,7 +205,7 @@ def main():
         wl = wl.scaled(comm_interval=args.comm_interval)
     # each rank owns an independent group of W workers on its own seeded shard (no cross-GPU exchange)
     wl_rank = wl.scaled(seed=dist.shard_seed(wl.seed, rank, world))
-    X, _ = inputs.make_samples(wl_rank, device=dev)
+    X, mu = inputs.make_samples(wl_rank, device=dev)
     w0 = inputs.initial_centres(wl_rank, X)
     cfg = pkg.make_config(N=wl.N, d=wl.d, k=wl.k, W=wl.W, b=wl.b, eps=wl.eps, comm_interval=wl.comm_interval,
                           fanout=wl.fanout, seed=wl_rank.seed, parzen=0 if args.no_parzen else 1,
@@ -237,6 +237,8 @@ def main():
     value = world * samples_per_pass * args.steps / (total_ms * 1e-3)
     E_final = ctx.eval(0)
     E_mean = ctx.eval(-1)
+    from paper_1505_04956_b200 import metrics
+    centre_err, _ = metrics.generator_centre_error(mu.cpu().numpy(), ctx.get_state(0).cpu().numpy())
     msgs = {"sent": 0, "received": 0, "accepted": 0, "overwritten": 0}
     for i in range(wl.W):
         st = ctx.get_stats(i)
@@ -263,6 +265,19 @@ def main():
                         "traffic": None, "peak_kind": "SMs x 128 fp32 lanes x 2 x max SM clock", "kernel": ctx.path_name(),
                         "launch_ms": launch_ms, "algorithmic_flops_per_launch": flops,
                         "hbm_GBs": achieved}
+    elif ctx.path_name() == "tcgen05-bf16":
+        # bound by the tensor pipe: the 2*k*d flops per sample of the -2 X W^T contraction against the measured
+        # sustained BF16 rate (the kernel is timed inside a long launch)
+        tpeak, tkind = 1400.0, "fallback (sustained)"
+        ppath = os.path.join(ROOT, "MEASURED_PEAKS.json")
+        if os.path.exists(ppath):
+            with open(ppath) as f:
+                tpeak, tkind = float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
+        flops = 2.0 * wl.k * wl.d * samples_per_pass
+        ach = flops / (launch_ms * 1e-3) / 1e12
+        roofline_alu = {"bound": "tensor", "achieved": ach, "peak": tpeak, "unit": "TFLOP/s", "frac": ach / tpeak,
+                        "traffic": None, "peak_kind": "of " + tkind, "kernel": ctx.path_name(), "launch_ms": launch_ms,
+                        "algorithmic_flops_per_launch": flops, "hbm_GBs": achieved}
     else:
         roofline_alu = None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -314,7 +329,7 @@ def main():
                        "steps_per_worker_per_bench_step": steps, "parallelism": "dp%d" % world,
                        "l2": "inputs larger than L2 (%.2f GB per pass)" % (bytes_per_launch / 1e9)},
             "roofline": roofline_alu or roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "quantization_error_worker0": E_final, "quantization_error_mean_state": E_mean, "messages": msgs, "messages_over_passes": args.warmup + args.steps,
+            "quantization_error_worker0": E_final, "quantization_error_mean_state": E_mean, "generator_centre_error_worker0": centre_err, "messages": msgs, "messages_over_passes": args.warmup + args.steps,
         }
         print(json.dumps(line), flush=True)
     dist.shutdown()

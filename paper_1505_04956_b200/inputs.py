@@ -52,13 +52,15 @@ class Workload:
         return dataclasses.replace(self, **kw)
 
 
-# The five workloads the library is measured and tested on.
+# The workloads the library is measured and tested on: five base shapes and the large-codebook shape
+# (k = 1000 prototypes of d = 128, the top of the codebook range of Section 5.2).
 WORKLOADS = {
     "tiny": Workload("tiny", 100_000, 10, 10, 4, 100, 0.05, 1000, 0, 10, 1, 0, "box:10", 1.0, "equal"),
     "stream": Workload("stream", 268_435_456, 10, 10, 592, 500, 0.01, 0, 1, 20, 1, 1, "box:10", 1.0, "equal"),
     "mid": Workload("mid", 16_777_216, 128, 100, 296, 1000, 0.01, 0, 2, 10, 2, 2, "normal:5", 1.0, "dirichlet"),
     "sweep": Workload("sweep", 67_108_864, 32, 64, 592, 256, 0.02, 0, 1, 10, 1, 3, "box:5", 0.5, "equal"),
     "dense": Workload("dense", 8_388_608, 256, 1024, 148, 4096, 0.005, 0, 1, 5, 1, 4, "normal:2", 1.0, "equal"),
+    "codebook": Workload("codebook", 8_388_608, 128, 1000, 148, 2048, 0.005, 0, 1, 5, 1, 5, "normal:3", 1.0, "equal"),
 }
 
 

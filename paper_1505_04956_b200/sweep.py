@@ -2,7 +2,8 @@
 
 For every point (W, c, Parzen window on/off, rows per message) of a grid it runs free-running passes of
 a workload through the library and prints one JSON line: samples/s of the last pass (CUDA events), the
-quantisation error E(w) of worker 0's state and of the mean state (Eq. 8), and the message counters
+quantisation error E(w) of worker 0's state and of the mean state (Eq. 8), the mean distance of worker 0's
+centres to the generator's centres under a greedy pairing (Section 5.4), and the message counters
 (sent, received, accepted = "good", overwritten) summed over the workers.  c = 0 is the silent mode
 (no communication at all), --no-parzen accepts every non-empty message.
 
@@ -25,13 +26,14 @@ def main():
 
     import torch
     import paper_1505_04956_b200 as pkg
-    from paper_1505_04956_b200 import inputs
+    from paper_1505_04956_b200 import inputs, metrics
 
     pkg.load()
     base = inputs.WORKLOADS[args.workload]
     if args.rows:
         base = base.scaled(N=args.rows)
-    X, _ = inputs.make_samples(base, device="cuda")
+    X, mu = inputs.make_samples(base, device="cuda")
+    mu = mu.cpu().numpy()
     w0 = inputs.initial_centres(base, X)
     ints = lambda text, default: [int(v) for v in text.split(",")] if text else [default]
     for W in ints(args.workers, base.W):
@@ -62,7 +64,9 @@ def main():
                         "workload": wl.name, "W": W, "comm_interval": c, "parzen": parzen, "partial_rows": rows,
                         "passes": args.passes, "steps_per_worker_per_pass": steps, "kernel": ctx.path_name(),
                         "ms_last_pass": ms, "samples_per_s": wl.W * steps * wl.b / (ms * 1e-3),
-                        "E_worker0": ctx.eval(0), "E_mean_state": ctx.eval(-1), "messages": msgs}), flush=True)
+                        "E_worker0": ctx.eval(0), "E_mean_state": ctx.eval(-1),
+                        "generator_centre_error_worker0": metrics.generator_centre_error(mu, ctx.get_state(0).cpu().numpy())[0],
+                        "messages": msgs}), flush=True)
                     ctx.destroy()
 
 

@@ -25,6 +25,7 @@ PARITY_WORKLOADS = {
     "mid": (scaled("mid", N=8 * 3000 + 5, W=8, comm_interval=2), 6),
     "sweep": (scaled("sweep", N=16 * 1024 + 3, W=16, comm_interval=1), 8),
     "dense": (scaled("dense", N=2 * 2048 + 1, W=2, b=1024, comm_interval=1), 3),
+    "codebook": (scaled("codebook", N=2 * 1536 + 7, W=2, b=512, comm_interval=1), 3),
 }
 
 

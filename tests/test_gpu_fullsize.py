@@ -1,4 +1,4 @@
-"""The five workloads at their full sizes, in the launch configuration bench.py times.
+"""The workloads at their full sizes, in the launch configuration bench.py times.
 
 The oracle cannot run a full pass of every workload in seconds, so it replays the first rounds: the rows
 those rounds touch are gathered (on the device, then copied) into a compact matrix in visiting order, on
@@ -16,12 +16,12 @@ from tests.gpu_util import CENTRE_TOL, CENTRE_TOL_BF16, decided
 
 pytestmark = pytest.mark.gpu
 
-REPLAY_ROUNDS = {"tiny": 40, "stream": 9, "mid": 2, "sweep": 3, "dense": 1}     # stream: the first 1 % of a pass
+REPLAY_ROUNDS = {"tiny": 40, "stream": 9, "mid": 2, "sweep": 3, "dense": 1, "codebook": 1}     # stream: the first 1 % of a pass
 
 
 def _setup(name, record_assign=1):
     wl = inputs.WORKLOADS[name]
-    need = wl.N * wl.d * 4 * (1.6 if name == "dense" else 1.1) + (2 << 30)
+    need = wl.N * wl.d * 4 * (1.6 if name in ("dense", "codebook") else 1.1) + (2 << 30)
     if torch.cuda.mem_get_info()[0] < need:
         pytest.skip("not enough free device memory for the full %s workload" % name)
     X, _ = inputs.make_samples(wl, device="cuda")
