@@ -26,9 +26,11 @@ enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2, P_TC_BF16 = 3 };
 // (d, k) shapes the streaming path is compiled for
 #define ASGD_STREAM_SHAPES(X) X(10, 10) X(16, 16) X(4, 5) X(2, 3)
 
-// (d, padded k, warps along samples, warps along centres, blocks per SM) the tiled path is compiled for;
-// the first shape with the same d and enough centres is taken
-#define ASGD_TILED_SHAPES(X) X(32, 64, 4, 2, 2) X(128, 128, 4, 4, 1)
+// (d, padded k, warps along samples, warps along centres, blocks per SM) the tiled path is compiled for.
+// Among the shapes with the same d and enough centres the one that keeps the most threads busy for the given
+// number of workers is taken (small blocks when there are enough workers to fill the GPU with them: a block that
+// serves one worker keeps its state on chip between steps); ties go to the later entry.
+#define ASGD_TILED_SHAPES(X) X(32, 64, 4, 2, 2) X(32, 64, 2, 2, 4) X(128, 128, 4, 4, 1)
 
 struct Layout {
   size_t state, mail, seq, seen, arb_win, arb_cnt, mail_rows, rowacc, rowin, stats, perm, status, assign_rec, accept_rec, gsum,
@@ -106,6 +108,7 @@ struct asgd_ctx {
   int path;
   int state_on_chip;
   int grid;               // blocks of the worker kernel (tiled path: a block may serve several workers)
+  int tiled_shape;        // index into ASGD_TILED_SHAPES of the shape in use
   size_t smem_bytes;
   long long t_host;       // steps every worker has done (uniform across workers)
   long long launches;
@@ -154,7 +157,7 @@ void stream_launch(asgd_ctx* c, bool det, long long steps) {
 }
 
 template <int D, int KP, int WS, int WK, int MINB>
-int tiled_prepare(asgd_ctx* c) {
+int tiled_prepare(asgd_ctx* c, long long* busy_threads) {
   c->smem_bytes = tiled_smem_bytes<D, KP, WS, WK>(c->cfg.k);
   CU(c, cudaFuncSetAttribute(asgd_tiled_kernel<D, KP, WS, WK, MINB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
   CU(c, cudaFuncSetAttribute(asgd_tiled_kernel<D, KP, WS, WK, MINB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
@@ -165,6 +168,7 @@ int tiled_prepare(asgd_ctx* c) {
   const int V = (c->cfg.W + resident - 1) / resident;          // workers per block, served in turn
   if (V > TILED_MAX_V) return ASGD_EUNSUPPORTED;
   c->grid = (c->cfg.W + V - 1) / V;
+  *busy_threads = (long long)(c->grid < resident ? c->grid : resident) * (32 * WS * WK);
   return ASGD_OK;
 }
 template <int D, int KP, int WS, int WK, int MINB>
@@ -241,8 +245,8 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
         asgd_tc_kernel<false><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapX, c->mapW);
       break;
     case P_TILED: {
-      bool done = false;
-#define X(D_, KP_, WS_, WK_, MB_) if (!done && p.d == D_ && p.k <= KP_) { tiled_launch<D_, KP_, WS_, WK_, MB_>(c, det, steps); done = true; }
+      int idx = 0;
+#define X(D_, KP_, WS_, WK_, MB_) if (idx++ == c->tiled_shape) tiled_launch<D_, KP_, WS_, WK_, MB_>(c, det, steps);
       ASGD_TILED_SHAPES(X)
 #undef X
       break;
@@ -287,14 +291,28 @@ int resolve_path(asgd_ctx* c) {
 #undef X
   }
   if (cfg.dist_path == ASGD_PATH_AUTO || cfg.dist_path == ASGD_PATH_FP32) {
+    int idx = 0, best = -1;
+    long long best_busy = -1;
 #define X(D_, KP_, WS_, WK_, MB_)                                                                  \
   if (cfg.d == D_ && cfg.k <= KP_ && tiled_smem_bytes<D_, KP_, WS_, WK_>(cfg.k) <= kMaxDynSmem) { \
-    c->path = P_TILED;                                                                             \
-    c->state_on_chip = 0;                                                                          \
-    return tiled_prepare<D_, KP_, WS_, WK_, MB_>(c);                                               \
-  }
+    long long busy = 0;                                                                            \
+    if (tiled_prepare<D_, KP_, WS_, WK_, MB_>(c, &busy) == ASGD_OK && busy >= best_busy) { best = idx; best_busy = busy; } \
+  }                                                                                                \
+  ++idx;
     ASGD_TILED_SHAPES(X)
 #undef X
+    if (best >= 0) {
+      idx = 0;
+      long long busy = 0;
+      int rc = ASGD_EUNSUPPORTED;
+#define X(D_, KP_, WS_, WK_, MB_) if (idx++ == best) rc = tiled_prepare<D_, KP_, WS_, WK_, MB_>(c, &busy);
+      ASGD_TILED_SHAPES(X)
+#undef X
+      c->path = P_TILED;
+      c->state_on_chip = 0;
+      c->tiled_shape = best;
+      return rc;
+    }
   }
   c->path = P_GENERIC;
   const int kd_pad = c->p.kd_pad;

@@ -134,34 +134,40 @@ asgd_tiled_kernel(const Params p, const long long steps) {
 
   int abort = 0;
   long long g = 0;
+  bool have_state = false;                        // shared memory holds the -2w rows and norms of the worker about to step
   for (long long st = 0; st < steps && !abort; ++st) {
     for (int v = 0; v < nv && !abort; ++v) {
       const int i = (int)blockIdx.x + v * G;
       const unsigned long long t = tbase[v] + (unsigned long long)st;
       float* wglob = p.state + (size_t)i * p.kd_pad;
 
-      // ---- the worker's state: -2w rows, ||w_a||^2, empty sums ----
-      for (int e = tid; e < KP * (D / 4); e += THREADS) {
-        const int a = e / (D / 4), j4 = e % (D / 4);
-        float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (a < k) {
-          v4 = *reinterpret_cast<const float4*>(wglob + (size_t)a * D + 4 * j4);
-          v4.x *= -2.f; v4.y *= -2.f; v4.z *= -2.f; v4.w *= -2.f;
+      // ---- the worker's state: -2w rows, ||w_a||^2 (kept from the last step when this block serves one worker
+      //      and that step took the fused update), empty sums ----
+      if (!have_state) {
+        for (int e = tid; e < KP * (D / 4); e += THREADS) {
+          const int a = e / (D / 4), j4 = e % (D / 4);
+          float4 v4 = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (a < k) {
+            v4 = *reinterpret_cast<const float4*>(wglob + (size_t)a * D + 4 * j4);
+            v4.x *= -2.f; v4.y *= -2.f; v4.z *= -2.f; v4.w *= -2.f;
+          }
+          *reinterpret_cast<float4*>(wR + (size_t)a * WST + 4 * j4) = v4;
         }
-        *reinterpret_cast<float4*>(wR + (size_t)a * WST + 4 * j4) = v4;
       }
       for (int e = tid; e < k * D; e += THREADS) S[e] = 0.f;
       for (int e = tid; e < KP; e += THREADS) cnt[e] = 0;
       __syncthreads();
-      for (int a = wid; a < KP; a += WARPS) {
-        float s = 0.f;
+      if (!have_state) {
+        for (int a = wid; a < KP; a += WARPS) {
+          float s = 0.f;
 #pragma unroll
-        for (int q = 0; q < DR; ++q) { const float u = wR[(size_t)a * WST + lane + 32 * q]; s = fmaf(u, u, s); }
+          for (int q = 0; q < DR; ++q) { const float u = wR[(size_t)a * WST + lane + 32 * q]; s = fmaf(u, u, s); }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if (lane == 0) cn[a] = (a < k) ? 0.25f * s : INF;
+          for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+          if (lane == 0) cn[a] = (a < k) ? 0.25f * s : INF;
+        }
+        __syncthreads();
       }
-      __syncthreads();
       if (wid == 0) {
         float m = 0.f;
         for (int a = lane; a < k; a += 32) m = fmaxf(m, cn[a]);
@@ -169,6 +175,9 @@ asgd_tiled_kernel(const Params p, const long long steps) {
         for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
         if (lane == 0) misc[0] = m;
       }
+      // a look at the receive buffers' sequence numbers (used after the last tile)
+      int news = 0;
+      if (tid < p.S) news = ld_relaxed_gpu(p.seq + (size_t)i * p.S + tid) != p.seen[(size_t)i * p.S + tid];
 
       for (int tl = 0; tl < tiles; ++tl, ++g) {
         const int slot = (int)(g & 1);
@@ -372,15 +381,59 @@ asgd_tiled_kernel(const Params p, const long long steps) {
       }
       if (abort) break;
 
-      // the tail works on the state in shared memory: turn the -2w rows back into w (exact)
-      for (int e = tid; e < k * (D / 4); e += THREADS) {
-        float4* q4 = reinterpret_cast<float4*>(wR + (size_t)(e / (D / 4)) * WST + 4 * (e % (D / 4)));
-        float4 u = *q4;
-        u.x *= -0.5f; u.y *= -0.5f; u.z *= -0.5f; u.w *= -0.5f;
-        *q4 = u;
+      if (__syncthreads_or(news)) {
+        // a message is waiting: the general tail works on the state in shared memory; turn the -2w rows back into w (exact)
+        for (int e = tid; e < k * (D / 4); e += THREADS) {
+          float4* q4 = reinterpret_cast<float4*>(wR + (size_t)(e / (D / 4)) * WST + 4 * (e % (D / 4)));
+          float4 u = *q4;
+          u.x *= -0.5f; u.y *= -0.5f; u.z *= -0.5f; u.w *= -0.5f;
+          *q4 = u;
+        }
+        __syncthreads();
+        step_tail<kDet>(p, i, t, wR, WST, S, cnt, wglob, ts);
+        have_state = false;
+      } else {
+        // common case: plain local step  w <- w - eps (n_a w - S) / b  on the -2w rows, new state to HBM, new ||w_a||^2
+        constexpr int RV = D / 4;                            // 128-bit pieces per centre row (8 or 32: a power of two <= 32)
+        const float inv_b = 1.0f / (float)b;
+        const int pieces = k * RV;
+        for (int e0 = 0; e0 < pieces; e0 += THREADS) {       // the same trip count for every thread (shuffles inside)
+          const int e = e0 + tid;
+          const bool on = e < pieces;
+          const int a = on ? e / RV : 0, j4 = e % RV;
+          float sq = 0.f;
+          if (on) {
+            float4* q4 = reinterpret_cast<float4*>(wR + (size_t)a * WST + 4 * j4);
+            const float4 m2 = *q4;
+            const float4 sm = *reinterpret_cast<const float4*>(S + (size_t)a * D + 4 * j4);
+            const float fn = (float)cnt[a];
+            float4 w4 = make_float4(-0.5f * m2.x, -0.5f * m2.y, -0.5f * m2.z, -0.5f * m2.w);
+            w4.x -= p.eps * ((fn * w4.x - sm.x) * inv_b); w4.y -= p.eps * ((fn * w4.y - sm.y) * inv_b);
+            w4.z -= p.eps * ((fn * w4.z - sm.z) * inv_b); w4.w -= p.eps * ((fn * w4.w - sm.w) * inv_b);
+            *reinterpret_cast<float4*>(wglob + (size_t)a * D + 4 * j4) = w4;
+            *q4 = make_float4(-2.f * w4.x, -2.f * w4.y, -2.f * w4.z, -2.f * w4.w);
+            sq = fmaf(w4.x, w4.x, fmaf(w4.y, w4.y, fmaf(w4.z, w4.z, w4.w * w4.w)));
+          }
+#pragma unroll
+          for (int o = 1; o < RV; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+          if (on && j4 == 0) cn[a] = sq;
+        }
+        unsigned long long n_sent = 0;
+        if (p.c > 0 && p.f > 0 && p.W > 1 && (t + 1) % (unsigned long long)p.c == 0) {
+          __syncthreads();                                   // the new state is complete in HBM for this block's threads
+          n_sent = step_send_any<kDet>(p, i, t, wglob, D, ts);
+        }
+        if (kDet && p.rows_m > 0)
+          for (int a = tid; a < p.k; a += THREADS) p.rowin[(size_t)i * p.k + a] = 0;
+        if (tid == 0) {
+          if (kDet)
+            for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
+          unsigned long long* st_ = p.stats + (size_t)i * ST_STRIDE;
+          st_[ST_STEPS] = t + 1;
+          if (n_sent) atomicAdd(st_ + ST_SENT, n_sent);
+        }
+        have_state = (nv == 1);                              // the -2w rows and norms in shared memory are this worker's next state
       }
-      __syncthreads();
-      step_tail<kDet>(p, i, t, wR, WST, S, cnt, wglob, ts);
       __syncthreads();
     }
   }

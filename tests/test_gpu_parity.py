@@ -137,6 +137,7 @@ EDGE_CASES = {
     # shapes of the register-tiled kernel: padded centres, ragged last tile, several workers per block
     "tiled_32_k37_ragged_tile": dict(N=5 * 100 * 3 + 1, d=32, k=37, W=5, b=100, comm_interval=2, fanout=2),
     "tiled_32_many_workers": dict(N=700 * 12, d=32, k=8, W=700, b=4, comm_interval=1, fanout=1),
+    "tiled_32_small_blocks_one_worker_each": dict(N=592 * 70 * 2, d=32, k=64, W=592, b=70, comm_interval=2, fanout=1),
     "tiled_128_k128": dict(N=3 * 200 * 2, d=128, k=128, W=3, b=200, comm_interval=1, fanout=1),
     "tiled_128_k5_tiny_batch": dict(N=4 * 7 * 3, d=128, k=5, W=4, b=7, comm_interval=1, fanout=3),
     # shapes of the tensor-core kernel: a centre block that is not full, one K chunk, a ragged last sample tile
