@@ -198,7 +198,7 @@ bool encode_bf16_map(CUtensorMap* map, const void* base, unsigned long long rows
 
 // Tensor-core path set-up: bf16 copy of X (unless the caller brought one), max ||x||^2, tensor maps.
 // max_i ||x_i||^2 into Params::xmax2 (one pass over the samples at initialisation): the rounding bounds of the
-// streaming and tensor-core paths use it.
+// streaming, tiled and tensor-core paths use it.
 int compute_xmax2(asgd_ctx* c) {
   Params& p = c->p;
   unsigned* xm = (unsigned*)(c->ws + c->L.xmax);
@@ -406,7 +406,7 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   if (c->path == P_TC_BF16) {
     rc = tc_prepare(c);
     if (rc != ASGD_OK) { delete c; return rc; }
-  } else if (c->path == P_STREAM) {
+  } else if (c->path == P_STREAM || c->path == P_TILED) {
     rc = compute_xmax2(c);
     if (rc != ASGD_OK) { delete c; return rc; }
   }

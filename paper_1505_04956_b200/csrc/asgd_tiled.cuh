@@ -44,7 +44,7 @@ struct TiledShape {
 template <int D, int KP, int WS, int WK>
 struct TiledSmem {
   using T = TiledShape<D, KP, WS, WK>;
-  size_t wR, cn, S, cnt, xt, best, x2, red, flagged, tbase, bars, misc, tail, total;
+  size_t wR, cn, S, cnt, xt, best, red, flagged, tbase, bars, misc, tail, total;
   __host__ __device__ explicit TiledSmem(int k) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) / 16 * 16; return o; };
@@ -54,7 +54,6 @@ struct TiledSmem {
     cnt = take((size_t)KP * 4);
     xt = take((size_t)2 * 4 * T::QS * 4);
     best = take((size_t)T::TS * 4);
-    x2 = take((size_t)T::TS * 4);
     red = take((size_t)WK * T::TS * 8);
     flagged = take((size_t)(T::TS + 4) * 4);
     tbase = take((size_t)TILED_MAX_V * 8);
@@ -81,7 +80,6 @@ asgd_tiled_kernel(const Params p, const long long steps) {
   int* cnt = reinterpret_cast<int*>(smem_raw + map.cnt);            // [KP]
   float* xt = reinterpret_cast<float*>(smem_raw + map.xt);          // [2][4 quarters][QR][XS] (+4 floats per quarter)
   int* best = reinterpret_cast<int*>(smem_raw + map.best);          // [TS]
-  float* x2s = reinterpret_cast<float*>(smem_raw + map.x2);         // [TS]
   float2* red = reinterpret_cast<float2*>(smem_raw + map.red);      // [WK][TS] (minimum, runner-up)
   int* flagged = reinterpret_cast<int*>(smem_raw + map.flagged);    // [0] count, [1..] tile rows to decide again
   unsigned long long* tbase = reinterpret_cast<unsigned long long*>(smem_raw + map.tbase);
@@ -241,21 +239,7 @@ asgd_tiled_kernel(const Params p, const long long steps) {
           fence_proxy_async_smem();
           issue_next();
         }
-        // ---- ||x||^2 of every tile row: 8 threads per row, 4 dimensions at a time ----
-        for (int r = tid >> 3; r < TS; r += THREADS / 8) {
-          const int h = tid & 7;
-          float xx = 0.f;
-#pragma unroll
-          for (int q = 0; q < D / 32; ++q) {
-            const float4 u = *reinterpret_cast<const float4*>(xrowp(r) + 4 * h + 32 * q);
-            xx = fmaf(u.x, u.x, xx); xx = fmaf(u.y, u.y, xx); xx = fmaf(u.z, u.z, xx); xx = fmaf(u.w, u.w, xx);
-          }
-          xx += __shfl_xor_sync(0xffffffffu, xx, 1);
-          xx += __shfl_xor_sync(0xffffffffu, xx, 2);
-          xx += __shfl_xor_sync(0xffffffffu, xx, 4);
-          if (h == 0) x2s[r] = xx;
-        }
-        __syncthreads();                                         // (1) red, x2s complete
+        __syncthreads();                                         // (1) red complete
 
         // ---- one thread per tile row: merge over the centre blocks, decide or flag ----
         if (tid < TS) {
@@ -270,7 +254,15 @@ asgd_tiled_kernel(const Params p, const long long steps) {
               if (r.x < s1) { s1 = r.x; qwin = q; }             // equal packed scores of two blocks: second look below
             }
             bst = qwin * 32 + (int)(__float_as_uint(s1) & T::INDEX_MASK);
-            if (k > 1 && (s2 - s1) <= tau_scale * (misc[0] + x2s[tid])) flagged[1 + atomicAdd(flagged, 1)] = tid;
+            if (k > 1 && (s2 - s1) <= tau_scale * (misc[0] + p.xmax2)) {       // cheap test with the bound on ||x||^2 over X first
+              const float* xr = xrowp(tid);
+              float xx = 0.f;
+              for (int j = 0; j < D; j += 4) {
+                const float4 u = *reinterpret_cast<const float4*>(xr + j);
+                xx = fmaf(u.x, u.x, xx); xx = fmaf(u.y, u.y, xx); xx = fmaf(u.z, u.z, xx); xx = fmaf(u.w, u.w, xx);
+              }
+              if ((s2 - s1) <= tau_scale * (misc[0] + xx)) flagged[1 + atomicAdd(flagged, 1)] = tid;
+            }
           }
           best[tid] = bst;
         }
