@@ -13,9 +13,9 @@
 //
 // Per-centre sums (Eq. 9): each warp files its 128 rows under the centres they chose (rank inside a
 // 32-row block from a match, so a warp's list of a centre is in row order; entries are byte offsets
-// into the tile, the unused tail of a list points at a row of zeros kept behind the tile).  Then one
-// thread per (half of the warps, centre, dimension pair) adds the listed rows from the shared-memory
-// tile.  Every sum has a fixed order, so a step is reproducible.  The plain local step needs three
+// into the tile, the unused tail of a list points at a row of zeros kept behind the tile).  Then lane
+// (centre, dimension pair) of the same warp adds the listed rows from the shared-memory
+// tile.  Every sum has a fixed order, so a step is reproducible.  The plain local step needs two
 // block-wide barriers.
 #pragma once
 
@@ -29,7 +29,7 @@ constexpr int STREAM_STAGES = 2;
 constexpr int STREAM_SPT = 4;                          // samples per thread = 32-row blocks per warp
 constexpr int STREAM_MAX_B = STREAM_THREADS * STREAM_SPT;
 constexpr int STREAM_WARP_SAMPLES = 32 * STREAM_SPT;
-constexpr int STREAM_PARTS = 2;                        // partial sums per centre: one per half of the warps
+constexpr int STREAM_PARTS = STREAM_WARPS;              // partial sums per centre: one per warp
 constexpr int STREAM_SEG = STREAM_WARP_SAMPLES;        // capacity of a warp's list of one centre
 constexpr unsigned STREAM_WAIT_LIMIT = 1u << 22;       // bounded mbarrier wait (iterations of try_wait)
 
@@ -56,6 +56,12 @@ __device__ inline bool mbar_wait_bounded(unsigned long long* bar, unsigned parit
 __device__ inline void bulk_g2s(void* dst, const void* src, unsigned bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// three-input minimum (one instruction on sm_100)
+__device__ inline float fmin3(float a, float b, float c) {
+  float r;
+  asm("min.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
 }
 __device__ inline void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ inline unsigned ld_relaxed_gpu(const unsigned* p) {
@@ -252,8 +258,8 @@ asgd_stream_kernel(const Params p, const long long steps) {
 #pragma unroll
     for (int q = 0; q < STREAM_SPT; ++q) { s1[q] = __int_as_float(0x7f800000); s2[q] = __int_as_float(0x7f800000); }
     float wmax2 = 0.f;
-#pragma unroll 2
-    for (int a = 0; a < K; ++a) {
+    // packed score of centre a for each of the thread's samples
+    auto scores_of = [&](int a, float (&sp)[STREAM_SPT]) {
       float2 wr[DP / 2];
 #pragma unroll
       for (int j4 = 0; j4 < DP / 4; ++j4) {
@@ -269,9 +275,29 @@ asgd_stream_kernel(const Params p, const long long steps) {
 #pragma unroll
         for (int jp = 0; jp < D2; ++jp) acc = __ffma2_rn(xv[q][jp], wr[jp], acc);
         const float sc = acc.x + acc.y;
-        const float sp = __uint_as_float((__float_as_uint(sc) & ~L::INDEX_MASK) | (unsigned)a);
-        s2[q] = fmaxf(s1[q], fminf(s2[q], sp));
-        s1[q] = fminf(s1[q], sp);
+        sp[q] = __uint_as_float((__float_as_uint(sc) & ~L::INDEX_MASK) | (unsigned)a);
+      }
+    };
+    // two centres at a time: with lo <= hi the new pair is  s1' = min(s1, lo),  s2' = min(max(s1, lo), s2, hi)
+#pragma unroll 1
+    for (int a = 0; a + 1 < K; a += 2) {
+      float pa[STREAM_SPT], pb[STREAM_SPT];
+      scores_of(a, pa);
+      scores_of(a + 1, pb);
+#pragma unroll
+      for (int q = 0; q < STREAM_SPT; ++q) {
+        const float lo = fminf(pa[q], pb[q]), hi = fmaxf(pa[q], pb[q]);
+        s2[q] = fmin3(fmaxf(s1[q], lo), s2[q], hi);
+        s1[q] = fminf(s1[q], lo);
+      }
+    }
+    if (K & 1) {
+      float pa[STREAM_SPT];
+      scores_of(K - 1, pa);
+#pragma unroll
+      for (int q = 0; q < STREAM_SPT; ++q) {
+        s2[q] = fmaxf(s1[q], fminf(s2[q], pa[q]));
+        s1[q] = fminf(s1[q], pa[q]);
       }
     }
 
@@ -324,36 +350,31 @@ asgd_stream_kernel(const Params p, const long long steps) {
     }
     if (tid < p.S && my_seq != seen_s[tid]) flags[0] = 1;
 
-    // ---- barrier B1: every warp's lists are complete ----
-    if (__syncthreads_or(abort)) { abort = 1; break; }
+    __syncwarp();
 
-    // ---- Eq. 9: thread (half, centre, dimension pair) adds the rows listed by its half of the warps ----
+    // ---- Eq. 9: lane (centre, dimension pair) adds the rows its own warp listed under the centre ----
     {
-      constexpr int ITEMS = STREAM_PARTS * K * D2, WPP = STREAM_WARPS / STREAM_PARTS;
-      for (int item = tid; item < ITEMS; item += STREAM_THREADS) {
-        const int h = item / (K * D2), rem = item - h * (K * D2), a = rem / D2, jp = rem - a * D2;
+      constexpr int ITEMS = K * D2;
+      for (int item = lane; item < ITEMS; item += 32) {
+        const int a = item / D2, jp = item - a * D2;
         const unsigned char* xb = reinterpret_cast<const unsigned char*>(xs) + jp * 8;
         auto row = [&](unsigned off) { return *reinterpret_cast<const float2*>(xb + off); };
         float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int ww = 0; ww < WPP; ++ww) {
-          const int wsrc = h * WPP + ww;
-          const int n = Cw[wsrc * CWS + a];
-          const uint4* seg = reinterpret_cast<const uint4*>(lists + (size_t)(wsrc * K + a) * STREAM_SEG);
-          for (int e0 = 0; e0 < n; e0 += 8) {                              // a list's tail points at the row of zeros
-            const uint4 pk = seg[e0 >> 3];
-            acc0 = __fadd2_rn(acc0, row(pk.x & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.x >> 16));
-            acc0 = __fadd2_rn(acc0, row(pk.y & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.y >> 16));
-            acc0 = __fadd2_rn(acc0, row(pk.z & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.z >> 16));
-            acc0 = __fadd2_rn(acc0, row(pk.w & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.w >> 16));
-          }
+        const int n = myCw[a];
+        const uint4* seg = reinterpret_cast<const uint4*>(myLists + (size_t)a * STREAM_SEG);
+        for (int e0 = 0; e0 < n; e0 += 8) {                                // a list's tail points at the row of zeros
+          const uint4 pk = seg[e0 >> 3];
+          acc0 = __fadd2_rn(acc0, row(pk.x & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.x >> 16));
+          acc0 = __fadd2_rn(acc0, row(pk.y & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.y >> 16));
+          acc0 = __fadd2_rn(acc0, row(pk.z & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.z >> 16));
+          acc0 = __fadd2_rn(acc0, row(pk.w & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.w >> 16));
         }
-        *reinterpret_cast<float2*>(Sw + (size_t)(h * K + a) * D + 2 * jp) = __fadd2_rn(acc0, acc1);
+        *reinterpret_cast<float2*>(Sw + (size_t)(wid * K + a) * D + 2 * jp) = __fadd2_rn(acc0, acc1);
       }
     }
 
-    // ---- barrier B2: partial sums complete, the ring slot is free again ----
-    __syncthreads();
+    // ---- barrier B: partial sums and list lengths complete, the ring slot is free again ----
+    if (__syncthreads_or(abort)) { abort = 1; break; }
 
     const bool put_now = (to_put == 1);
     if (flags[0] != 0) {
