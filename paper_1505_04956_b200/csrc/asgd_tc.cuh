@@ -354,18 +354,36 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       };
       auto settle_finish = [&](const float4 (&xv)[TC_MAX_D / 32], const float4 (&a1)[TC_MAX_D / 32], const float4 (&a2)[TC_MAX_D / 32],
                                int r, int i1, int i2) {
-        double d1 = 0.0, d2 = 0.0;
+        // direct differences in fp32 first: each squared distance is off by at most (d + 2) u relative, so a gap
+        // above (4 d + 16) u of the larger one decides; only rows closer than that are summed again in fp64
+        float f1 = 0.f, f2 = 0.f;
 #pragma unroll
         for (int q = 0; q < TC_MAX_D / 32; ++q) {
-          double u;
-          u = (double)xv[q].x - (double)a1[q].x; d1 = fma(u, u, d1); u = (double)xv[q].y - (double)a1[q].y; d1 = fma(u, u, d1);
-          u = (double)xv[q].z - (double)a1[q].z; d1 = fma(u, u, d1); u = (double)xv[q].w - (double)a1[q].w; d1 = fma(u, u, d1);
-          u = (double)xv[q].x - (double)a2[q].x; d2 = fma(u, u, d2); u = (double)xv[q].y - (double)a2[q].y; d2 = fma(u, u, d2);
-          u = (double)xv[q].z - (double)a2[q].z; d2 = fma(u, u, d2); u = (double)xv[q].w - (double)a2[q].w; d2 = fma(u, u, d2);
+          float u;
+          u = xv[q].x - a1[q].x; f1 = fmaf(u, u, f1); u = xv[q].y - a1[q].y; f1 = fmaf(u, u, f1);
+          u = xv[q].z - a1[q].z; f1 = fmaf(u, u, f1); u = xv[q].w - a1[q].w; f1 = fmaf(u, u, f1);
+          u = xv[q].x - a2[q].x; f2 = fmaf(u, u, f2); u = xv[q].y - a2[q].y; f2 = fmaf(u, u, f2);
+          u = xv[q].z - a2[q].z; f2 = fmaf(u, u, f2); u = xv[q].w - a2[q].w; f2 = fmaf(u, u, f2);
         }
 #pragma unroll
-        for (int o = 1; o < 8; o <<= 1) { d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); }
-        if (r >= 0 && l8 == 0 && (d2 < d1 || (d2 == d1 && i2 < i1))) best[r] = (unsigned short)i2;
+        for (int o = 1; o < 8; o <<= 1) { f1 += __shfl_xor_sync(0xffffffffu, f1, o); f2 += __shfl_xor_sync(0xffffffffu, f2, o); }
+        bool second = f2 < f1;
+        const bool close = fabsf(f1 - f2) <= (float)(4 * TC_MAX_D + 16) * 5.9604645e-8f * fmaxf(f1, f2);
+        if (__any_sync(0xffffffffu, close && r >= 0)) {       // warp-uniform: the shuffles below need every lane
+          double d1 = 0.0, d2 = 0.0;
+#pragma unroll
+          for (int q = 0; q < TC_MAX_D / 32; ++q) {
+            double u;
+            u = (double)xv[q].x - (double)a1[q].x; d1 = fma(u, u, d1); u = (double)xv[q].y - (double)a1[q].y; d1 = fma(u, u, d1);
+            u = (double)xv[q].z - (double)a1[q].z; d1 = fma(u, u, d1); u = (double)xv[q].w - (double)a1[q].w; d1 = fma(u, u, d1);
+            u = (double)xv[q].x - (double)a2[q].x; d2 = fma(u, u, d2); u = (double)xv[q].y - (double)a2[q].y; d2 = fma(u, u, d2);
+            u = (double)xv[q].z - (double)a2[q].z; d2 = fma(u, u, d2); u = (double)xv[q].w - (double)a2[q].w; d2 = fma(u, u, d2);
+          }
+#pragma unroll
+          for (int o = 1; o < 8; o <<= 1) { d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); }
+          if (close) second = (d2 < d1 || (d2 == d1 && i2 < i1));
+        }
+        if (r >= 0 && l8 == 0 && second) best[r] = (unsigned short)i2;
       };
       const int groups = TC_WARPS * 4;
       for (int fb = wid * 4; fb < nflag; fb += groups) {       // the same trip count for all lanes of a warp (shuffles inside)
