@@ -5,7 +5,7 @@
 // One worker = one thread block = one SM.  Warp roles while the scores are computed:
 //   warp 0   one lane issues the TMA loads: a 128-row sample tile in 128-byte-swizzled K-chunks of 64,
 //            resident while all centre blocks pass, and 256-centre blocks of bf16(-2w) through a
-//            4-slot ring (they come from L2: all workers' bf16 states fit there);
+//            4-slot ring of K-chunks (they come from L2: all workers' bf16 states fit there);
 //   warp 1   allocates tensor memory; one lane issues tcgen05.mma (128 x 256 x 16 per instruction)
 //            into one of two 256-column accumulator stages and commits to mbarriers;
 //   warps 4-7  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread), add
@@ -29,7 +29,8 @@ constexpr int TC_WARPS = TC_THREADS / 32;
 constexpr int TC_M = 128, TC_N = 256, TC_KC = 64;        // one MMA's output tile; K chunk = 64 bf16 = one swizzled 128-byte row
 constexpr int TC_MH = 1;                                  // 128-row parts of the resident sample tile (TC_MH * TC_N <= 256 accumulator columns per stage)
 constexpr int TC_A_STAGES = 4;                            // K chunks of the resident sample tile (d <= 256)
-constexpr int TC_B_STAGES = 4;                            // ring of centre-block chunks
+constexpr int TC_B_STAGES = 4;                            // ring slots for the centre blocks
+constexpr int TC_BG = 1;                                  // K chunks per ring slot (one wait and one commit per slot; 2 x 2 was no faster than 4 x 1)
 constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB per part
 constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;       // 32 KB
 constexpr int TC_MAX_K = 1024, TC_MAX_D = 256, TC_MAX_B = 8192;
@@ -41,7 +42,7 @@ struct TcSmem {
     size_t off = 0;
     auto take = [&](size_t bytes, size_t align) { off = (off + align - 1) / align * align; size_t o = off; off += bytes; return o; };
     A = take((size_t)TC_A_STAGES * TC_MH * TC_A_STAGE_BYTES, 1024);   // [K chunk][part]
-    B = take((size_t)TC_B_STAGES * TC_B_CHUNK_BYTES, 1024);
+    B = take((size_t)TC_B_STAGES * TC_BG * TC_B_CHUNK_BYTES, 1024);
     cn = take((size_t)((k + TC_N - 1) / TC_N) * TC_N * 4, 16);
     cnt = take((size_t)k * 4, 16);
     best = take((size_t)b * 2, 16);
@@ -120,6 +121,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int i = blockIdx.x;
   const int nkc = d / TC_KC;                                           // K chunks per tile
+  const int ngr = (nkc + TC_BG - 1) / TC_BG;                           // ring slots a centre block passes through
   const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_MH * TC_M - 1) / (TC_MH * TC_M);
   float* wglob = p.state + (size_t)i * p.kd_pad;
   float* gsum = p.gsum + (size_t)i * p.kd_pad;
@@ -170,7 +172,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
 
     // ================= scores: -2 X W^T + ||w||^2, two best per sample =================
     // A sample tile (TC_MH parts of 128 rows, nkc K-chunks each) stays in shared memory while the centre blocks stream
-    // past it through a 4-slot ring (the bf16 states of all workers fit in L2; the samples are read from HBM once).
+    // past it through the ring (the bf16 states of all workers fit in L2; the samples are read from HBM once).
     if (wid == 0) {
       if (lane == 0) {
         unsigned um = it_m, ibc = it_bc;
@@ -186,12 +188,14 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
                           (int)(row0 + (long long)(m * TC_MH + h) * TC_M), bars + TCB_AFULL + kc);
           }
           for (int n = 0; n < n_tiles && ok; ++n) {
-            for (int kc = 0; kc < nkc; ++kc, ++ibc) {
+            for (int g = 0; g < ngr; ++g, ++ibc) {
               const int st = ibc % TC_B_STAGES;
               if (ibc >= TC_B_STAGES) ok = mbar_wait_bounded(bars + TCB_BEMPTY + st, ((ibc / TC_B_STAGES) - 1) & 1);
               if (!ok) break;
-              mbar_expect_tx(bars + TCB_BFULL + st, TC_B_CHUNK_BYTES);
-              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, kc * TC_KC, i * k + n * TC_N, bars + TCB_BFULL + st);
+              const int cnt_kc = min(TC_BG, nkc - g * TC_BG);
+              mbar_expect_tx(bars + TCB_BFULL + st, (unsigned)(cnt_kc * TC_B_CHUNK_BYTES));
+              for (int c = 0; c < cnt_kc; ++c)
+                tma_load_2d(sB + (size_t)(st * TC_BG + c) * TC_B_CHUNK_BYTES, &mapW, (g * TC_BG + c) * TC_KC, i * k + n * TC_N, bars + TCB_BFULL + st);
             }
           }
         }
@@ -201,6 +205,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       if (lane == 0) {
         unsigned um = it_m, ibc = it_bc, iacc = it_acc;
         bool ok = true;
+        const unsigned long long dA0 = tc_smem_desc(sA, 0), dB0 = tc_smem_desc(sB, 0);
         for (int m = 0; m < m_tiles && ok; ++m, ++um) {
           const int halves = min(TC_MH, (b - m * TC_MH * TC_M + TC_M - 1) / TC_M);
           for (int n = 0; n < n_tiles && ok; ++n, ++iacc) {
@@ -208,20 +213,30 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             if (iacc >= 2) ok = mbar_wait_bounded(bars + TCB_ACCEMPTY + buf, ((iacc >> 1) - 1) & 1);
             if (!ok) break;
             tc_fence_after();
-            for (int kc = 0; kc < nkc && ok; ++kc, ++ibc) {
+            for (int g = 0; g < ngr && ok; ++g, ++ibc) {
               const int st = ibc % TC_B_STAGES;
-              if (n == 0) ok = mbar_wait_bounded(bars + TCB_AFULL + kc, um & 1);
+              const int cnt_kc = min(TC_BG, nkc - g * TC_BG);
+              if (n == 0)
+                for (int c = 0; c < cnt_kc && ok; ++c) ok = mbar_wait_bounded(bars + TCB_AFULL + g * TC_BG + c, um & 1);
               if (ok) ok = mbar_wait_bounded(bars + TCB_BFULL + st, (ibc / TC_B_STAGES) & 1);
               if (!ok) break;
               tc_fence_after();
-              for (int h = 0; h < halves; ++h) {
+              for (int c = 0; c < cnt_kc; ++c) {
+                const int kc = g * TC_BG + c;
+                // operand descriptors: the base descriptor plus the chunk's offset in 16-byte units (the address field
+                // holds address >> 4 and shared memory is below 256 KB, so the sum stays inside the field)
+                const unsigned long long db = dB0 + (unsigned long long)((st * TC_BG + c) * (TC_B_CHUNK_BYTES >> 4));
+                for (int h = 0; h < halves; ++h) {
+                  const unsigned long long da = dA0 + (unsigned long long)((kc * TC_MH + h) * (TC_A_STAGE_BYTES >> 4));
 #pragma unroll
-                for (int k4 = 0; k4 < TC_KC / 16; ++k4)
-                  tc_mma_bf16(tmem + (unsigned)((buf * TC_MH + h) * TC_N), tc_smem_desc(sA + (size_t)(kc * TC_MH + h) * TC_A_STAGE_BYTES, k4 * 32),
-                              tc_smem_desc(sB + (size_t)st * TC_B_CHUNK_BYTES, k4 * 32), idesc, (kc | k4) != 0);
+                  for (int k4 = 0; k4 < TC_KC / 16; ++k4)
+                    tc_mma_bf16(tmem + (unsigned)((buf * TC_MH + h) * TC_N), da + (unsigned long long)(2 * k4), db + (unsigned long long)(2 * k4),
+                                idesc, (kc | k4) != 0);
+                }
               }
               tc_commit(bars + TCB_BEMPTY + st);                        // the ring slot is free when these MMAs have read it
-              if (n == n_tiles - 1) tc_commit(bars + TCB_AEMPTY + kc);  // and so is the sample chunk after its last centre block
+              if (n == n_tiles - 1)                                     // and so are the sample chunks after their last centre block
+                for (int c = 0; c < cnt_kc; ++c) tc_commit(bars + TCB_AEMPTY + g * TC_BG + c);
             }
             tc_commit(bars + TCB_ACCFULL + buf);                        // the accumulator stage is complete
           }
@@ -295,7 +310,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       if (!ok && lane == 0) atomicExch(&misc[2], 1);
     }
     it_m += (unsigned)m_tiles;
-    it_bc += (unsigned)(m_tiles * n_tiles * nkc);
+    it_bc += (unsigned)(m_tiles * n_tiles * ngr);
     it_acc += (unsigned)(n_tiles * m_tiles);
     if (tid == 0) misc[1] = 0;
     for (int a = tid; a < k; a += TC_THREADS) cnt[a] = 0;
