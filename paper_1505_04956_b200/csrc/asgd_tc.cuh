@@ -33,6 +33,7 @@ constexpr int TC_B_STAGES = 4;                            // ring slots for the 
 constexpr int TC_BG = 1;                                  // K chunks per ring slot (one wait and one commit per slot; 2 x 2 was no faster than 4 x 1)
 constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB per part
 constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;       // 32 KB
+constexpr int TC_SUM_ROWS = 4;                            // sample rows a centre's adders keep in flight
 constexpr int TC_MAX_K = 1024, TC_MAX_D = 256, TC_MAX_B = 8192;
 constexpr unsigned TC_INDEX_MASK = 1023u;
 
@@ -93,6 +94,28 @@ __global__ void tc_convert_x_kernel(const float* __restrict__ X, __nv_bfloat16* 
     __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
     *reinterpret_cast<__nv_bfloat162*>(out + e) = lo;
     *reinterpret_cast<__nv_bfloat162*>(out + e + 2) = hi;
+  }
+}
+
+// Adds the n listed sample rows (fp32 master) into S4, ROWS rows in flight, in list order.  Eight lanes share a
+// row: lane l8 holds dimensions 4*l8 + 32*q, q < nq <= QMAX.
+template <int ROWS, int QMAX>
+__device__ inline void tc_add_rows(const float* __restrict__ X, long long row0, int d, int nq, int l8,
+                                   const unsigned short* __restrict__ list, int n, float4 (&S4)[TC_MAX_D / 32]) {
+  for (int e0 = 0; e0 < n; e0 += ROWS) {
+    float4 v[ROWS][QMAX];
+#pragma unroll
+    for (int u = 0; u < ROWS; ++u) {
+      const bool have = e0 + u < n;
+      const float* x = X + (size_t)(row0 + (have ? (int)list[e0 + u] : 0)) * d + 4 * l8;
+#pragma unroll
+      for (int q = 0; q < QMAX; ++q)
+        v[u][q] = (q < nq && have) ? __ldg(reinterpret_cast<const float4*>(x + 32 * q)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < ROWS; ++u)
+#pragma unroll
+      for (int q = 0; q < QMAX; ++q) { S4[q].x += v[u][q].x; S4[q].y += v[u][q].y; S4[q].z += v[u][q].z; S4[q].w += v[u][q].w; }
   }
 }
 
@@ -500,21 +523,8 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         float4 S4[TC_MAX_D / 32];
 #pragma unroll
         for (int q = 0; q < TC_MAX_D / 32; ++q) S4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int e0 = 0; e0 < n; e0 += 2) {                 // two rows in flight; the adds keep ascending row order
-          float4 v[2][TC_MAX_D / 32];
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const bool have = e0 + u < n;
-            const float* x = p.X + (size_t)(row0 + (have ? (int)order[p0 + e0 + u] : 0)) * d + 4 * l8;
-#pragma unroll
-            for (int q = 0; q < TC_MAX_D / 32; ++q)
-              v[u][q] = (q < nq && have) ? __ldg(reinterpret_cast<const float4*>(x + 32 * q)) : make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-#pragma unroll
-          for (int u = 0; u < 2; ++u)
-#pragma unroll
-            for (int q = 0; q < TC_MAX_D / 32; ++q) { S4[q].x += v[u][q].x; S4[q].y += v[u][q].y; S4[q].z += v[u][q].z; S4[q].w += v[u][q].w; }
-        }
+        if (nq <= TC_MAX_D / 64) tc_add_rows<2 * TC_SUM_ROWS, TC_MAX_D / 64>(p.X, row0, d, nq, l8, order + p0, n, S4);
+        else tc_add_rows<TC_SUM_ROWS, TC_MAX_D / 32>(p.X, row0, d, nq, l8, order + p0, n, S4);
         float sq = 0.f;
         if (on) {
           if (plain) {
