@@ -11,12 +11,13 @@
 // whose two best scores are closer than the rounding bound of this form is decided again in the
 // direct difference form.
 //
-// Per-centre sums (Eq. 9): each warp files its 128 rows under the centres they chose (rank inside a
-// 32-row block from a match, so a warp's list of a centre is in row order; entries are byte offsets
-// into the tile, the unused tail of a list points at a row of zeros kept behind the tile).  Then lane
-// (centre, dimension pair) of the same warp adds the listed rows from the shared-memory
-// tile.  Every sum has a fixed order, so a step is reproducible.  The plain local step needs two
-// block-wide barriers.
+// Per-centre sums (Eq. 9): each warp orders its 128 rows by the centre they chose (rank inside a
+// 32-row block from a match, so a centre's rows stay in row order; entries are byte offsets into the
+// tile).  A centre's run starts at a multiple of eight entries and its unused tail points at a row of
+// zeros kept behind the tile, so the order falls into groups of eight rows of one centre.  Lane g of
+// the same warp adds the eight rows of group g over all dimensions; the update adds a centre's group
+// sums in order.  The work per lane does not depend on how unevenly the centres are chosen, every sum
+// has a fixed order (a step is reproducible), and the plain local step needs two block-wide barriers.
 #pragma once
 
 #include "asgd_step_tail.cuh"
@@ -29,8 +30,7 @@ constexpr int STREAM_STAGES = 2;
 constexpr int STREAM_SPT = 4;                          // samples per thread = 32-row blocks per warp
 constexpr int STREAM_MAX_B = STREAM_THREADS * STREAM_SPT;
 constexpr int STREAM_WARP_SAMPLES = 32 * STREAM_SPT;
-constexpr int STREAM_PARTS = STREAM_WARPS;              // partial sums per centre: one per warp
-constexpr int STREAM_SEG = STREAM_WARP_SAMPLES;        // capacity of a warp's list of one centre
+constexpr int STREAM_GROUP = 8;                        // rows of one centre added by one lane
 constexpr unsigned STREAM_WAIT_LIMIT = 1u << 22;       // bounded mbarrier wait (iterations of try_wait)
 
 __device__ inline unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -80,14 +80,18 @@ struct StreamLayout {
   static constexpr int CPW = 32 / D;                // centres a warp updates at a time
   static constexpr int ROWB = D * 4;                // bytes per sample
   static constexpr int ZR_EXTRA = (16 + ROWB - 1) / ROWB;   // rows between the batch's last row and the row of zeros (a copy may overrun by < 16 bytes)
-  static constexpr int CWS = (K + 1 + 3) / 4 * 4;   // a warp's list lengths, one spare counter for rows past the batch
+  static constexpr int CWS = (K + 1 + 3) / 4 * 4;   // a warp's counts per centre, one spare counter for rows past the batch
+  // a warp's rows ordered by centre, every centre's run padded to whole groups
+  static constexpr int CAP = (STREAM_WARP_SAMPLES + (STREAM_GROUP - 1) * K + STREAM_GROUP - 1) / STREAM_GROUP * STREAM_GROUP;
+  static constexpr int NGRP = CAP / STREAM_GROUP;   // groups a warp can have
+  static_assert(NGRP <= 32, "one lane per group");
 };
 
 // Shared-memory map of the streaming kernel (byte offsets, every region 16-byte aligned).
 template <int D, int K>
 struct StreamSmem {
   using L = StreamLayout<D, K>;
-  size_t ring, bars, flags, tail, wneg2, cnorm, w, sd, sw, cw, cnt, seen, lists, total;
+  size_t ring, bars, flags, tail, wneg2, cnorm, w, sd, cw, cq, first, cnt, seen, order, gsum, total;
   // a ring slot: the batch (source rounded out to 16-byte bounds), then a row of zeros wherever the batch starts in the slot
   __host__ __device__ static size_t slot_bytes(int b) {
     return ((size_t)(b + L::ZR_EXTRA) * L::ROWB + 16 + L::ROWB + 127) / 128 * 128;
@@ -103,11 +107,13 @@ struct StreamSmem {
     cnorm = take((size_t)K * 8);                                // (||w_a||^2, 0) pairs
     w = take((size_t)K * D * 4);
     sd = take((size_t)K * D * 4);
-    sw = take((size_t)STREAM_PARTS * K * D * 4);                // partial sums
-    cw = take((size_t)STREAM_WARPS * L::CWS * 4);               // list lengths
+    cw = take((size_t)STREAM_WARPS * L::CWS * 4);               // rows per (warp, centre)
+    cq = take((size_t)STREAM_WARPS * STREAM_SPT * L::CWS * 4);  // rows per (warp, 32-row block, centre)
+    first = take((size_t)STREAM_WARPS * L::CWS * 4);            // first group of (warp, centre); entry K = groups of the warp
     cnt = take((size_t)K * 4);
     seen = take((size_t)MAX_SLOTS * 4);
-    lists = take((size_t)STREAM_WARPS * K * STREAM_SEG * 2);    // u16 byte offsets of rows in the tile
+    order = take((size_t)STREAM_WARPS * L::CAP * 2);            // u16 byte offsets of rows in the tile, by centre
+    gsum = take((size_t)STREAM_WARPS * L::NGRP * D * 4);        // sums of the groups
     total = (off + 127) / 128 * 128;
   }
 };
@@ -118,7 +124,7 @@ template <int D, int K, bool kDet>
 __global__ void __launch_bounds__(STREAM_THREADS, 4)
 asgd_stream_kernel(const Params p, const long long steps) {
   using L = StreamLayout<D, K>;
-  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, ROWB = L::ROWB, CWS = L::CWS;
+  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, ROWB = L::ROWB, CWS = L::CWS, CAP = L::CAP, NGRP = L::NGRP;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int b = p.b;
   const unsigned slot_bytes = (unsigned)StreamSmem<D, K>::slot_bytes(b);
@@ -132,11 +138,13 @@ asgd_stream_kernel(const Params p, const long long steps) {
   float2* cnorm = reinterpret_cast<float2*>(smem_raw + map.cnorm);
   float* w = reinterpret_cast<float*>(smem_raw + map.w);
   float* SD = reinterpret_cast<float*>(smem_raw + map.sd);
-  float* Sw = reinterpret_cast<float*>(smem_raw + map.sw);
   int* Cw = reinterpret_cast<int*>(smem_raw + map.cw);
+  int* Cq = reinterpret_cast<int*>(smem_raw + map.cq);
+  int* First = reinterpret_cast<int*>(smem_raw + map.first);
+  float* Gsum = reinterpret_cast<float*>(smem_raw + map.gsum);
   int* cnt = reinterpret_cast<int*>(smem_raw + map.cnt);
   unsigned* seen_s = reinterpret_cast<unsigned*>(smem_raw + map.seen);
-  unsigned short* lists = reinterpret_cast<unsigned short*>(smem_raw + map.lists);
+  unsigned short* order = reinterpret_cast<unsigned short*>(smem_raw + map.order);
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int i = blockIdx.x;
@@ -209,7 +217,30 @@ asgd_stream_kernel(const Params p, const long long steps) {
   const float tau_scale = (float)(4 * D + 72) * 5.9604645e-8f;
   const float xmax2 = p.xmax2;                                              // max ||x||^2 over the samples
   int* myCw = Cw + wid * CWS;
-  unsigned short* myLists = lists + (size_t)wid * (K * STREAM_SEG);
+  int* myCq = Cq + wid * (STREAM_SPT * CWS);
+  int* myFirst = First + wid * CWS;
+  unsigned short* myOrder = order + (size_t)wid * CAP;
+  float* myGsum = Gsum + (size_t)wid * (NGRP * D);
+  // total of centre a, dimension j over the warps' groups, in a fixed order
+  auto centre_sum = [&](int a, int j) {
+    constexpr int AHEAD = 4;                         // groups of a (warp, centre) whose loads are issued at once
+    int g0[STREAM_WARPS], g1[STREAM_WARPS];
+#pragma unroll
+    for (int q = 0; q < STREAM_WARPS; ++q) { g0[q] = First[q * CWS + a]; g1[q] = First[q * CWS + a + 1]; }
+    float v[STREAM_WARPS][AHEAD];
+#pragma unroll
+    for (int q = 0; q < STREAM_WARPS; ++q)
+#pragma unroll
+      for (int u = 0; u < AHEAD; ++u) v[q][u] = (g0[q] + u < g1[q]) ? Gsum[(size_t)(q * NGRP + g0[q] + u) * D + j] : 0.f;
+    float ssum = 0.f;
+#pragma unroll
+    for (int q = 0; q < STREAM_WARPS; ++q) {
+#pragma unroll
+      for (int u = 0; u < AHEAD; ++u) ssum += v[q][u];
+      for (int g = g0[q] + AHEAD; g < g1[q]; ++g) ssum += Gsum[(size_t)(q * NGRP + g) * D + j];
+    }
+    return ssum;
+  };
   int abort = 0;
   for (long long step = 0; step < steps; ++step, ++t) {
     const int slot = (int)(step & 1);
@@ -225,11 +256,10 @@ asgd_stream_kernel(const Params p, const long long steps) {
     const int pos2 = next_pos(pos1);
     const int batch_nn = myperm[pos2];
     {
-      // this warp's lists: every entry points at the row of zeros, lengths zero
+      // this warp's order: every entry points at the row of zeros, counts zero
       const unsigned zz = zr_off | (zr_off << 16);
-      uint4* dst = reinterpret_cast<uint4*>(myLists);
-      for (int e = lane; e < K * STREAM_SEG / 8; e += 32) dst[e] = make_uint4(zz, zz, zz, zz);
-      for (int e = lane; e <= K; e += 32) myCw[e] = 0;
+      if (lane < NGRP) reinterpret_cast<uint4*>(myOrder)[lane] = make_uint4(zz, zz, zz, zz);
+      if (lane < STREAM_SPT * CWS / 4) reinterpret_cast<uint4*>(myCq)[lane] = make_uint4(0u, 0u, 0u, 0u);
     }
 
     unsigned head, bytes;
@@ -336,55 +366,79 @@ asgd_stream_kernel(const Params p, const long long steps) {
         if (r < b) p.assign_rec[(size_t)i * b + r] = best[q];
       }
     }
-    // ---- lists: this warp's rows under the centres they chose, in row order ----
+    // ---- order: this warp's rows by the centre they chose, in row order inside a centre ----
     __syncwarp();
+    int rank[STREAM_SPT];
+    int ngroups;
 #pragma unroll
     for (int q = 0; q < STREAM_SPT; ++q) {
       const unsigned grp = __match_any_sync(0xffffffffu, best[q]);
       const unsigned below = grp & ((1u << lane) - 1u);
-      const int base = myCw[best[q]];                                      // rows past the batch count into the spare counter
-      __syncwarp();
-      if (best[q] < K) myLists[best[q] * STREAM_SEG + base + __popc(below)] = (unsigned short)((wid * STREAM_WARP_SAMPLES + q * 32 + lane) * ROWB);
-      if (below == 0) myCw[best[q]] = base + __popc(grp);
-      __syncwarp();
+      rank[q] = __popc(below);
+      if (below == 0) myCq[q * CWS + best[q]] = __popc(grp);               // rows past the batch count into the spare counter
     }
     if (tid < p.S && my_seq != seen_s[tid]) flags[0] = 1;
-
+    __syncwarp();
+    {
+      // a row's place inside its centre: the centre's rows in the earlier 32-row blocks, then its rank in its own
+#pragma unroll
+      for (int q = 1; q < STREAM_SPT; ++q) {
+        int before = 0;
+#pragma unroll
+        for (int r = 0; r < q; ++r) before += myCq[r * CWS + best[q]];
+        rank[q] += before;
+      }
+      // lane = centre: its rows, its groups, and the first group by a running sum (lane K gets the total)
+      int n = 0;
+      if (lane < K) {
+#pragma unroll
+        for (int q = 0; q < STREAM_SPT; ++q) n += myCq[q * CWS + lane];
+        myCw[lane] = n;
+      }
+      const int ng = (n + STREAM_GROUP - 1) / STREAM_GROUP;
+      int inc = ng;
+#pragma unroll
+      for (int o = 1; o <= K; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += up;
+      }
+      const int first = inc - ng;
+      if (lane <= K) myFirst[lane] = first;
+      ngroups = __shfl_sync(0xffffffffu, inc, K);
+#pragma unroll
+      for (int q = 0; q < STREAM_SPT; ++q) {
+        const int f = __shfl_sync(0xffffffffu, first, best[q]);            // best[q] <= K
+        if (best[q] < K)
+          myOrder[f * STREAM_GROUP + rank[q]] = (unsigned short)((wid * STREAM_WARP_SAMPLES + q * 32 + lane) * ROWB);
+      }
+    }
     __syncwarp();
 
-    // ---- Eq. 9: lane (centre, dimension pair) adds the rows its own warp listed under the centre ----
+    // ---- Eq. 9: lanes (group, dimension pair) add the eight rows of a group (all of one centre) from the tile ----
     {
-      constexpr int ITEMS = K * D2;
-      for (int item = lane; item < ITEMS; item += 32) {
-        const int a = item / D2, jp = item - a * D2;
-        const unsigned char* xb = reinterpret_cast<const unsigned char*>(xs) + jp * 8;
-        auto row = [&](unsigned off) { return *reinterpret_cast<const float2*>(xb + off); };
-        float2 acc0 = make_float2(0.f, 0.f), acc1 = make_float2(0.f, 0.f);
-        const int n = myCw[a];
-        const uint4* seg = reinterpret_cast<const uint4*>(myLists + (size_t)a * STREAM_SEG);
-        for (int e0 = 0; e0 < n; e0 += 8) {                                // a list's tail points at the row of zeros
-          const uint4 pk = seg[e0 >> 3];
-          acc0 = __fadd2_rn(acc0, row(pk.x & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.x >> 16));
+      constexpr int GPR = 32 / D2;                                         // groups a warp adds at a time
+      const int gl = lane / D2, jp = lane - gl * D2;
+      const unsigned char* xb = reinterpret_cast<const unsigned char*>(xs) + jp * 8;
+      auto row = [&](unsigned off) { return *reinterpret_cast<const float2*>(xb + off); };
+      for (int g = gl; g < ngroups; g += GPR) {
+        if (gl < GPR) {
+          const uint4 pk = reinterpret_cast<const uint4*>(myOrder)[g];
+          float2 acc0 = row(pk.x & 0xffffu), acc1 = row(pk.x >> 16);
           acc0 = __fadd2_rn(acc0, row(pk.y & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.y >> 16));
           acc0 = __fadd2_rn(acc0, row(pk.z & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.z >> 16));
           acc0 = __fadd2_rn(acc0, row(pk.w & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.w >> 16));
+          *reinterpret_cast<float2*>(myGsum + (size_t)g * D + 2 * jp) = __fadd2_rn(acc0, acc1);
         }
-        *reinterpret_cast<float2*>(Sw + (size_t)(wid * K + a) * D + 2 * jp) = __fadd2_rn(acc0, acc1);
       }
     }
 
-    // ---- barrier B: partial sums and list lengths complete, the ring slot is free again ----
+    // ---- barrier B: group sums and counts complete, the ring slot is free again ----
     if (__syncthreads_or(abort)) { abort = 1; break; }
 
     const bool put_now = (to_put == 1);
     if (flags[0] != 0) {
       // a message is waiting: totals into SD, then the general tail (which also sends when a put is due)
-      for (int e = tid; e < KD; e += STREAM_THREADS) {
-        float ssum = 0.f;
-#pragma unroll
-        for (int q = 0; q < STREAM_PARTS; ++q) ssum += Sw[(size_t)q * KD + e];
-        SD[e] = ssum;
-      }
+      for (int e = tid; e < KD; e += STREAM_THREADS) SD[e] = centre_sum(e / D, e % D);
       if (tid < K) {
         int n = 0;
 #pragma unroll
@@ -414,9 +468,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
           int n = 0;
 #pragma unroll
           for (int q = 0; q < STREAM_WARPS; ++q) n += Cw[q * CWS + a];
-          float ssum = 0.f;
-#pragma unroll
-          for (int q = 0; q < STREAM_PARTS; ++q) ssum += Sw[(size_t)(q * K + a) * D + j];
+          const float ssum = centre_sum(a, j);
           const float ww = w[a * D + j];
           const float Dg = ((float)n * ww - ssum) * inv_b;
           const float nw = ww - eps * Dg;
