@@ -70,6 +70,46 @@ __device__ inline unsigned ld_relaxed_gpu(const unsigned* p) {
   return v;
 }
 
+// Shared-memory accesses of the order and sum phases: 32-bit shared addresses with constant offsets, so that an
+// access costs one instruction and no 64-bit address arithmetic.
+template <int OFF> __device__ __forceinline__ unsigned lds_u32(unsigned a) {
+  unsigned v;
+  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(a), "n"(OFF) : "memory");
+  return v;
+}
+template <int OFF> __device__ __forceinline__ uint4 lds_v4(unsigned a) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a), "n"(OFF) : "memory");
+  return v;
+}
+template <int OFF> __device__ __forceinline__ float2 lds_f2(unsigned a) {
+  float2 v;
+  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(v.x), "=f"(v.y) : "r"(a), "n"(OFF) : "memory");
+  return v;
+}
+template <int OFF> __device__ __forceinline__ void sts_u32(unsigned a, unsigned v) {
+  asm volatile("st.shared.u32 [%0+%2], %1;" ::"r"(a), "r"(v), "n"(OFF) : "memory");
+}
+template <int OFF> __device__ __forceinline__ void sts_u32_if(unsigned a, unsigned v, unsigned on) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.u32 p, %3, 0;\n @p st.shared.u32 [%0+%2], %1;\n}" ::"r"(a), "r"(v), "n"(OFF), "r"(on) : "memory");
+}
+template <int OFF> __device__ __forceinline__ void sts_v4(unsigned a, unsigned v) {
+  asm volatile("st.shared.v4.u32 [%0+%2], {%1,%1,%1,%1};" ::"r"(a), "r"(v), "n"(OFF) : "memory");
+}
+template <int OFF> __device__ __forceinline__ void sts_f2(unsigned a, float2 v) {
+  asm volatile("st.shared.v2.f32 [%0+%3], {%1,%2};" ::"r"(a), "f"(v.x), "f"(v.y), "n"(OFF) : "memory");
+}
+// running sum step: v += (value of the lane `o` below), lanes below `o` keep v
+__device__ __forceinline__ int scan_step(int v, int o) {
+  int r;
+  asm volatile("{\n .reg .pred p;\n .reg .b32 t;\n shfl.sync.up.b32 t|p, %1, %2, 0, 0xffffffff;\n @p add.s32 t, t, %1;\n @!p mov.b32 t, %1;\n mov.b32 %0, t;\n}" : "=r"(r) : "r"(v), "r"(o));
+  return r;
+}
+
+constexpr size_t stream_up16(size_t x) { return (x + 15) / 16 * 16; }
+
+// Sizes and the shared-memory map of the streaming kernel.  Everything but the ring has a place that depends on
+// (d, k) only, so those byte offsets are constants in the code; the ring (whose slots depend on b) comes last.
 template <int D, int K>
 struct StreamLayout {
   static_assert(D % 2 == 0 && D <= 16 && K <= 16, "streaming path: even d <= 16, k <= 16");
@@ -77,74 +117,62 @@ struct StreamLayout {
   static constexpr int D2 = D / 2;                  // dimension pairs
   static constexpr int INDEX_BITS = (K <= 2) ? 1 : (K <= 4) ? 2 : (K <= 8) ? 3 : 4;
   static constexpr unsigned INDEX_MASK = (1u << INDEX_BITS) - 1u;
-  static constexpr int CPW = 32 / D;                // centres a warp updates at a time
   static constexpr int ROWB = D * 4;                // bytes per sample
-  static constexpr int ZR_EXTRA = (16 + ROWB - 1) / ROWB;   // rows between the batch's last row and the row of zeros (a copy may overrun by < 16 bytes)
   static constexpr int CWS = (K + 1 + 3) / 4 * 4;   // a warp's counts per centre, one spare counter for rows past the batch
-  // a warp's rows ordered by centre, every centre's run padded to whole groups
-  static constexpr int CAP = (STREAM_WARP_SAMPLES + (STREAM_GROUP - 1) * K + STREAM_GROUP - 1) / STREAM_GROUP * STREAM_GROUP;
-  static constexpr int NGRP = CAP / STREAM_GROUP;   // groups a warp can have
-  static_assert(NGRP <= 32, "one lane per group");
-};
+  static constexpr int GPR = 32 / D2;               // groups a warp adds at a time: lanes (group, dimension pair)
+  static constexpr int CPW = GPR;                   // centres a warp updates: lanes (centre, dimension pair)
+  static constexpr int UPD_WARPS = (K + CPW - 1) / CPW;
+  static_assert(UPD_WARPS <= STREAM_WARPS, "update: every centre has a warp");
+  // a warp's rows ordered by centre, every centre's run padded to whole groups of eight
+  static constexpr int NGRP = (STREAM_WARP_SAMPLES + (STREAM_GROUP - 1) * K + STREAM_GROUP - 1) / STREAM_GROUP;
+  static constexpr int GCAP = (NGRP + 2 * GPR - 1) / (2 * GPR) * (2 * GPR);   // groups the adders may touch (whole double rounds)
+  static_assert(NGRP <= 32, "a running sum over one warp covers the groups");
 
-// Shared-memory map of the streaming kernel (byte offsets, every region 16-byte aligned).
-template <int D, int K>
-struct StreamSmem {
-  using L = StreamLayout<D, K>;
-  size_t ring, bars, flags, tail, wneg2, cnorm, w, sd, cw, cq, first, cnt, seen, order, gsum, total;
-  // a ring slot: the batch (source rounded out to 16-byte bounds), then a row of zeros wherever the batch starts in the slot
-  __host__ __device__ static size_t slot_bytes(int b) {
-    return ((size_t)(b + L::ZR_EXTRA) * L::ROWB + 16 + L::ROWB + 127) / 128 * 128;
-  }
-  __host__ __device__ explicit StreamSmem(int b) {
-    size_t off = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 15) / 16 * 16; return o; };
-    ring = take(STREAM_STAGES * slot_bytes(b));
-    bars = take(64);
-    flags = take(64);
-    tail = take(sizeof(TailScratch));
-    wneg2 = take((size_t)K * L::DP * 4);
-    cnorm = take((size_t)K * 8);                                // (||w_a||^2, 0) pairs
-    w = take((size_t)K * D * 4);
-    sd = take((size_t)K * D * 4);
-    cw = take((size_t)STREAM_WARPS * L::CWS * 4);               // rows per (warp, centre)
-    cq = take((size_t)STREAM_WARPS * STREAM_SPT * L::CWS * 4);  // rows per (warp, 32-row block, centre)
-    first = take((size_t)STREAM_WARPS * L::CWS * 4);            // first group of (warp, centre); entry K = groups of the warp
-    cnt = take((size_t)K * 4);
-    seen = take((size_t)MAX_SLOTS * 4);
-    order = take((size_t)STREAM_WARPS * L::CAP * 2);            // u16 byte offsets of rows in the tile, by centre
-    gsum = take((size_t)STREAM_WARPS * L::NGRP * D * 4);        // sums of the groups
-    total = (off + 127) / 128 * 128;
-  }
+  // fixed part of the map (byte offsets)
+  static constexpr size_t BARS = 0;
+  static constexpr size_t FLAGS = 64;
+  static constexpr size_t ZROW = 128;                                    // a row of zeros for the unused tail of a group
+  static constexpr size_t TAIL = ZROW + stream_up16(ROWB + 16);
+  static constexpr size_t WNEG2 = TAIL + stream_up16(sizeof(TailScratch));
+  static constexpr size_t CNORM = WNEG2 + stream_up16((size_t)K * DP * 4);   // (||w_a||^2, 0) pairs
+  static constexpr size_t W = CNORM + stream_up16((size_t)K * 8);
+  static constexpr size_t SD = W + stream_up16((size_t)K * D * 4);
+  static constexpr size_t CNT = SD + stream_up16((size_t)K * D * 4);
+  static constexpr size_t SEEN = CNT + stream_up16((size_t)K * 4);
+  static constexpr size_t WARP0 = SEEN + stream_up16((size_t)MAX_SLOTS * 4);
+  // per warp: rows per (32-row block, centre); rows per centre; first group per centre; the order; the group sums
+  static constexpr size_t W_CQ = 0;
+  static constexpr size_t W_CW = W_CQ + (size_t)STREAM_SPT * CWS * 4;
+  static constexpr size_t W_FIRST = W_CW + (size_t)CWS * 4;
+  static constexpr size_t W_ORDER = W_FIRST + (size_t)CWS * 4;           // u32 shared addresses of rows
+  static constexpr size_t W_GSUM = W_ORDER + (size_t)GCAP * STREAM_GROUP * 4;
+  static constexpr size_t WARP_STRIDE = stream_up16(W_GSUM + (size_t)GCAP * D * 4);
+  static constexpr size_t RING = (WARP0 + STREAM_WARPS * WARP_STRIDE + 127) / 128 * 128;
+  // a ring slot: the batch with its source rounded out to 16-byte bounds
+  __host__ __device__ static size_t slot_bytes(int b) { return ((size_t)b * ROWB + 32 + 127) / 128 * 128; }
+  __host__ __device__ static size_t total(int b) { return RING + STREAM_STAGES * slot_bytes(b); }
 };
 template <int D, int K>
-inline size_t stream_smem_bytes(int b) { return StreamSmem<D, K>(b).total; }
+inline size_t stream_smem_bytes(int b) { return StreamLayout<D, K>::total(b); }
 
 template <int D, int K, bool kDet>
 __global__ void __launch_bounds__(STREAM_THREADS, 4)
 asgd_stream_kernel(const Params p, const long long steps) {
   using L = StreamLayout<D, K>;
-  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, ROWB = L::ROWB, CWS = L::CWS, CAP = L::CAP, NGRP = L::NGRP;
+  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, ROWB = L::ROWB, CWS = L::CWS, GCAP = L::GCAP, GPR = L::GPR;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int b = p.b;
-  const unsigned slot_bytes = (unsigned)StreamSmem<D, K>::slot_bytes(b);
-  const unsigned zr_off = (unsigned)(b + L::ZR_EXTRA) * ROWB;              // from a batch's first row to the row of zeros
-  const StreamSmem<D, K> map(b);
-  unsigned char* ring = smem_raw + map.ring;
-  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + map.bars);   // [STAGES]
-  int* flags = reinterpret_cast<int*>(smem_raw + map.flags);                               // [0] a buffer has news
-  TailScratch* ts = reinterpret_cast<TailScratch*>(smem_raw + map.tail);
-  float* wneg2 = reinterpret_cast<float*>(smem_raw + map.wneg2);
-  float2* cnorm = reinterpret_cast<float2*>(smem_raw + map.cnorm);
-  float* w = reinterpret_cast<float*>(smem_raw + map.w);
-  float* SD = reinterpret_cast<float*>(smem_raw + map.sd);
-  int* Cw = reinterpret_cast<int*>(smem_raw + map.cw);
-  int* Cq = reinterpret_cast<int*>(smem_raw + map.cq);
-  int* First = reinterpret_cast<int*>(smem_raw + map.first);
-  float* Gsum = reinterpret_cast<float*>(smem_raw + map.gsum);
-  int* cnt = reinterpret_cast<int*>(smem_raw + map.cnt);
-  unsigned* seen_s = reinterpret_cast<unsigned*>(smem_raw + map.seen);
-  unsigned short* order = reinterpret_cast<unsigned short*>(smem_raw + map.order);
+  const unsigned slot_bytes = (unsigned)L::slot_bytes(b);
+  unsigned char* ring = smem_raw + L::RING;
+  unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + L::BARS);   // [STAGES]
+  int* flags = reinterpret_cast<int*>(smem_raw + L::FLAGS);                               // [0] a buffer has news
+  TailScratch* ts = reinterpret_cast<TailScratch*>(smem_raw + L::TAIL);
+  float* wneg2 = reinterpret_cast<float*>(smem_raw + L::WNEG2);
+  float2* cnorm = reinterpret_cast<float2*>(smem_raw + L::CNORM);
+  float* w = reinterpret_cast<float*>(smem_raw + L::W);
+  float* SD = reinterpret_cast<float*>(smem_raw + L::SD);
+  int* cnt = reinterpret_cast<int*>(smem_raw + L::CNT);
+  unsigned* seen_s = reinterpret_cast<unsigned*>(smem_raw + L::SEEN);
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int i = blockIdx.x;
@@ -154,11 +182,15 @@ asgd_stream_kernel(const Params p, const long long steps) {
   const unsigned batch_bytes = (unsigned)b * D * 4;
   const float inv_b = 1.0f / (float)b;
   const float eps = p.eps;
+  // shared addresses (32 bit): the block's base, this warp's arrays, the row of zeros
+  const unsigned sbase = smem_u32(smem_raw);
+  const unsigned wb = sbase + (unsigned)L::WARP0 + (unsigned)wid * (unsigned)L::WARP_STRIDE;
+  const unsigned zrow = sbase + (unsigned)L::ZROW;
+  auto warp_ptr = [&](int q, size_t off) { return smem_raw + L::WARP0 + (size_t)q * L::WARP_STRIDE + off; };
 
   // state on chip: w, -2w (padded rows), (||w_a||^2, 0)
   for (int e = tid; e < K * DP; e += STREAM_THREADS) wneg2[e] = 0.f;
-  for (int e = tid; e < STREAM_STAGES * (4 + D); e += STREAM_THREADS)       // the zeros behind each slot's batch, never overwritten
-    reinterpret_cast<float*>(ring + (size_t)(e / (4 + D)) * slot_bytes + zr_off)[e % (4 + D)] = 0.f;
+  for (int e = tid; e < (ROWB + 16) / 4; e += STREAM_THREADS) reinterpret_cast<float*>(smem_raw + L::ZROW)[e] = 0.f;
   __syncthreads();
   for (int e = tid; e < KD; e += STREAM_THREADS) {
     const float v = wglob[e];
@@ -211,61 +243,64 @@ asgd_stream_kernel(const Params p, const long long steps) {
   int pos1 = next_pos(pos);
   int batch_cur = myperm[pos];
   int batch_nxt = myperm[pos1];
-  if (tid == 0 && steps > 0) issue(batch_cur, 0);
+  if (tid == 0 && steps > 0) {
+    issue(batch_cur, 0);
+    if (steps > 1) issue(batch_nxt, 1);
+  }
   __syncthreads();
 
   const float tau_scale = (float)(4 * D + 72) * 5.9604645e-8f;
   const float xmax2 = p.xmax2;                                              // max ||x||^2 over the samples
-  int* myCw = Cw + wid * CWS;
-  int* myCq = Cq + wid * (STREAM_SPT * CWS);
-  int* myFirst = First + wid * CWS;
-  unsigned short* myOrder = order + (size_t)wid * CAP;
-  float* myGsum = Gsum + (size_t)wid * (NGRP * D);
-  // total of centre a, dimension j over the warps' groups, in a fixed order
-  auto centre_sum = [&](int a, int j) {
+  const unsigned lane_lt = (1u << lane) - 1u;
+  const int lane_c = min(lane, K);                                         // lanes past the centres share the spare column
+  const unsigned row0 = (unsigned)((wid * STREAM_WARP_SAMPLES + lane) * ROWB);   // this thread's first row in a tile
+
+  // total of centre a, dimension pair jp over the warps' groups, in a fixed order
+  auto centre_sum = [&](int a, int jp) {
     constexpr int AHEAD = 4;                         // groups of a (warp, centre) whose loads are issued at once
-    int g0[STREAM_WARPS], g1[STREAM_WARPS];
-#pragma unroll
-    for (int q = 0; q < STREAM_WARPS; ++q) { g0[q] = First[q * CWS + a]; g1[q] = First[q * CWS + a + 1]; }
-    float v[STREAM_WARPS][AHEAD];
-#pragma unroll
-    for (int q = 0; q < STREAM_WARPS; ++q)
-#pragma unroll
-      for (int u = 0; u < AHEAD; ++u) v[q][u] = (g0[q] + u < g1[q]) ? Gsum[(size_t)(q * NGRP + g0[q] + u) * D + j] : 0.f;
-    float ssum = 0.f;
+    float2 part[STREAM_WARPS];
 #pragma unroll
     for (int q = 0; q < STREAM_WARPS; ++q) {
+      const int* first = reinterpret_cast<const int*>(warp_ptr(q, L::W_FIRST));
+      const float2* gs = reinterpret_cast<const float2*>(warp_ptr(q, L::W_GSUM));
+      const int g0 = first[a], ng = first[a + 1] - g0;
+      const float2* src = gs + (size_t)g0 * D2 + jp;
+      float2 v[AHEAD];
 #pragma unroll
-      for (int u = 0; u < AHEAD; ++u) ssum += v[q][u];
-      for (int g = g0[q] + AHEAD; g < g1[q]; ++g) ssum += Gsum[(size_t)(q * NGRP + g) * D + j];
+      for (int u = 0; u < AHEAD; ++u) v[u] = (u < ng) ? src[u * D2] : make_float2(0.f, 0.f);
+      part[q] = __fadd2_rn(__fadd2_rn(v[0], v[1]), __fadd2_rn(v[2], v[3]));
+      for (int u = AHEAD; u < ng; ++u) part[q] = __fadd2_rn(part[q], src[u * D2]);
     }
-    return ssum;
+    return __fadd2_rn(__fadd2_rn(part[0], part[1]), __fadd2_rn(part[2], part[3]));
   };
+  auto centre_rows = [&](int a) {
+    int n = 0;
+#pragma unroll
+    for (int q = 0; q < STREAM_WARPS; ++q) n += reinterpret_cast<const int*>(warp_ptr(q, L::W_CW))[a];
+    return n;
+  };
+
   int abort = 0;
-  for (long long step = 0; step < steps; ++step, ++t) {
-    const int slot = (int)(step & 1);
-    const unsigned parity = (unsigned)((step >> 1) & 1);
-
-    // start the next batch's copy; peek at the receive buffers' sequence numbers (used after the sums)
-    if (tid == 0 && step + 1 < steps) {
-      fence_proxy_async_smem();
-      issue(batch_nxt, slot ^ 1);
-    }
-    unsigned my_seq = 0;
-    if (tid < p.S) my_seq = ld_relaxed_gpu(p.seq + (size_t)i * p.S + tid);
-    const int pos2 = next_pos(pos1);
-    const int batch_nn = myperm[pos2];
+  // A step's samples: the thread's rows of the batch in registers, the tile's shared address for the sums.
+  float2 xv[STREAM_SPT][D2];
+  unsigned xsa = 0;
+  // Gets batch `batch` (the one of step `s`) ready: resets this warp's order and counts, waits for the copy
+  // and loads the thread's rows.  Runs between the two barriers of the step before, beside the update.
+  auto stage_in = [&](long long s, int batch) {
     {
-      // this warp's order: every entry points at the row of zeros, counts zero
-      const unsigned zz = zr_off | (zr_off << 16);
-      if (lane < NGRP) reinterpret_cast<uint4*>(myOrder)[lane] = make_uint4(zz, zz, zz, zz);
-      if (lane < STREAM_SPT * CWS / 4) reinterpret_cast<uint4*>(myCq)[lane] = make_uint4(0u, 0u, 0u, 0u);
+      // this warp's order: every entry points at the row of zeros; counts zero
+#pragma unroll
+      for (int e = 0; e < (GCAP * STREAM_GROUP / 4 + 31) / 32; ++e)
+        if (e * 32 + lane < GCAP * STREAM_GROUP / 4) {
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(wb + (unsigned)L::W_ORDER + (unsigned)(e * 32 + lane) * 16u), "r"(zrow) : "memory");
+        }
+      if (lane < STREAM_SPT * CWS / 4)
+        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(wb + (unsigned)L::W_CQ + (unsigned)lane * 16u), "r"(0u) : "memory");
     }
-
     unsigned head, bytes;
-    const unsigned char* src = tile_src(batch_cur, head, bytes);
-    unsigned char* tile = ring + (size_t)slot * slot_bytes;
-    if (!mbar_wait_bounded(bars + slot, parity)) abort = 1;
+    const unsigned char* src = tile_src(batch, head, bytes);
+    unsigned char* tile = ring + (size_t)(s & 1) * slot_bytes;
+    if (!mbar_wait_bounded(bars + (s & 1), (unsigned)((s >> 1) & 1))) abort = 1;
     if (src + bytes > Xend) {
       // last rows of X: a rounded bulk copy would run past the array, use plain loads
       const float* g = reinterpret_cast<const float*>(src + head);
@@ -274,9 +309,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
       __syncthreads();
     }
     const float* xs = reinterpret_cast<const float*>(tile + head);
-
-    // ---- Eq. 8: scores of this thread's samples against every centre ----
-    float2 xv[STREAM_SPT][D2];
+    xsa = smem_u32(xs);
 #pragma unroll
     for (int q = 0; q < STREAM_SPT; ++q) {
       const int r = min(wid * STREAM_WARP_SAMPLES + q * 32 + lane, b - 1);   // rows past the batch re-read its last row
@@ -284,6 +317,18 @@ asgd_stream_kernel(const Params p, const long long steps) {
 #pragma unroll
       for (int jp = 0; jp < D2; ++jp) xv[q][jp] = xrow[jp];
     }
+  };
+  if (steps > 0) stage_in(0, batch_cur);
+  for (long long step = 0; step < steps; ++step, ++t) {
+    const int slot = (int)(step & 1);
+
+    // peek at the receive buffers' sequence numbers (used after the sums); next batch index but one
+    unsigned my_seq = 0;
+    if (tid < p.S) my_seq = ld_relaxed_gpu(p.seq + (size_t)i * p.S + tid);
+    const int pos2 = next_pos(pos1);
+    const int batch_nn = myperm[pos2];
+
+    // ---- Eq. 8: scores of this thread's samples against every centre ----
     float s1[STREAM_SPT], s2[STREAM_SPT];
 #pragma unroll
     for (int q = 0; q < STREAM_SPT; ++q) { s1[q] = __int_as_float(0x7f800000); s2[q] = __int_as_float(0x7f800000); }
@@ -369,65 +414,69 @@ asgd_stream_kernel(const Params p, const long long steps) {
     // ---- order: this warp's rows by the centre they chose, in row order inside a centre ----
     __syncwarp();
     int rank[STREAM_SPT];
-    int ngroups;
+    unsigned cqa[STREAM_SPT];                                              // address of this row's centre in the block counts
 #pragma unroll
     for (int q = 0; q < STREAM_SPT; ++q) {
       const unsigned grp = __match_any_sync(0xffffffffu, best[q]);
-      const unsigned below = grp & ((1u << lane) - 1u);
+      const unsigned below = grp & lane_lt;
       rank[q] = __popc(below);
-      if (below == 0) myCq[q * CWS + best[q]] = __popc(grp);               // rows past the batch count into the spare counter
+      cqa[q] = wb + (unsigned)L::W_CQ + ((unsigned)best[q] << 2);          // rows past the batch count into the spare column
+      if (q == 0) sts_u32_if<0 * CWS * 4>(cqa[q], (unsigned)__popc(grp), below == 0);
+      if (q == 1) sts_u32_if<1 * CWS * 4>(cqa[q], (unsigned)__popc(grp), below == 0);
+      if (q == 2) sts_u32_if<2 * CWS * 4>(cqa[q], (unsigned)__popc(grp), below == 0);
+      if (q == 3) sts_u32_if<3 * CWS * 4>(cqa[q], (unsigned)__popc(grp), below == 0);
     }
     if (tid < p.S && my_seq != seen_s[tid]) flags[0] = 1;
     __syncwarp();
+    int ngroups;
     {
       // a row's place inside its centre: the centre's rows in the earlier 32-row blocks, then its rank in its own
-#pragma unroll
-      for (int q = 1; q < STREAM_SPT; ++q) {
-        int before = 0;
-#pragma unroll
-        for (int r = 0; r < q; ++r) before += myCq[r * CWS + best[q]];
-        rank[q] += before;
-      }
-      // lane = centre: its rows, its groups, and the first group by a running sum (lane K gets the total)
-      int n = 0;
-      if (lane < K) {
-#pragma unroll
-        for (int q = 0; q < STREAM_SPT; ++q) n += myCq[q * CWS + lane];
-        myCw[lane] = n;
-      }
+      static_assert(STREAM_SPT == 4, "four 32-row blocks per warp");
+      rank[1] += (int)lds_u32<0>(cqa[1]);
+      rank[2] += (int)(lds_u32<0>(cqa[2]) + lds_u32<CWS * 4>(cqa[2]));
+      rank[3] += (int)(lds_u32<0>(cqa[3]) + lds_u32<CWS * 4>(cqa[3]) + lds_u32<2 * CWS * 4>(cqa[3]));
+      // lane = centre: its rows, its groups, and the first group by a running sum (entry K holds the total)
+      const unsigned ca = wb + (unsigned)L::W_CQ + ((unsigned)lane_c << 2);
+      int n = (int)(lds_u32<0>(ca) + lds_u32<CWS * 4>(ca) + lds_u32<2 * CWS * 4>(ca) + lds_u32<3 * CWS * 4>(ca));
+      n = (lane < K) ? n : 0;
+      sts_u32<(int)(L::W_CW - L::W_CQ)>(ca, (unsigned)n);
       const int ng = (n + STREAM_GROUP - 1) / STREAM_GROUP;
       int inc = ng;
 #pragma unroll
-      for (int o = 1; o <= K; o <<= 1) {
-        const int up = __shfl_up_sync(0xffffffffu, inc, o);
-        if (lane >= o) inc += up;
-      }
+      for (int o = 1; o < K; o <<= 1) inc = scan_step(inc, o);
       const int first = inc - ng;
-      if (lane <= K) myFirst[lane] = first;
-      ngroups = __shfl_sync(0xffffffffu, inc, K);
+      ngroups = __shfl_sync(0xffffffffu, inc, K - 1);                      // the running sum reaches K - 1 lanes down
+      sts_u32<(int)(L::W_FIRST - L::W_CQ)>(ca, (unsigned)((lane < K) ? first : ngroups));
 #pragma unroll
       for (int q = 0; q < STREAM_SPT; ++q) {
         const int f = __shfl_sync(0xffffffffu, first, best[q]);            // best[q] <= K
-        if (best[q] < K)
-          myOrder[f * STREAM_GROUP + rank[q]] = (unsigned short)((wid * STREAM_WARP_SAMPLES + q * 32 + lane) * ROWB);
+        const unsigned at = wb + (unsigned)L::W_ORDER + (((unsigned)f * STREAM_GROUP + (unsigned)rank[q]) << 2);
+        sts_u32_if<0>(at, xsa + row0 + (unsigned)(q * 32 * ROWB), best[q] < K);
       }
     }
     __syncwarp();
 
     // ---- Eq. 9: lanes (group, dimension pair) add the eight rows of a group (all of one centre) from the tile ----
     {
-      constexpr int GPR = 32 / D2;                                         // groups a warp adds at a time
       const int gl = lane / D2, jp = lane - gl * D2;
-      const unsigned char* xb = reinterpret_cast<const unsigned char*>(xs) + jp * 8;
-      auto row = [&](unsigned off) { return *reinterpret_cast<const float2*>(xb + off); };
-      for (int g = gl; g < ngroups; g += GPR) {
-        if (gl < GPR) {
-          const uint4 pk = reinterpret_cast<const uint4*>(myOrder)[g];
-          float2 acc0 = row(pk.x & 0xffffu), acc1 = row(pk.x >> 16);
-          acc0 = __fadd2_rn(acc0, row(pk.y & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.y >> 16));
-          acc0 = __fadd2_rn(acc0, row(pk.z & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.z >> 16));
-          acc0 = __fadd2_rn(acc0, row(pk.w & 0xffffu)); acc1 = __fadd2_rn(acc1, row(pk.w >> 16));
-          *reinterpret_cast<float2*>(myGsum + (size_t)g * D + 2 * jp) = __fadd2_rn(acc0, acc1);
+      const unsigned jo = (unsigned)jp * 8u;
+      auto group_sum = [&](const uint4& lo, const uint4& hi) {
+        float2 acc0 = lds_f2<0>(lo.x + jo), acc1 = lds_f2<0>(lo.y + jo);
+        acc0 = __fadd2_rn(acc0, lds_f2<0>(lo.z + jo)); acc1 = __fadd2_rn(acc1, lds_f2<0>(lo.w + jo));
+        acc0 = __fadd2_rn(acc0, lds_f2<0>(hi.x + jo)); acc1 = __fadd2_rn(acc1, lds_f2<0>(hi.y + jo));
+        acc0 = __fadd2_rn(acc0, lds_f2<0>(hi.z + jo)); acc1 = __fadd2_rn(acc1, lds_f2<0>(hi.w + jo));
+        return __fadd2_rn(acc0, acc1);
+      };
+      // two groups per lane in flight; groups past the last one hold the row of zeros
+      if (gl < GPR) {
+        for (int g = gl; g < ngroups; g += 2 * GPR) {
+          const unsigned oa = wb + (unsigned)L::W_ORDER + (unsigned)g * (STREAM_GROUP * 4);
+          const uint4 a0 = lds_v4<0>(oa), a1 = lds_v4<16>(oa);
+          const uint4 b0 = lds_v4<GPR * STREAM_GROUP * 4>(oa), b1 = lds_v4<GPR * STREAM_GROUP * 4 + 16>(oa);
+          const float2 sa = group_sum(a0, a1), sb = group_sum(b0, b1);
+          const unsigned ga = wb + (unsigned)L::W_GSUM + (unsigned)g * (D * 4) + jo;
+          sts_f2<0>(ga, sa);
+          sts_f2<GPR * D * 4>(ga, sb);
         }
       }
     }
@@ -435,16 +484,17 @@ asgd_stream_kernel(const Params p, const long long steps) {
     // ---- barrier B: group sums and counts complete, the ring slot is free again ----
     if (__syncthreads_or(abort)) { abort = 1; break; }
 
+    // the slot's rows have been added: start the copy of the batch after the next into it
+    if (tid == 0 && step + 2 < steps) {
+      fence_proxy_async_smem();
+      issue(batch_nn, slot);
+    }
     const bool put_now = (to_put == 1);
     if (flags[0] != 0) {
       // a message is waiting: totals into SD, then the general tail (which also sends when a put is due)
-      for (int e = tid; e < KD; e += STREAM_THREADS) SD[e] = centre_sum(e / D, e % D);
-      if (tid < K) {
-        int n = 0;
-#pragma unroll
-        for (int q = 0; q < STREAM_WARPS; ++q) n += Cw[q * CWS + tid];
-        cnt[tid] = n;
-      }
+      for (int e = tid; e < K * D2; e += STREAM_THREADS)
+        reinterpret_cast<float2*>(SD)[e] = centre_sum(e / D2, e % D2);
+      if (tid < K) cnt[tid] = centre_rows(tid);
       __syncthreads();
       step_tail<kDet>(p, i, t, w, D, SD, cnt, wglob, ts);
       if (tid < p.S) seen_s[tid] = p.seen[(size_t)i * p.S + tid];
@@ -458,32 +508,31 @@ asgd_stream_kernel(const Params p, const long long steps) {
         cnorm[tid] = make_float2(s, 0.f);
       }
     } else {
-      // common case: plain local step  w <- w - eps * D,  D = (n_a w - S) / b.  A warp updates CPW
-      // centres at a time, lane = (centre, dimension), and reduces ||w_a||^2 over the centre's lanes.
-      for (int a0 = wid * L::CPW; a0 < K; a0 += STREAM_WARPS * L::CPW) {
-        const int a = a0 + lane / D, j = lane % D;
-        const bool on = (lane < L::CPW * D) && (a < K);
+      // common case: plain local step  w <- w - eps * D,  D = (n_a w - S) / b.  The first warps update CPW
+      // centres each, lane = (centre, dimension pair), and reduce ||w_a||^2 over the centre's lanes.
+      if (wid < L::UPD_WARPS) {
+        const int al = lane / D2, jp = lane - al * D2;
+        const int a = wid * L::CPW + al;
+        const bool on = (al < L::CPW) && (a < K);
         float sq = 0.f;
         if (on) {
-          int n = 0;
-#pragma unroll
-          for (int q = 0; q < STREAM_WARPS; ++q) n += Cw[q * CWS + a];
-          const float ssum = centre_sum(a, j);
-          const float ww = w[a * D + j];
-          const float Dg = ((float)n * ww - ssum) * inv_b;
-          const float nw = ww - eps * Dg;
-          w[a * D + j] = nw;
-          wneg2[a * DP + j] = -2.f * nw;
-          wglob[a * D + j] = nw;
-          sq = nw * nw;
+          const int n = centre_rows(a);
+          const float2 ssum = centre_sum(a, jp);
+          const float2 ww = *reinterpret_cast<const float2*>(w + a * D + 2 * jp);
+          float2 nw;
+          nw.x = ww.x - eps * (((float)n * ww.x - ssum.x) * inv_b);
+          nw.y = ww.y - eps * (((float)n * ww.y - ssum.y) * inv_b);
+          *reinterpret_cast<float2*>(w + a * D + 2 * jp) = nw;
+          *reinterpret_cast<float2*>(wneg2 + a * DP + 2 * jp) = make_float2(-2.f * nw.x, -2.f * nw.y);
+          *reinterpret_cast<float2*>(wglob + a * D + 2 * jp) = nw;
+          sq = fmaf(nw.y, nw.y, nw.x * nw.x);
         }
 #pragma unroll
-        for (int o = 1; o < D; o <<= 1) {
+        for (int o = 1; o < D2; o <<= 1) {
           const float up = __shfl_down_sync(0xffffffffu, sq, o);
-          if (j + o < D) sq += up;
+          if (jp + o < D2) sq += up;
         }
-        __syncwarp();
-        if (on && j == 0) cnorm[a] = make_float2(sq, 0.f);
+        if (on && jp == 0) cnorm[a] = make_float2(sq, 0.f);
       }
       unsigned long long n_sent = 0;
       if (put_now) {
@@ -504,6 +553,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
     batch_nxt = batch_nn;
     pos1 = pos2;
     if (puts_on) to_put = (to_put == 1) ? p.c : to_put - 1;
+    if (step + 1 < steps) stage_in(step + 1, batch_cur);
     __syncthreads();                                   // barrier E: w, -2w, ||w||^2 ready for the next step
   }
 
