@@ -162,6 +162,34 @@ def test_edge_cases(case, parzen):
     pr.close()
 
 
+@pytest.mark.parametrize("shape", [(10, 10, 512), (10, 10, 500), (16, 16, 300), (4, 5, 111), (2, 3, 257)])
+@pytest.mark.parametrize("split", ["one_centre_takes_all", "two_centres_share", "one_centre_takes_most"])
+def test_stream_kernel_with_unbalanced_centres(shape, split):
+    """Centres that take very different numbers of rows: a warp's rows of one centre then span many groups of
+    eight (up to all sixteen), which is what the group sums and their totals in the update have to get right."""
+    d, k, b = shape
+    W = 3
+    wl = scaled("tiny", N=W * b * 4 + 5, d=d, k=k, W=W, b=b, comm_interval=2, fanout=1, eps=0.1)
+    rng = np.random.default_rng(1234 + d + k)
+    X = rng.standard_normal((wl.N, d)).astype(np.float32)
+    w0 = (50.0 + 10.0 * rng.standard_normal((k, d))).astype(np.float32)       # far from every sample
+    if split == "one_centre_takes_all":
+        w0[k - 1] = 0.0
+    elif split == "two_centres_share":
+        w0[0] = 0.3
+        w0[k - 1] = -0.3
+    else:
+        w0[1] = 0.0
+        w0[0] = 1.2                                                            # a small share for a second centre
+    pr = Pair(wl, X=X, w0=w0)
+    assert pr.gpu.path_name() == "fp32-stream"
+    pr.rounds(9)
+    pr.gpu.sync()
+    assert pr.max_rel_l2() < CENTRE_TOL, (shape, split, pr.max_rel_l2())
+    _compare_stats(pr, exact_accept=False)
+    pr.close()
+
+
 def test_specialised_and_general_kernels_agree():
     wl = scaled("tiny", N=30_000)
     a = Pair(wl, oracle=False)
