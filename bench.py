@@ -28,7 +28,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the stream kernel per algorithmic byte, from one ncu
 # capture of a 2^24-row case (profiles/asgd_stream_kernel__stream_workload.md); it grows in proportion to the rows
 # a launch processes.  Valid only for the kernel source it was taken on (first 12 hex digits of its SHA-1).
-TRAFFIC_CAPTURE = {"kernel_sha1": "5d1f14e76fbc", "traffic_per_algorithmic_byte": 670.99 / 663.51}
+TRAFFIC_CAPTURE = {"kernel_sha1": "7fe2a89ee610", "traffic_per_algorithmic_byte": 671.08 / 663.51}
 
 
 def env_int(name, default):
