@@ -509,7 +509,15 @@ int asgd_eval(asgd_ctx* c, int32_t worker, double* E_host) {
   const size_t smem = 32 * sizeof(double) + (on_chip ? wbytes : 0);
   CU(c, cudaFuncSetAttribute(eval_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   double* partial = (double*)(c->ws + c->L.eval_partial);
-  eval_kernel<<<kEvalBlocks, EVAL_THREADS, smem, c->stream>>>(p.X, p.N, p.d, p.k, w, on_chip, partial);
+  bool small = false;
+#define X(D_, K_)                                                                                     \
+  if (!small && p.d == D_ && p.k == K_) {                                                             \
+    eval_small_kernel<D_, K_><<<kEvalBlocks, EVAL_THREADS, 0, c->stream>>>(p.X, p.N, w, partial);     \
+    small = true;                                                                                     \
+  }
+  ASGD_STREAM_SHAPES(X)
+#undef X
+  if (!small) eval_kernel<<<kEvalBlocks, EVAL_THREADS, smem, c->stream>>>(p.X, p.N, p.d, p.k, w, on_chip, partial);
   c->launches += 1;
   CU(c, cudaGetLastError());
   std::vector<double> host(kEvalBlocks);

@@ -116,6 +116,47 @@ eval_kernel(const float* __restrict__ X, long long N, int d, int k, const float*
   }
 }
 
+// Eq. 8 for small states (even d <= 16, k <= 16): a thread keeps its row in registers (64-bit loads) and takes
+// the k direct-difference distances with packed two-wide adds and FMAs (even and odd dimensions in the two halves);
+// -w lies in shared memory as dimension pairs.  Same partials as eval_kernel: one fp64 sum per block.
+template <int D, int K>
+__global__ void __launch_bounds__(EVAL_THREADS)
+eval_small_kernel(const float* __restrict__ X, long long N, const float* __restrict__ wg, double* partial) {
+  static_assert(D % 2 == 0 && D <= 16 && K <= 16, "small states only");
+  constexpr int D2 = D / 2;
+  __shared__ float2 wneg[K * D2];
+  __shared__ double red[EVAL_THREADS / 32];
+  for (int e = threadIdx.x; e < K * D2; e += blockDim.x) wneg[e] = make_float2(-wg[2 * e], -wg[2 * e + 1]);
+  __syncthreads();
+  double acc = 0.0;
+  for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < N; r += (long long)gridDim.x * blockDim.x) {
+    const float2* x = reinterpret_cast<const float2*>(X + (size_t)r * D);     // rows are 8-byte aligned: D is even
+    float2 xv[D2];
+#pragma unroll
+    for (int jp = 0; jp < D2; ++jp) xv[jp] = __ldg(x + jp);
+    float bd = __int_as_float(0x7f800000);
+#pragma unroll
+    for (int a = 0; a < K; ++a) {
+      float2 s = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int jp = 0; jp < D2; ++jp) {
+        const float2 df = __fadd2_rn(xv[jp], wneg[a * D2 + jp]);
+        s = __ffma2_rn(df, df, s);
+      }
+      bd = fminf(bd, s.x + s.y);
+    }
+    acc += 0.5 * (double)bd;
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w_ = 0; w_ < (int)(blockDim.x >> 5); ++w_) s += red[w_];
+    partial[blockIdx.x] = s;
+  }
+}
+
 // max_i ||x_i||^2 over the rows the workers can touch (one pass at initialisation).
 __global__ void xmax2_kernel(const float* __restrict__ X, long long N, int d, unsigned* out_bits) {
   float m = 0.f;
