@@ -100,7 +100,7 @@ __device__ inline unsigned long long step_send(const Params& p, int i, unsigned 
 }
 
 // w     [k rows of d, row stride wstride]  this worker's state (shared or global memory), updated in place
-// SD    [kd]  in: per-centre sums S_k of the mini-batch; out: the local gradient D
+// SD    [kd]  per-centre sums S_k of the mini-batch (read only)
 // cnt   [k]   per-centre counts n_k
 // wglob       the worker's row of Params::state when w lives in shared memory, else nullptr
 // sd_l2       the sums in SD were produced by reductions in L2: read them past L1
@@ -117,19 +117,16 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
   const float inv_b = 1.0f / (float)p.b;
   const float eps = p.eps;
 
-  // Eq. 9 (true-gradient sign, mean over the mini-batch size): D_k = (n_k w_k - S_k) / b
-#pragma unroll 4
-  for (int q = tid; q < nvec; q += nt) {
-    const int e = q * V;
+  // Eq. 9 (true-gradient sign, mean over the mini-batch size): D_k = (n_k w_k - S_k) / b, formed from the sums where
+  // it is needed (in the acceptance test and in the update) instead of in a pass of its own over the state
+  auto gradient = [&](int e, const TailVec<V>& ww) {
     const float n = (float)cnt[e / d];
     const TailVec<V> sums = sd_l2 ? tail_ldcg<V>(SD + e) : tail_ld<V>(SD + e);
-    const TailVec<V> ww = tail_ld<V>(w + widx(e));
     TailVec<V> D;
 #pragma unroll
     for (int u = 0; u < V; ++u) D.v[u] = (n * ww.v[u] - sums.v[u]) * inv_b;
-    tail_st<V>(SD + e, D);
-  }
-  __syncthreads();
+    return D;
+  };
 
   // receive buffers: thread s looks at buffer s (all buffers at once, one L2 round trip)
   int m = 0;
@@ -161,8 +158,8 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
         for (int q = tid; q < nvec; q += nt) {
           const int e = q * V;
           const TailVec<V> vv = tail_ldcg<V>(v + e);
-          const TailVec<V> D = tail_ld<V>(SD + e);
           const TailVec<V> ww = tail_ld<V>(w + widx(e));
+          const TailVec<V> D = gradient(e, ww);
 #pragma unroll
           for (int u = 0; u < V; ++u) {
             const float df = ww.v[u] - vv.v[u];
@@ -199,7 +196,8 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
         const float* __restrict__ v = p.mail + si * (size_t)p.kd_pad + (size_t)a * d;
         double dot = 0.0, dd = 0.0, nv = 0.0;
         for (int j = lane; j < d; j += 32) {
-          const float vv = __ldcg(v + j), D = SD[a * d + j], ww = w[widx(a * d + j)];
+          const float vv = __ldcg(v + j), ww = w[widx(a * d + j)];
+          const float D = ((float)cnt[a] * ww - (sd_l2 ? __ldcg(SD + a * d + j) : SD[a * d + j])) * inv_b;
           const float df = ww - vv;
           dot += (double)D * (double)df;
           dd += (double)D * (double)D;
@@ -242,7 +240,7 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
       }
     const int we = widx(e);
     const TailVec<V> ww = tail_ld<V>(w + we);
-    const TailVec<V> D = tail_ld<V>(SD + e);
+    const TailVec<V> D = gradient(e, ww);
     TailVec<V> nw;
 #pragma unroll
     for (int u = 0; u < V; ++u) {
