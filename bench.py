@@ -27,8 +27,18 @@ CPU_SAMPLE_ROWS = 1 << 25          # prefix of the workload the CPU baseline run
 NOMINAL_HBM_GBS = 8000.0
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the stream kernel per algorithmic byte, from one ncu
 # capture of a 2^24-row case (profiles/asgd_stream_kernel__stream_workload.md); it grows in proportion to the rows
-# a launch processes.  Valid only for the kernel source it was taken on (first 12 hex digits of its SHA-1).
-TRAFFIC_CAPTURE = {"kernel_sha1": "7fe2a89ee610", "traffic_per_algorithmic_byte": 671.08 / 663.51}
+# a launch processes.  Valid only for the kernel sources it was taken on (stream_kernel_sha1()).
+TRAFFIC_CAPTURE = {"kernel_sha1": "3dee0be9b006", "traffic_per_algorithmic_byte": 670.41 / 663.51}
+
+
+def stream_kernel_sha1():
+    """First 12 hex digits of the SHA-1 over the sources the streaming kernel is compiled from."""
+    import hashlib
+    h = hashlib.sha1()
+    for name in ("asgd_common.cuh", "asgd_step_tail.cuh", "asgd_stream.cuh"):
+        with open(os.path.join(ROOT, "paper_1505_04956_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
 
 
 def env_int(name, default):
@@ -251,10 +261,8 @@ def main():
     bytes_per_launch = algorithmic_bytes_per_pass(wl, steps, args.partial_rows)
     achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
     traffic = None
-    with open(os.path.join(ROOT, "paper_1505_04956_b200", "csrc", "asgd_stream.cuh"), "rb") as f:
-        import hashlib
-        if ctx.path_name() == "fp32-stream" and hashlib.sha1(f.read()).hexdigest()[:12] == TRAFFIC_CAPTURE["kernel_sha1"]:
-            traffic = bytes_per_launch * TRAFFIC_CAPTURE["traffic_per_algorithmic_byte"]
+    if ctx.path_name() == "fp32-stream" and stream_kernel_sha1() == TRAFFIC_CAPTURE["kernel_sha1"]:
+        traffic = bytes_per_launch * TRAFFIC_CAPTURE["traffic_per_algorithmic_byte"]
     if ctx.path_name() in ("fp32-tiled",):
         # bound by the fp32 pipe: 2*k*d flops per sample against SMs x 128 lanes x 2 x max SM clock
         props = torch.cuda.get_device_properties(dev)
