@@ -30,7 +30,11 @@ struct TiledShape {
   static_assert(D % 32 == 0 && KP == 32 * WK && WK <= 4, "tiled path: d a multiple of 32, KP = 32 * WK, WK <= 4");
   static constexpr int THREADS = 32 * WS * WK;
   static constexpr int WARPS = WS * WK;
-  static constexpr int TS = 16 * WS;              // samples per tile
+  static constexpr int TS0 = 16 * WS;             // samples the warps score at a time (a sub-tile)
+  static constexpr int RB = (D == 32) ? 128 / TS0 : 1;   // sub-tiles per tile: short rows (d = 32) come 128 at a time, so that
+                                                  // the merge, second-look and sum phases and their barriers run once per 128 rows
+  static constexpr int TS = TS0 * RB;             // samples per tile
+  static_assert(TS <= THREADS && TS <= 128, "a thread per tile row in the merge phase; the sums take up to 128 rows");
   static constexpr int XS = D;                    // row stride inside a quarter of a sample tile (floats)
   static constexpr int QR = 4 * WS;               // rows per quarter; a lane's sample group sg reads quarter sg
   static constexpr int QS = QR * D + 4;           // quarter stride: each quarter starts 4 floats (one bank group) later,
@@ -52,7 +56,7 @@ struct TiledSmem {
     cn = take((size_t)KP * 4);
     S = take((size_t)k * D * 4);
     cnt = take((size_t)KP * 4);
-    xt = take((size_t)2 * 4 * T::QS * 4);
+    xt = take((size_t)2 * T::RB * 4 * T::QS * 4);
     best = take((size_t)T::TS * 4);
     red = take((size_t)WK * T::TS * 8);
     flagged = take((size_t)(T::TS + 4) * 4);
@@ -70,7 +74,7 @@ template <int D, int KP, int WS, int WK, int MINB, bool kDet>
 __global__ void __launch_bounds__(32 * WS * WK, MINB)
 asgd_tiled_kernel(const Params p, const long long steps) {
   using T = TiledShape<D, KP, WS, WK>;
-  constexpr int TS = T::TS, XS = T::XS, QR = T::QR, QS = T::QS, WST = T::WST, THREADS = T::THREADS, WARPS = T::WARPS, DR = T::DR;
+  constexpr int TS = T::TS, TS0 = T::TS0, RB = T::RB, XS = T::XS, QR = T::QR, QS = T::QS, WST = T::WST, THREADS = T::THREADS, WARPS = T::WARPS, DR = T::DR;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int k = p.k, b = p.b;
   const TiledSmem<D, KP, WS, WK> map(k);
@@ -78,7 +82,7 @@ asgd_tiled_kernel(const Params p, const long long steps) {
   float* cn = reinterpret_cast<float*>(smem_raw + map.cn);          // [KP]      ||w_a||^2 (+inf for padding)
   float* S = reinterpret_cast<float*>(smem_raw + map.S);            // [k][D]
   int* cnt = reinterpret_cast<int*>(smem_raw + map.cnt);            // [KP]
-  float* xt = reinterpret_cast<float*>(smem_raw + map.xt);          // [2][4 quarters][QR][XS] (+4 floats per quarter)
+  float* xt = reinterpret_cast<float*>(smem_raw + map.xt);          // [2][RB sub-tiles][4 quarters][QR][XS] (+4 floats per quarter)
   int* best = reinterpret_cast<int*>(smem_raw + map.best);          // [TS]
   float2* red = reinterpret_cast<float2*>(smem_raw + map.red);      // [WK][TS] (minimum, runner-up)
   int* flagged = reinterpret_cast<int*>(smem_raw + map.flagged);    // [0] count, [1..] tile rows to decide again
@@ -116,13 +120,14 @@ asgd_tiled_kernel(const Params p, const long long steps) {
     const long long batch = p.perm[(size_t)i * p.B + (size_t)(t % (unsigned long long)p.B)];
     const int rows = min(TS, b - tl * TS);
     const int slot = (int)(nx_g & 1);
-    float* dst = xt + (size_t)slot * 4 * QS;
+    float* dst = xt + (size_t)slot * RB * 4 * QS;
     const float* src = p.X + ((size_t)i * p.H + (size_t)batch * b + (size_t)tl * TS) * D;
     if (lane == 0) mbar_expect_tx(bars + slot, (unsigned)rows * D * 4);
     __syncwarp();
-    if (lane < 4) {                                   // one copy per quarter of the tile
-      const int qrows = min(QR, rows - lane * QR);
-      if (qrows > 0) bulk_g2s(dst + (size_t)lane * QS, src + (size_t)lane * QR * D, (unsigned)qrows * D * 4, bars + slot);
+    if (lane < 4 * RB) {                              // one copy per quarter of every sub-tile
+      const int first = (lane / 4) * TS0 + (lane % 4) * QR;          // the quarter's first row in the tile
+      const int qrows = min(QR, rows - first);
+      if (qrows > 0) bulk_g2s(dst + (size_t)lane * QS, src + (size_t)first * D, (unsigned)qrows * D * 4, bars + slot);
     }
     ++nx_g;
     if (++nx_tl == tiles) { nx_tl = 0; if (++nx_v == nv) { nx_v = 0; ++nx_st; } }
@@ -181,58 +186,60 @@ asgd_tiled_kernel(const Params p, const long long steps) {
         const int slot = (int)(g & 1);
         const unsigned parity = (unsigned)((g >> 1) & 1);
         const int rows = min(TS, b - tl * TS);
-        const float* xb = xt + (size_t)slot * 4 * QS;
-        auto xrowp = [&](int r) { return xb + (size_t)(r / QR) * QS + (size_t)(r % QR) * XS; };   // tile row r
+        const float* xb = xt + (size_t)slot * RB * 4 * QS;
+        auto xrowp = [&](int r) { return xb + (size_t)(r / QR) * QS + (size_t)(r % QR) * XS; };   // tile row r (quarters of all sub-tiles are QS apart)
         if (tid == 0) flagged[0] = 0;
         if (!mbar_wait_bounded(bars + slot, parity)) abort = 1;
 
-        // ---- scores of the warp's 16 x 32 block: acc[m][i] = sum_j x[row m][j] * (-2 w[centre i][j]) ----
-        float acc[4][4];
-#pragma unroll
-        for (int m = 0; m < 4; ++m)
-#pragma unroll
-          for (int c = 0; c < 4; ++c) acc[m][c] = 0.f;
-        const float* xrow = xb + (size_t)sg * QS + (size_t)(wsi * 4) * XS;    // rows sg*QR + wsi*4 + m
-        const float* wrow = wR + (size_t)(wk * 32 + cg) * WST;
-#pragma unroll 2
-        for (int j = 0; j < D; j += 4) {
-          float4 xv[4], wv[4];
-#pragma unroll
-          for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xrow + (size_t)m * XS + j);
-#pragma unroll
-          for (int c = 0; c < 4; ++c) wv[c] = *reinterpret_cast<const float4*>(wrow + (size_t)(8 * c) * WST + j);
-#pragma unroll
+        for (int rb = 0; rb < RB && rb * TS0 < rows; ++rb) {   // the tile's sub-tiles in turn (the same trip count for every thread)
+          // ---- scores of the warp's 16 x 32 block: acc[m][i] = sum_j x[row m][j] * (-2 w[centre i][j]) ----
+          float acc[4][4];
+  #pragma unroll
           for (int m = 0; m < 4; ++m)
-#pragma unroll
+  #pragma unroll
+            for (int c = 0; c < 4; ++c) acc[m][c] = 0.f;
+          const float* xrow = xb + (size_t)(rb * 4 + sg) * QS + (size_t)(wsi * 4) * XS;    // rows rb*TS0 + sg*QR + wsi*4 + m
+          const float* wrow = wR + (size_t)(wk * 32 + cg) * WST;
+  #pragma unroll 2
+          for (int j = 0; j < D; j += 4) {
+            float4 xv[4], wv[4];
+  #pragma unroll
+            for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xrow + (size_t)m * XS + j);
+  #pragma unroll
+            for (int c = 0; c < 4; ++c) wv[c] = *reinterpret_cast<const float4*>(wrow + (size_t)(8 * c) * WST + j);
+  #pragma unroll
+            for (int m = 0; m < 4; ++m)
+  #pragma unroll
+              for (int c = 0; c < 4; ++c) {
+                acc[m][c] = fmaf(xv[m].x, wv[c].x, acc[m][c]);
+                acc[m][c] = fmaf(xv[m].y, wv[c].y, acc[m][c]);
+                acc[m][c] = fmaf(xv[m].z, wv[c].z, acc[m][c]);
+                acc[m][c] = fmaf(xv[m].w, wv[c].w, acc[m][c]);
+              }
+          }
+          // minimum and runner-up over the lane's 4 centres, then over the 8 lanes that share the rows
+          float cnv[4];
+  #pragma unroll
+          for (int c = 0; c < 4; ++c) cnv[c] = cn[wk * 32 + 8 * c + cg];
+  #pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            float s1 = INF, s2 = INF;
+  #pragma unroll
             for (int c = 0; c < 4; ++c) {
-              acc[m][c] = fmaf(xv[m].x, wv[c].x, acc[m][c]);
-              acc[m][c] = fmaf(xv[m].y, wv[c].y, acc[m][c]);
-              acc[m][c] = fmaf(xv[m].z, wv[c].z, acc[m][c]);
-              acc[m][c] = fmaf(xv[m].w, wv[c].w, acc[m][c]);
+              const float sc = acc[m][c] + cnv[c];
+              const float sp = __uint_as_float((__float_as_uint(sc) & ~T::INDEX_MASK) | (unsigned)(8 * c + cg));
+              s2 = fmaxf(s1, fminf(s2, sp));
+              s1 = fminf(s1, sp);
             }
-        }
-        // minimum and runner-up over the lane's 4 centres, then over the 8 lanes that share the rows
-        float cnv[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) cnv[c] = cn[wk * 32 + 8 * c + cg];
-#pragma unroll
-        for (int m = 0; m < 4; ++m) {
-          float s1 = INF, s2 = INF;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const float sc = acc[m][c] + cnv[c];
-            const float sp = __uint_as_float((__float_as_uint(sc) & ~T::INDEX_MASK) | (unsigned)(8 * c + cg));
-            s2 = fmaxf(s1, fminf(s2, sp));
-            s1 = fminf(s1, sp);
+  #pragma unroll
+            for (int o = 1; o < 8; o <<= 1) {
+              const float o1 = __shfl_xor_sync(0xffffffffu, s1, o);
+              const float o2 = __shfl_xor_sync(0xffffffffu, s2, o);
+              s2 = fminf(fmaxf(s1, o1), fminf(s2, o2));
+              s1 = fminf(s1, o1);
+            }
+            if (cg == 0) red[(size_t)wk * TS + rb * TS0 + sg * QR + wsi * 4 + m] = make_float2(s1, s2);
           }
-#pragma unroll
-          for (int o = 1; o < 8; o <<= 1) {
-            const float o1 = __shfl_xor_sync(0xffffffffu, s1, o);
-            const float o2 = __shfl_xor_sync(0xffffffffu, s2, o);
-            s2 = fminf(fmaxf(s1, o1), fminf(s2, o2));
-            s1 = fminf(s1, o1);
-          }
-          if (cg == 0) red[(size_t)wk * TS + sg * QR + wsi * 4 + m] = make_float2(s1, s2);
         }
         // the ring slot of the previous tile is free since that tile's last barrier: fetch the next tile now
         if (wid == ISSUER && g + 1 < total_tiles) {
