@@ -116,7 +116,7 @@ int asgd_set_state(asgd_ctx *ctx, int32_t worker, const float *w_dev /* DEVICE [
 /* A put from outside: write a whole message into receive buffer `slot` of `worker`. */
 int asgd_put(asgd_ctx *ctx, int32_t worker, int32_t slot, const float *payload_dev /* DEVICE [k*d] */);
 
-/* Per-centre messages (Section 4.4: updates are partitioned "along the individual cluster centers"),
+/* Per-centre messages (Section 4.4: K-Means updates are split per centre row of the state),
  * cfg.partial_rows = m >= 1.  The paper states no formulas for them; the library applies Eq. 3, Eq. 4
  * and Eq. 6 to each centre row on its own: a put after step t carries the m consecutive rows (cyclic)
  * that start at row h(seed, 4, i, t, j) mod k of the sender's new state; for every new message that
@@ -136,18 +136,22 @@ int asgd_get_accept_rows(asgd_ctx *ctx, int32_t worker, int32_t *out_host /* HOS
 /* Eq. 8: E(w) of the given worker's state (-1 = mean state) over all N rows.  Synchronises. */
 int asgd_eval(asgd_ctx *ctx, int32_t worker, double *E_host /* HOST out */);
 
-/* out_host[5] = steps, messages sent, received, accepted ("good", delta = 1), overwritten unread.
+/* The per-worker message counters of Fig. 12 (messages sent, received, and "good" ones, i.e. those the
+ * Parzen window of Eq. 4 let through), plus the steps done and the messages overwritten before their
+ * owner looked:  out_host[5] = steps, sent, received, accepted (delta = 1), overwritten unread.
  * Synchronises. */
 int asgd_get_stats(asgd_ctx *ctx, int32_t worker, uint64_t *out_host /* HOST [5] */);
 
 /* Assignments s_i(w) of the last deterministic round, [W*b] int32 in worker-major order.
  * Needs cfg.record_assign = 1.  out_dev: DEVICE, caller's. */
 int asgd_get_assign(asgd_ctx *ctx, int32_t *out_dev);
-/* Per-slot acceptance of the last step of `worker`: out_host[S], -1 nothing new, 0 rejected,
- * 1 accepted.  Synchronises. */
+/* Outcome of the acceptance test of Eq. 4 (times lambda of Eq. 3) per receive buffer in the last step of
+ * `worker`: out_host[S], -1 nothing new, 0 rejected, 1 accepted.  Synchronises. */
 int asgd_get_accept(asgd_ctx *ctx, int32_t worker, int32_t *out_host /* HOST [S] */);
 
-/* Wait for the stream and return the device status word (ASGD_OK or ASGD_ETIMEOUT ...). */
+/* Wait for the stream and return the device status word (ASGD_OK, or ASGD_ETIMEOUT when a worker kernel
+ * gave up a bounded wait on one of its own copies).  Housekeeping of this library: the paper has no
+ * counterpart (its workers never wait, Section 1.2; neither do these, on one another). */
 int asgd_sync(asgd_ctx *ctx);
 /* Number of kernels this context has launched so far. */
 int64_t asgd_launch_count(const asgd_ctx *ctx);

@@ -17,12 +17,13 @@
 //   Parzen acceptance delta     -- Eq. 4 (literal two-norm form, strict "<")
 //   lambda (buffer non-empty)   -- Eq. 3
 //   merged step                 -- Eq. 6 / Eq. 7, then  w <- w - eps * Dbar  (Algorithm 5)
-//   send                        -- Algorithm 5 "send w_{t+1} to random node != i"
+//   send                        -- Algorithm 5, send line: the new state goes to random workers other than i
 //   partial (per-centre) puts   -- Section 4.4: a message carries some of the centre rows, lambda and
 //                                  delta are then taken row by row (the reading is stated at worker_step_rows)
 //
 // Parity status: every function here is pinned by the CPU tests (brute force, closed forms,
-// special cases, invariants).  The free-running asynchronous mode of the CUDA library has no
+// special cases, invariants); the optional parallel loop over the workers of a round is pinned
+// bit for bit against the single-threaded loop.  The free-running asynchronous mode of the CUDA library has no
 // step-wise counterpart here ("parity unpinned" for that mode only): races are part of the
 // method, so it is compared statistically through E(w).
 //
@@ -103,7 +104,7 @@ struct Oracle {
   int threads = 1;
 };
 
-// Algorithm 5 "shuffle samples on node i", at mini-batch granularity: Fisher-Yates from the top.
+// Algorithm 5, shuffle line (each worker shuffles its own samples), at mini-batch granularity: Fisher-Yates from the top.
 void make_perm(const Config& c, int64_t B, int32_t worker, std::vector<int32_t>& perm) {
   perm.resize(B);
   for (int64_t p = 0; p < B; ++p) perm[p] = (int32_t)p;
@@ -114,7 +115,7 @@ void make_perm(const Config& c, int64_t B, int32_t worker, std::vector<int32_t>&
   }
 }
 
-// Algorithm 5 "random node != i": the j-th recipient of the put that follows step t.
+// Algorithm 5, send line (a random worker other than i): the j-th recipient of the put that follows step t.
 // Uniform over the W-1 other workers; a repeat of an earlier recipient moves on to the next
 // worker (cyclically, skipping the sender) until it is new.
 void recipients(const Config& c, int32_t i, uint64_t t, int32_t* peers, int32_t* slots) {
@@ -222,8 +223,8 @@ void worker_step(const Oracle& o, Worker& me, int32_t i) {
   }
 }
 
-// The same step when messages carry single centre rows (Section 4.4: "for K-Means we partition along the
-// individual cluster centers of the states").  The paper gives no formulas for this case; the reading
+// The same step when messages carry single centre rows (Section 4.4: K-Means updates are split per
+// centre row of the state).  The paper gives no formulas for this case; the reading
 // taken here applies Eq. 3, Eq. 4 and Eq. 6 to each centre row k on its own:
 //   lambda_{s,k} = 1 if buffer s holds a new message that carries row k and that row is not all zero,
 //   delta_{s,k}  = [ ||(w_k - eps D_k) - v_{s,k}||^2 < ||w_k - v_{s,k}||^2 ],

@@ -520,7 +520,8 @@ int asgd_eval(asgd_ctx* c, int32_t worker, double* E_host) {
   if (!small) eval_kernel<<<kEvalBlocks, EVAL_THREADS, smem, c->stream>>>(p.X, p.N, p.d, p.k, w, on_chip, partial);
   c->launches += 1;
   CU(c, cudaGetLastError());
-  std::vector<double> host(kEvalBlocks);
+  std::vector<double> host;
+  try { host.resize(kEvalBlocks); } catch (...) { return ASGD_ENOMEM; }
   CU(c, cudaMemcpyAsync(host.data(), partial, sizeof(double) * kEvalBlocks, cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
   double E = 0.0;

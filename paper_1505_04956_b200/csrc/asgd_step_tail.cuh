@@ -12,7 +12,7 @@ constexpr int MAX_FANOUT = 16;
 constexpr int MAX_SLOTS = 16;
 
 // Scratch every path reserves in shared memory for this tail.
-struct TailScratch {
+struct alignas(16) TailScratch {
   double red[96];
   int accept[MAX_SLOTS];
   int fresh[MAX_SLOTS];
@@ -21,6 +21,7 @@ struct TailScratch {
   int flag;
   int m;
 };
+static_assert(sizeof(TailScratch) % 16 == 0, "arrays placed behind the scratch keep their 16-byte alignment");
 
 // V floats at a time (V = 4: 128-bit accesses).
 template <int V> struct TailVec { float v[V]; };

@@ -88,8 +88,11 @@ def test_single_step_assignments_bit_exact(name):
             assert ((tr["d2"] - tr["d1"])[wrong] <= tau).all()
         else:
             assert (got[i][ok] == tr["assign"][ok]).all(), (name, i)
-            if ok.all():
-                assert np.bincount(got[i], minlength=wl.k).tolist() == tr["counts"].tolist()
+            # counts n_k of Eq. 9: equal to the oracle's per centre, up to the undecided rows either side gave it
+            und = ~ok
+            slack = np.bincount(got[i][und], minlength=wl.k) + np.bincount(tr["assign"][und], minlength=wl.k)
+            diff = np.abs(np.bincount(got[i], minlength=wl.k) - tr["counts"])
+            assert (diff <= slack).all(), (name, i, diff, slack)
         checked += int(ok.sum())
     assert checked >= 0.99 * wl.W * wl.b
     assert pr.max_rel_l2() < pr.centre_tol()

@@ -391,6 +391,37 @@ def test_communication_pulls_workers_together():
             assert spread(o) == pytest.approx(s0)
 
 
+@pytest.mark.parametrize("partial_rows", [0, 2])
+def test_round_loop_on_several_threads_is_bit_identical_to_one_thread(partial_rows):
+    # Algorithm 5: within a round a worker touches only its own state and its own receive buffers (the puts are
+    # delivered after the round), so running the workers of a round on n threads must change nothing at all:
+    # states, traces of the last step, counters and buffer contents, with communication switched on.
+    rng = np.random.default_rng(11)
+    W, k, d, b = 12, 5, 4, 16
+    mu = rng.uniform(-4, 4, size=(k, d))
+    X = (mu[rng.integers(0, k, W * b * 6 + 3)] + rng.normal(size=(W * b * 6 + 3, d))).astype(np.float32)
+    w0 = X[rng.choice(X.shape[0], k, replace=False)].copy()
+    kw = dict(W=W, b=b, eps=0.2, comm_interval=1, fanout=2, slots=2, seed=5, partial_rows=partial_rows)
+    one = orc.Oracle(X, w0, threads=1, **kw)
+    many = orc.Oracle(X, w0, threads=min(4, orc.max_threads()), **kw)
+    if many.threads < 2:
+        pytest.skip("the oracle was built without a parallel round loop")
+    for T in (1, 7, 13):
+        one.rounds(T)
+        many.rounds(T)
+        assert np.array_equal(one.states(), many.states())
+        for i in range(W):
+            assert one.stats(i) == many.stats(i)
+            a, m = one.last_step(i), many.last_step(i)
+            for key in a:
+                assert np.array_equal(a[key], m[key]), (T, i, key)
+            for s in range(2):
+                va, m_seq, m_seen = one.mail(i, s)
+                vb, n_seq, n_seen = many.mail(i, s)
+                assert np.array_equal(va, vb) and (m_seq, m_seen) == (n_seq, n_seen)
+    assert sum(one.stats(i)["accepted"] for i in range(W)) > 0        # messages did flow and were merged
+
+
 # ---------------------------------------------------------------------------------------------
 # Per-centre messages (Section 4.4): a put carries some of the centre rows; lambda, delta and the
 # merge are taken row by row.

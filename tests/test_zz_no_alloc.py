@@ -11,6 +11,7 @@ import torch
 
 import paper_1505_04956_b200 as pkg
 from paper_1505_04956_b200 import binding, inputs
+from oracle import asgd_oracle as orc
 
 pytestmark = pytest.mark.gpu
 REL_TOL = 1e-5          # the tolerance the evaluation tests use against the oracle
@@ -33,6 +34,9 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     want = ctx.eval(0)
     got = float(E.cpu())
     assert abs(got - want) <= REL_TOL * want, (got, want)
+    Xh = X.cpu().numpy()
+    truth = orc.quantization_error(Xh, w0.cpu().numpy())     # Eq. 8 by the CPU oracle on the copied buffer
+    assert abs(got - truth) <= REL_TOL * truth, (got, truth)
     # second call right after, other centres: the shared scratch still holds the first call's sums
     ctx.step(25)
     w1 = ctx.get_state(0)
@@ -40,11 +44,13 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point():
     want1 = ctx.eval(0)
     got1 = float(E.cpu())
     assert abs(got1 - want1) <= REL_TOL * want1, (got1, want1)
+    truth1 = orc.quantization_error(Xh, w1.cpu().numpy())
+    assert abs(got1 - truth1) <= REL_TOL * truth1, (got1, truth1)
     assert got1 < got                                        # 25 rounds of descent did lower the error
     # fewer rows than before: entries left over from the longer call must not leak into the sum
     Xs = X[:70_000]
     assert pkg.asgd_eval_noalloc(Xs, w1, E) == binding.ASGD_OK
-    ref = 0.5 * torch.cdist(Xs.double(), w1.double()).min(dim=1).values.pow(2).sum().item()
+    ref = orc.quantization_error(Xh[:70_000], w1.cpu().numpy())
     assert abs(float(E.cpu()) - ref) <= REL_TOL * ref
     ctx.destroy()
 
