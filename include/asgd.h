@@ -153,6 +153,17 @@ int asgd_get_accept(asgd_ctx *ctx, int32_t worker, int32_t *out_host /* HOST [S]
  * gave up a bounded wait on one of its own copies).  Housekeeping of this library: the paper has no
  * counterpart (its workers never wait, Section 1.2; neither do these, on one another). */
 int asgd_sync(asgd_ctx *ctx);
+/*
+ * Failure drill for the bounded waits (no counterpart in the paper).  A worker kernel waits only for its
+ * own asynchronous copies of samples, and gives each wait up after `wait_limit` polls (default 2^22):
+ * the block then raises the device status word, gives the copies it still has in flight the same bounded
+ * chance to land, releases what it holds and returns, so the context stays usable and asgd_sync() reports
+ * ASGD_ETIMEOUT.  With withhold_step = s >= 0 the first sample copy of step s of every following launch
+ * (counted from the launch's first step) is announced to its barrier but never issued, which makes that
+ * wait run out without any fault; -1 switches the drill off.  The generic kernel has no such waits.
+ * Affects launches made after the call.  ASGD_EINVAL for a NULL context or wait_limit = 0.
+ */
+int asgd_set_wait_drill(asgd_ctx *ctx, uint32_t wait_limit, int64_t withhold_step);
 /* Number of kernels this context has launched so far. */
 int64_t asgd_launch_count(const asgd_ctx *ctx);
 /* Name of the distance path the context resolved to ("fp32-generic", "fp32-stream", ...). */

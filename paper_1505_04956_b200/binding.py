@@ -17,7 +17,7 @@ PATH_AUTO, PATH_FP32, PATH_TC_3XTF32, PATH_TC_BF16, PATH_FP32_GENERAL = 0, 1, 2,
 EXPORTS = (
     "asgd_workspace_bytes", "asgd_init", "asgd_step", "asgd_run", "asgd_get_state", "asgd_set_state",
     "asgd_put", "asgd_put_rows", "asgd_get_accept_rows", "asgd_eval", "asgd_get_stats", "asgd_get_assign", "asgd_get_accept", "asgd_sync",
-    "asgd_launch_count", "asgd_path_name", "asgd_last_cuda_error", "asgd_strerror", "asgd_destroy",
+    "asgd_set_wait_drill", "asgd_launch_count", "asgd_path_name", "asgd_last_cuda_error", "asgd_strerror", "asgd_destroy",
     "asgd_fit_host_bytes", "asgd_fit_host", "asgd_eval_noalloc",
 )
 
@@ -69,6 +69,7 @@ def load():
     L.asgd_get_assign.argtypes = [vp, vp]
     L.asgd_get_accept.argtypes = [vp, i32, C.POINTER(C.c_int32)]
     L.asgd_sync.argtypes = [vp]
+    L.asgd_set_wait_drill.argtypes = [vp, C.c_uint32, i64]
     L.asgd_launch_count.argtypes = [vp]
     L.asgd_launch_count.restype = i64
     L.asgd_path_name.argtypes = [vp]
@@ -222,6 +223,9 @@ class Asgd:
 
     def sync(self):
         self._chk(self._L.asgd_sync(self._h), "asgd_sync")
+
+    def set_wait_drill(self, wait_limit: int, withhold_step: int = -1):
+        self._chk(self._L.asgd_set_wait_drill(self._h, int(wait_limit), int(withhold_step)), "asgd_set_wait_drill")
 
     def launch_count(self) -> int:
         return int(self._L.asgd_launch_count(self._h))

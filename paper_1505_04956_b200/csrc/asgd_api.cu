@@ -391,6 +391,8 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   p.rowin = (unsigned*)(c->ws + L.rowin);
   p.gsum = (float*)(c->ws + L.gsum);
   p.xmax2 = 0.f;
+  p.wait_limit = DEFAULT_WAIT_LIMIT;
+  p.withhold_step = -1;
   p.wbf = nullptr;
   p.top2 = nullptr;
 
@@ -573,6 +575,13 @@ int asgd_sync(asgd_ctx* c) {
   CU(c, cudaMemcpyAsync(st, c->p.status, sizeof(st), cudaMemcpyDeviceToHost, c->stream));
   CU(c, cudaStreamSynchronize(c->stream));
   if (st[0] == DEV_TIMEOUT) return ASGD_ETIMEOUT;
+  return ASGD_OK;
+}
+
+int asgd_set_wait_drill(asgd_ctx* c, uint32_t wait_limit, int64_t withhold_step) {
+  if (!c || wait_limit == 0) return ASGD_EINVAL;
+  c->p.wait_limit = wait_limit;
+  c->p.withhold_step = withhold_step < 0 ? -1 : withhold_step;
   return ASGD_OK;
 }
 

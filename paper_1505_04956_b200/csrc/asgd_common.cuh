@@ -41,6 +41,8 @@ struct Params {
   int2* mail_rows;         // [W][S] (first row, number of rows) of the buffer's last message (per-centre mode)
   unsigned* rowacc;        // [W][k] bit s: row accepted from buffer s in the worker's last step (per-centre mode)
   unsigned* rowin;         // [W][k] bit s: buffer s held a new message carrying the row
+  unsigned wait_limit;     // iterations of try_wait after which a wait on one of the block's own copies is given up
+  long long withhold_step; // failure drill: the first sample copy of this step of a launch is announced but not issued (-1 = never)
 };
 
 // ---------------------------------------------------------------------------------------------

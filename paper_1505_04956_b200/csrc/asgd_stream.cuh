@@ -31,7 +31,7 @@ constexpr int STREAM_SPT = 4;                          // samples per thread = 3
 constexpr int STREAM_MAX_B = STREAM_THREADS * STREAM_SPT;
 constexpr int STREAM_WARP_SAMPLES = 32 * STREAM_SPT;
 constexpr int STREAM_GROUP = 8;                        // rows of one centre added by one lane
-constexpr unsigned STREAM_WAIT_LIMIT = 1u << 22;       // bounded mbarrier wait (iterations of try_wait)
+constexpr unsigned DEFAULT_WAIT_LIMIT = 1u << 22;      // bounded mbarrier wait (iterations of try_wait), Params::wait_limit
 
 __device__ inline unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
 __device__ inline void mbar_init(unsigned long long* bar, unsigned count) {
@@ -48,8 +48,8 @@ __device__ inline bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
   return ok != 0;
 }
 // Returns false when the wait ran out (the caller reports it and leaves).
-__device__ inline bool mbar_wait_bounded(unsigned long long* bar, unsigned parity) {
-  for (unsigned it = 0; it < STREAM_WAIT_LIMIT; ++it)
+__device__ inline bool mbar_wait_bounded(unsigned long long* bar, unsigned parity, unsigned limit) {
+  for (unsigned it = 0; it < limit; ++it)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
@@ -228,12 +228,12 @@ asgd_stream_kernel(const Params p, const long long steps) {
     bytes = (head + batch_bytes + 15u) & ~15u;
     return src - head;
   };
-  auto issue = [&](int batch, int slot) {
+  auto issue = [&](int batch, int slot, long long s) {   // s: the step of this launch that uses the batch
     unsigned head, bytes;
     const unsigned char* src = tile_src(batch, head, bytes);
     if (src + bytes <= Xend) {
       mbar_expect_tx(bars + slot, bytes);
-      bulk_g2s(ring + (size_t)slot * slot_bytes, src, bytes, bars + slot);
+      if (s != p.withhold_step) bulk_g2s(ring + (size_t)slot * slot_bytes, src, bytes, bars + slot);
     } else {
       mbar_expect_tx(bars + slot, 0);       // phase completes at once; consumers load the tile themselves
     }
@@ -244,8 +244,8 @@ asgd_stream_kernel(const Params p, const long long steps) {
   int batch_cur = myperm[pos];
   int batch_nxt = myperm[pos1];
   if (tid == 0 && steps > 0) {
-    issue(batch_cur, 0);
-    if (steps > 1) issue(batch_nxt, 1);
+    issue(batch_cur, 0, 0);
+    if (steps > 1) issue(batch_nxt, 1, 1);
   }
   __syncthreads();
 
@@ -300,7 +300,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
     unsigned head, bytes;
     const unsigned char* src = tile_src(batch, head, bytes);
     unsigned char* tile = ring + (size_t)(s & 1) * slot_bytes;
-    if (!mbar_wait_bounded(bars + (s & 1), (unsigned)((s >> 1) & 1))) abort = 1;
+    if (!mbar_wait_bounded(bars + (s & 1), (unsigned)((s >> 1) & 1), p.wait_limit)) abort = 1;
     if (src + bytes > Xend) {
       // last rows of X: a rounded bulk copy would run past the array, use plain loads
       const float* g = reinterpret_cast<const float*>(src + head);
@@ -487,7 +487,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
     // the slot's rows have been added: start the copy of the batch after the next into it
     if (tid == 0 && step + 2 < steps) {
       fence_proxy_async_smem();
-      issue(batch_nn, slot);
+      issue(batch_nn, slot, step + 2);
     }
     const bool put_now = (to_put == 1);
     if (flags[0] != 0) {
@@ -561,8 +561,8 @@ asgd_stream_kernel(const Params p, const long long steps) {
     if (tid == 0) atomicExch(p.status, DEV_TIMEOUT);
     // a copy may still be in flight into this block's shared memory: give it a bounded chance to land
     for (int q = 0; q < STREAM_STAGES; ++q) {
-      mbar_wait_bounded(bars + q, 0);
-      mbar_wait_bounded(bars + q, 1);
+      mbar_wait_bounded(bars + q, 0, p.wait_limit);
+      mbar_wait_bounded(bars + q, 1, p.wait_limit);
     }
   }
 }

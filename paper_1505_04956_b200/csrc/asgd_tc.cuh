@@ -203,17 +203,18 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         for (int m = 0; m < m_tiles && ok; ++m, ++um) {
           const int halves = min(TC_MH, (b - m * TC_MH * TC_M + TC_M - 1) / TC_M);
           for (int kc = 0; kc < nkc && ok; ++kc) {
-            if (um > 0) ok = mbar_wait_bounded(bars + TCB_AEMPTY + kc, (um - 1) & 1);     // last use of the chunk by the previous tile
+            if (um > 0) ok = mbar_wait_bounded(bars + TCB_AEMPTY + kc, (um - 1) & 1, p.wait_limit);     // last use of the chunk by the previous tile
             if (!ok) break;
             mbar_expect_tx(bars + TCB_AFULL + kc, (unsigned)(halves * TC_A_STAGE_BYTES));
-            for (int h = 0; h < halves; ++h)
+            const bool withheld = (m == 0 && kc == 0 && step == p.withhold_step);   // failure drill: announced, never copied
+            for (int h = 0; h < halves && !withheld; ++h)
               tma_load_2d(sA + (size_t)(kc * TC_MH + h) * TC_A_STAGE_BYTES, &mapX, kc * TC_KC,
                           (int)(row0 + (long long)(m * TC_MH + h) * TC_M), bars + TCB_AFULL + kc);
           }
           for (int n = 0; n < n_tiles && ok; ++n) {
             for (int g = 0; g < ngr; ++g, ++ibc) {
               const int st = ibc % TC_B_STAGES;
-              if (ibc >= TC_B_STAGES) ok = mbar_wait_bounded(bars + TCB_BEMPTY + st, ((ibc / TC_B_STAGES) - 1) & 1);
+              if (ibc >= TC_B_STAGES) ok = mbar_wait_bounded(bars + TCB_BEMPTY + st, ((ibc / TC_B_STAGES) - 1) & 1, p.wait_limit);
               if (!ok) break;
               const int cnt_kc = min(TC_BG, nkc - g * TC_BG);
               mbar_expect_tx(bars + TCB_BFULL + st, (unsigned)(cnt_kc * TC_B_CHUNK_BYTES));
@@ -233,15 +234,15 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           const int halves = min(TC_MH, (b - m * TC_MH * TC_M + TC_M - 1) / TC_M);
           for (int n = 0; n < n_tiles && ok; ++n, ++iacc) {
             const int buf = iacc & 1;
-            if (iacc >= 2) ok = mbar_wait_bounded(bars + TCB_ACCEMPTY + buf, ((iacc >> 1) - 1) & 1);
+            if (iacc >= 2) ok = mbar_wait_bounded(bars + TCB_ACCEMPTY + buf, ((iacc >> 1) - 1) & 1, p.wait_limit);
             if (!ok) break;
             tc_fence_after();
             for (int g = 0; g < ngr && ok; ++g, ++ibc) {
               const int st = ibc % TC_B_STAGES;
               const int cnt_kc = min(TC_BG, nkc - g * TC_BG);
               if (n == 0)
-                for (int c = 0; c < cnt_kc && ok; ++c) ok = mbar_wait_bounded(bars + TCB_AFULL + g * TC_BG + c, um & 1);
-              if (ok) ok = mbar_wait_bounded(bars + TCB_BFULL + st, (ibc / TC_B_STAGES) & 1);
+                for (int c = 0; c < cnt_kc && ok; ++c) ok = mbar_wait_bounded(bars + TCB_AFULL + g * TC_BG + c, um & 1, p.wait_limit);
+              if (ok) ok = mbar_wait_bounded(bars + TCB_BFULL + st, (ibc / TC_B_STAGES) & 1, p.wait_limit);
               if (!ok) break;
               tc_fence_after();
               for (int c = 0; c < cnt_kc; ++c) {
@@ -278,7 +279,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         for (int h = 0; h < TC_MH; ++h) { m1[h][0] = m1[h][1] = INF; m2[h][0] = m2[h][1] = INF; }
         for (int n = 0; n < n_tiles; ++n, ++iacc) {
           const int buf = iacc & 1;
-          if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bars + TCB_ACCFULL + buf, (iacc >> 1) & 1));
+          if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bars + TCB_ACCFULL + buf, (iacc >> 1) & 1, p.wait_limit));
           if (!ok) continue;
           tc_fence_after();
 #pragma unroll 1
@@ -593,7 +594,12 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     __syncthreads();
   }
 
-  if (misc[2] && tid == 0) atomicExch(p.status, DEV_TIMEOUT);
+  if (misc[2] && tid == 0) {
+    atomicExch(p.status, DEV_TIMEOUT);
+    // copies may still be on their way into this block's shared memory: give each a bounded chance to land
+    for (int q = 0; q < TC_B_STAGES; ++q) { mbar_wait_bounded(bars + TCB_BFULL + q, 0, p.wait_limit); mbar_wait_bounded(bars + TCB_BFULL + q, 1, p.wait_limit); }
+    for (int q = 0; q < TC_A_STAGES; ++q) { mbar_wait_bounded(bars + TCB_AFULL + q, 0, p.wait_limit); mbar_wait_bounded(bars + TCB_AFULL + q, 1, p.wait_limit); }
+  }
   tc_fence_before();
   __syncthreads();
   if (wid == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");

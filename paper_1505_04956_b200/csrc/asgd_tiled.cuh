@@ -124,7 +124,8 @@ asgd_tiled_kernel(const Params p, const long long steps) {
     const float* src = p.X + ((size_t)i * p.H + (size_t)batch * b + (size_t)tl * TS) * D;
     if (lane == 0) mbar_expect_tx(bars + slot, (unsigned)rows * D * 4);
     __syncwarp();
-    if (lane < 4 * RB) {                              // one copy per quarter of every sub-tile
+    const bool withheld = (tl == 0 && v == 0 && nx_st == p.withhold_step);      // failure drill: announced, never copied
+    if (lane < 4 * RB && !withheld) {                 // one copy per quarter of every sub-tile
       const int first = (lane / 4) * TS0 + (lane % 4) * QR;          // the quarter's first row in the tile
       const int qrows = min(QR, rows - first);
       if (qrows > 0) bulk_g2s(dst + (size_t)lane * QS, src + (size_t)first * D, (unsigned)qrows * D * 4, bars + slot);
@@ -189,7 +190,7 @@ asgd_tiled_kernel(const Params p, const long long steps) {
         const float* xb = xt + (size_t)slot * RB * 4 * QS;
         auto xrowp = [&](int r) { return xb + (size_t)(r / QR) * QS + (size_t)(r % QR) * XS; };   // tile row r (quarters of all sub-tiles are QS apart)
         if (tid == 0) flagged[0] = 0;
-        if (!mbar_wait_bounded(bars + slot, parity)) abort = 1;
+        if (!mbar_wait_bounded(bars + slot, parity, p.wait_limit)) abort = 1;
 
         for (int rb = 0; rb < RB && rb * TS0 < rows; ++rb) {   // the tile's sub-tiles in turn (the same trip count for every thread)
           // ---- scores of the warp's 16 x 32 block: acc[m][i] = sum_j x[row m][j] * (-2 w[centre i][j]) ----
@@ -439,8 +440,8 @@ asgd_tiled_kernel(const Params p, const long long steps) {
 
   if (abort) {
     if (tid == 0) atomicExch(p.status, DEV_TIMEOUT);
-    mbar_wait_bounded(bars + 0, 0); mbar_wait_bounded(bars + 0, 1);
-    mbar_wait_bounded(bars + 1, 0); mbar_wait_bounded(bars + 1, 1);
+    mbar_wait_bounded(bars + 0, 0, p.wait_limit); mbar_wait_bounded(bars + 0, 1, p.wait_limit);
+    mbar_wait_bounded(bars + 1, 0, p.wait_limit); mbar_wait_bounded(bars + 1, 1, p.wait_limit);
   }
 }
 
