@@ -11,26 +11,31 @@
 // whose two best scores are closer than the rounding bound of this form is decided again in the
 // direct difference form.
 //
-// Per-centre sums (Eq. 9): each warp orders its 128 rows by the centre they chose (rank inside a
-// 32-row block from a match, so a centre's rows stay in row order; entries are byte offsets into the
-// tile).  A centre's run starts at a multiple of eight entries and its unused tail points at a row of
-// zeros kept behind the tile, so the order falls into groups of eight rows of one centre.  Lane g of
-// the same warp adds the eight rows of group g over all dimensions; the update adds a centre's group
-// sums in order.  The work per lane does not depend on how unevenly the centres are chosen, every sum
-// has a fixed order (a step is reproducible), and the plain local step needs two block-wide barriers.
+// Per-centre sums and counts (Eq. 9): S = X^T . onehot(s) is formed by the warp on the tensor cores
+// (mma.sync m16n8k8, TF32 operands, fp32 accumulators kept in registers over the warp's 128 rows).
+// The one-hot operand is exact; every sample value goes in as two terms, hi = x with the 13 low
+// mantissa bits cleared and lo = x - hi (exact in fp32; the tensor core keeps its leading bits), so a
+// value enters a sum with a relative error below 2^-21.  The sample fragments come straight from the
+// tile (a thread reads the dimension pair 2g, 2g+1 of rows 4 apart: 160 bytes for d = 10, which
+// spreads the four rows of an access over all banks).  The counts n_k come out of the same products:
+// the threads whose dimension pair lies past d read (1, 0) pairs instead of samples, which makes result
+// row d/2 the number of rows per centre (for d = 16, where no result row is spare, a third product with a
+// row of ones).  No row is gathered, nothing is sorted, and every sum has a fixed order (a step is
+// reproducible bit for bit).
 #pragma once
 
 #include "asgd_step_tail.cuh"
 
 namespace asgd {
 
-constexpr int STREAM_THREADS = 128;
-constexpr int STREAM_WARPS = STREAM_THREADS / 32;
-constexpr int STREAM_STAGES = 2;
 constexpr int STREAM_SPT = 4;                          // samples per thread = 32-row blocks per warp
-constexpr int STREAM_MAX_B = STREAM_THREADS * STREAM_SPT;
+constexpr int STREAM_MAX_B = 512;
 constexpr int STREAM_WARP_SAMPLES = 32 * STREAM_SPT;
-constexpr int STREAM_GROUP = 8;                        // rows of one centre added by one lane
+constexpr int STREAM_WARPS = (STREAM_MAX_B + STREAM_WARP_SAMPLES - 1) / STREAM_WARP_SAMPLES;
+constexpr int STREAM_THREADS = 32 * STREAM_WARPS;
+constexpr int STREAM_ROWS = STREAM_WARPS * STREAM_WARP_SAMPLES;   // rows the warps cover (>= the largest batch)
+constexpr int STREAM_STAGES = 2;
+constexpr int STREAM_KSTEPS = STREAM_WARP_SAMPLES / 8; // tensor-core products of 8 rows per warp and step
 constexpr unsigned DEFAULT_WAIT_LIMIT = 1u << 22;      // bounded mbarrier wait (iterations of try_wait), Params::wait_limit
 
 __device__ inline unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
@@ -69,106 +74,86 @@ __device__ inline unsigned ld_relaxed_gpu(const unsigned* p) {
   asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+// 1.0f where a == b, else 0.0f (one instruction)
+__device__ __forceinline__ unsigned onehot_bits(float a, float b) {
+  float r;
+  asm("set.eq.f32.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return __float_as_uint(r);
+}
+// C[16x8] += A[16x8] . B[8x8] on the tensor cores, TF32 operands, fp32 accumulate.  Thread (g = lane / 4, t = lane % 4)
+// holds A[g][t], A[g+8][t], A[g][t+4], A[g+8][t+4];  B[t][g], B[t+4][g];  C[g][2t], C[g][2t+1], C[g+8][2t], C[g+8][2t+1].
+__device__ __forceinline__ void mma_tf32_16x8x8(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0,
+                                                unsigned b1) {
+  asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 
-// Shared-memory accesses of the order and sum phases: 32-bit shared addresses with constant offsets, so that an
-// access costs one instruction and no 64-bit address arithmetic.
-template <int OFF> __device__ __forceinline__ unsigned lds_u32(unsigned a) {
-  unsigned v;
-  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(a), "n"(OFF) : "memory");
-  return v;
-}
-template <int OFF> __device__ __forceinline__ uint4 lds_v4(unsigned a) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a), "n"(OFF) : "memory");
-  return v;
-}
-template <int OFF> __device__ __forceinline__ float2 lds_f2(unsigned a) {
-  float2 v;
-  asm volatile("ld.shared.v2.f32 {%0,%1}, [%2+%3];" : "=f"(v.x), "=f"(v.y) : "r"(a), "n"(OFF) : "memory");
-  return v;
-}
-template <int OFF> __device__ __forceinline__ void sts_u32(unsigned a, unsigned v) {
-  asm volatile("st.shared.u32 [%0+%2], %1;" ::"r"(a), "r"(v), "n"(OFF) : "memory");
-}
-template <int OFF> __device__ __forceinline__ void sts_u32_if(unsigned a, unsigned v, unsigned on) {
-  asm volatile("{\n .reg .pred p;\n setp.ne.u32 p, %3, 0;\n @p st.shared.u32 [%0+%2], %1;\n}" ::"r"(a), "r"(v), "n"(OFF), "r"(on) : "memory");
-}
-template <int OFF> __device__ __forceinline__ void sts_v4(unsigned a, unsigned v) {
-  asm volatile("st.shared.v4.u32 [%0+%2], {%1,%1,%1,%1};" ::"r"(a), "r"(v), "n"(OFF) : "memory");
-}
-template <int OFF> __device__ __forceinline__ void sts_f2(unsigned a, float2 v) {
-  asm volatile("st.shared.v2.f32 [%0+%3], {%1,%2};" ::"r"(a), "f"(v.x), "f"(v.y), "n"(OFF) : "memory");
-}
-// running sum step: v += (value of the lane `o` below), lanes below `o` keep v
-__device__ __forceinline__ int scan_step(int v, int o) {
-  int r;
-  asm volatile("{\n .reg .pred p;\n .reg .b32 t;\n shfl.sync.up.b32 t|p, %1, %2, 0, 0xffffffff;\n @p add.s32 t, t, %1;\n @!p mov.b32 t, %1;\n mov.b32 %0, t;\n}" : "=r"(r) : "r"(v), "r"(o));
-  return r;
+// The same product started from C = 0.
+__device__ __forceinline__ void mma_tf32_16x8x8_first(float (&c)[4], unsigned a0, unsigned a1, unsigned a2, unsigned a3, unsigned b0,
+                                                      unsigned b1) {
+  asm("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+      : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.f));
 }
 
 constexpr size_t stream_up16(size_t x) { return (x + 15) / 16 * 16; }
 
 // Sizes and the shared-memory map of the streaming kernel.  Everything but the ring has a place that depends on
-// (d, k) only, so those byte offsets are constants in the code; the ring (whose slots depend on b) comes last.
+// (d, k) only, so those byte offsets are constants in the code; the ring comes last.
 template <int D, int K>
 struct StreamLayout {
   static_assert(D % 2 == 0 && D <= 16 && K <= 16, "streaming path: even d <= 16, k <= 16");
-  static constexpr int DP = (D + 3) / 4 * 4;        // padded row of -2w for 128-bit loads
+  static constexpr int DP = (D + 2 + 3) / 4 * 4;    // row of -2w, then (||w_a||^2, 0), padded for 128-bit loads
   static constexpr int D2 = D / 2;                  // dimension pairs
   static constexpr int INDEX_BITS = (K <= 2) ? 1 : (K <= 4) ? 2 : (K <= 8) ? 3 : 4;
   static constexpr unsigned INDEX_MASK = (1u << INDEX_BITS) - 1u;
   static constexpr int ROWB = D * 4;                // bytes per sample
-  static constexpr int CWS = (K + 1 + 3) / 4 * 4;   // a warp's counts per centre, one spare counter for rows past the batch
-  static constexpr int GPR = 32 / D2;               // groups a warp adds at a time: lanes (group, dimension pair)
-  static constexpr int CPW = GPR;                   // centres a warp updates: lanes (centre, dimension pair)
+  static constexpr int NT = (K + 1 + 7) / 8;        // blocks of 8 one-hot columns: centres 0..K-1 and the spare index K of rows past the batch
+  static constexpr int CPW = 32 / D2;               // centres a warp updates: lanes (centre, dimension pair)
   static constexpr int UPD_WARPS = (K + CPW - 1) / CPW;
   static_assert(UPD_WARPS <= STREAM_WARPS, "update: every centre has a warp");
-  // a warp's rows ordered by centre, every centre's run padded to whole groups of eight
-  static constexpr int NGRP = (STREAM_WARP_SAMPLES + (STREAM_GROUP - 1) * K + STREAM_GROUP - 1) / STREAM_GROUP;
-  static constexpr int GCAP = (NGRP + 2 * GPR - 1) / (2 * GPR) * (2 * GPR);   // groups the adders may touch (whole double rounds)
-  static_assert(NGRP <= 32, "a running sum over one warp covers the groups");
+  static constexpr int BEST_RUN = 160;              // bytes between the four runs of the best-centre table (128 used; 160 spreads them over the banks)
 
   // fixed part of the map (byte offsets)
   static constexpr size_t BARS = 0;
   static constexpr size_t FLAGS = 64;
-  static constexpr size_t ZROW = 128;                                    // a row of zeros for the unused tail of a group
-  static constexpr size_t TAIL = ZROW + stream_up16(ROWB + 16);
+  static constexpr size_t WMAX = 96;                                    // max_a ||w_a||^2 as found by each updating warp
+  static constexpr size_t TAIL = 128;
   static constexpr size_t WNEG2 = TAIL + stream_up16(sizeof(TailScratch));
-  static constexpr size_t CNORM = WNEG2 + stream_up16((size_t)K * DP * 4);   // (||w_a||^2, 0) pairs
-  static constexpr size_t W = CNORM + stream_up16((size_t)K * 8);
+  static constexpr size_t W = WNEG2 + stream_up16((size_t)K * DP * 4);
   static constexpr size_t SD = W + stream_up16((size_t)K * D * 4);
   static constexpr size_t CNT = SD + stream_up16((size_t)K * D * 4);
   static constexpr size_t SEEN = CNT + stream_up16((size_t)K * 4);
   static constexpr size_t WARP0 = SEEN + stream_up16((size_t)MAX_SLOTS * 4);
-  // per warp: rows per (32-row block, centre); rows per centre; first group per centre; the order; the group sums
-  static constexpr size_t W_CQ = 0;
-  static constexpr size_t W_CW = W_CQ + (size_t)STREAM_SPT * CWS * 4;
-  static constexpr size_t W_FIRST = W_CW + (size_t)CWS * 4;
-  static constexpr size_t W_ORDER = W_FIRST + (size_t)CWS * 4;           // u32 shared addresses of rows
-  static constexpr size_t W_GSUM = W_ORDER + (size_t)GCAP * STREAM_GROUP * 4;
-  static constexpr size_t WARP_STRIDE = stream_up16(W_GSUM + (size_t)GCAP * D * 4);
-  static constexpr size_t RING = (WARP0 + STREAM_WARPS * WARP_STRIDE + 127) / 128 * 128;
-  // a ring slot: the batch with its source rounded out to 16-byte bounds
-  __host__ __device__ static size_t slot_bytes(int b) { return ((size_t)b * ROWB + 32 + 127) / 128 * 128; }
-  __host__ __device__ static size_t total(int b) { return RING + STREAM_STAGES * slot_bytes(b); }
+  // per warp: the best centre of its rows in the order the one-hot operand reads them; its sums [K][D]; its counts [K]
+  static constexpr size_t W_BEST = 0;
+  static constexpr size_t W_SUM = W_BEST + 4 * BEST_RUN;
+  static constexpr size_t W_CNT = W_SUM + stream_up16((size_t)K * D * 4);
+  static constexpr size_t WARP_STRIDE = stream_up16(W_CNT + (size_t)K * 4);
+  static constexpr size_t ONES = (WARP0 + STREAM_WARPS * WARP_STRIDE + 15) / 16 * 16;   // (1, 0) pairs: the rows of ones of the counts
+  static constexpr size_t ONES_BYTES = (size_t)STREAM_WARP_SAMPLES * ROWB + 16;
+  static constexpr size_t RING = (ONES + ONES_BYTES + 127) / 128 * 128;
+  // a ring slot: up to 15 bytes in front of the batch (its source is rounded out to 16-byte bounds), room for the
+  // rows of a full block (the tensor-core sums read all of them; rows past the batch hold old or zero data and
+  // count for no centre) and for the dimension pairs past d that the last rows' fragments touch
+  static constexpr size_t SLOT = ((size_t)16 + (size_t)STREAM_ROWS * ROWB + 64 + 127) / 128 * 128;
+  static constexpr size_t TOTAL = RING + STREAM_STAGES * SLOT;
 };
 template <int D, int K>
-inline size_t stream_smem_bytes(int b) { return StreamLayout<D, K>::total(b); }
+inline size_t stream_smem_bytes(int /*b*/) { return StreamLayout<D, K>::TOTAL; }
 
 template <int D, int K, bool kDet>
 __global__ void __launch_bounds__(STREAM_THREADS, 4)
 asgd_stream_kernel(const Params p, const long long steps) {
   using L = StreamLayout<D, K>;
-  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, ROWB = L::ROWB, CWS = L::CWS, GCAP = L::GCAP, GPR = L::GPR;
+  constexpr int DP = L::DP, D2 = L::D2, KD = K * D, ROWB = L::ROWB, NT = L::NT;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   const int b = p.b;
-  const unsigned slot_bytes = (unsigned)L::slot_bytes(b);
   unsigned char* ring = smem_raw + L::RING;
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem_raw + L::BARS);   // [STAGES]
   int* flags = reinterpret_cast<int*>(smem_raw + L::FLAGS);                               // [0] a buffer has news
+  float* wmaxs = reinterpret_cast<float*>(smem_raw + L::WMAX);                            // [UPD_WARPS]
   TailScratch* ts = reinterpret_cast<TailScratch*>(smem_raw + L::TAIL);
   float* wneg2 = reinterpret_cast<float*>(smem_raw + L::WNEG2);
-  float2* cnorm = reinterpret_cast<float2*>(smem_raw + L::CNORM);
   float* w = reinterpret_cast<float*>(smem_raw + L::W);
   float* SD = reinterpret_cast<float*>(smem_raw + L::SD);
   int* cnt = reinterpret_cast<int*>(smem_raw + L::CNT);
@@ -182,15 +167,18 @@ asgd_stream_kernel(const Params p, const long long steps) {
   const unsigned batch_bytes = (unsigned)b * D * 4;
   const float inv_b = 1.0f / (float)b;
   const float eps = p.eps;
-  // shared addresses (32 bit): the block's base, this warp's arrays, the row of zeros
-  const unsigned sbase = smem_u32(smem_raw);
-  const unsigned wb = sbase + (unsigned)L::WARP0 + (unsigned)wid * (unsigned)L::WARP_STRIDE;
-  const unsigned zrow = sbase + (unsigned)L::ZROW;
   auto warp_ptr = [&](int q, size_t off) { return smem_raw + L::WARP0 + (size_t)q * L::WARP_STRIDE + off; };
+  const bool warp_on = wid * STREAM_WARP_SAMPLES < b;                   // warps whose rows all lie past the batch sit a step out
 
-  // state on chip: w, -2w (padded rows), (||w_a||^2, 0)
+  // state on chip: w, -2w (padded rows), (||w_a||^2, 0); ring and per-warp sums start at zero (rows past the batch
+  // and idle warps must read finite numbers)
   for (int e = tid; e < K * DP; e += STREAM_THREADS) wneg2[e] = 0.f;
-  for (int e = tid; e < (ROWB + 16) / 4; e += STREAM_THREADS) reinterpret_cast<float*>(smem_raw + L::ZROW)[e] = 0.f;
+  for (size_t e = tid; e < STREAM_STAGES * L::SLOT / 16; e += STREAM_THREADS)
+    reinterpret_cast<float4*>(ring)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (size_t e = tid; e < STREAM_WARPS * L::WARP_STRIDE / 4; e += STREAM_THREADS)
+    reinterpret_cast<float*>(smem_raw + L::WARP0)[e] = 0.f;
+  for (size_t e = tid; e < L::ONES_BYTES / 8; e += STREAM_THREADS)
+    reinterpret_cast<float2*>(smem_raw + L::ONES)[e] = make_float2(1.f, 0.f);
   __syncthreads();
   for (int e = tid; e < KD; e += STREAM_THREADS) {
     const float v = wglob[e];
@@ -209,8 +197,15 @@ asgd_stream_kernel(const Params p, const long long steps) {
     float s = 0.f;
 #pragma unroll
     for (int j = 0; j < D; ++j) s = fmaf(w[tid * D + j], w[tid * D + j], s);
-    cnorm[tid] = make_float2(s, 0.f);
+    wneg2[tid * DP + D] = s;
   }
+  __syncthreads();
+  if (tid < L::UPD_WARPS) {
+    float m = 0.f;
+    for (int a = 0; a < K; ++a) m = fmaxf(m, wneg2[a * DP + D]);
+    wmaxs[tid] = m;
+  }
+  fence_proxy_async_smem();                                              // the zeroed ring is written by bulk copies next
 
   unsigned long long t = p.stats[(size_t)i * ST_STRIDE + ST_STEPS];
   // 32-bit running positions: place in the batch order, steps left until the next put
@@ -233,7 +228,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
     const unsigned char* src = tile_src(batch, head, bytes);
     if (src + bytes <= Xend) {
       mbar_expect_tx(bars + slot, bytes);
-      if (s != p.withhold_step) bulk_g2s(ring + (size_t)slot * slot_bytes, src, bytes, bars + slot);
+      if (s != p.withhold_step) bulk_g2s(ring + (size_t)slot * L::SLOT, src, bytes, bars + slot);
     } else {
       mbar_expect_tx(bars + slot, 0);       // phase completes at once; consumers load the tile themselves
     }
@@ -243,79 +238,70 @@ asgd_stream_kernel(const Params p, const long long steps) {
   int pos1 = next_pos(pos);
   int batch_cur = myperm[pos];
   int batch_nxt = myperm[pos1];
+  __syncthreads();
   if (tid == 0 && steps > 0) {
     issue(batch_cur, 0, 0);
     if (steps > 1) issue(batch_nxt, 1, 1);
   }
-  __syncthreads();
 
   const float tau_scale = (float)(4 * D + 72) * 5.9604645e-8f;
   const float xmax2 = p.xmax2;                                              // max ||x||^2 over the samples
-  const unsigned lane_lt = (1u << lane) - 1u;
-  const int lane_c = min(lane, K);                                         // lanes past the centres share the spare column
-  const unsigned row0 = (unsigned)((wid * STREAM_WARP_SAMPLES + lane) * ROWB);   // this thread's first row in a tile
 
-  // total of centre a, dimension pair jp over the warps' groups, in a fixed order
+  // tensor-core fragments: thread (g, t4) reads the dimension pair (2g, 2g+1) of rows 4*t4 + 16*block + r of the
+  // warp's rows; for g >= d/2 it reads past the row (finite numbers of the next rows) into result rows nobody uses
+  const int g = lane >> 2, t4 = lane & 3;
+  const unsigned frag_off = (unsigned)((wid * STREAM_WARP_SAMPLES + 4 * t4) * ROWB + 8 * g);
+  // the best centre of row 32*q + lane goes to run (lane % 16) / 4, entry 8*q + 4*(lane / 16) + lane % 4, so that
+  // thread (g, t4) finds the rows of its products, two rows per product, in order in run t4
+  float* best_w = reinterpret_cast<float*>(warp_ptr(wid, L::W_BEST) + ((lane & 15) >> 2) * L::BEST_RUN) + 4 * (lane >> 4) + (lane & 3);
+  const float4* best_r = reinterpret_cast<const float4*>(warp_ptr(wid, L::W_BEST) + t4 * L::BEST_RUN);
+  const float2 neg1 = make_float2(-1.f, -1.f);
+  float cg[NT];                                                            // this thread's one-hot columns (centres g, 8 + g)
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) cg[nt] = (float)(8 * nt + g);
+
+  // total of centre a, dimension pair jp over the warps, in a fixed order
   auto centre_sum = [&](int a, int jp) {
-    constexpr int AHEAD = 4;                         // groups of a (warp, centre) whose loads are issued at once
     float2 part[STREAM_WARPS];
 #pragma unroll
-    for (int q = 0; q < STREAM_WARPS; ++q) {
-      const int* first = reinterpret_cast<const int*>(warp_ptr(q, L::W_FIRST));
-      const float2* gs = reinterpret_cast<const float2*>(warp_ptr(q, L::W_GSUM));
-      const int g0 = first[a], ng = first[a + 1] - g0;
-      const float2* src = gs + (size_t)g0 * D2 + jp;
-      float2 v[AHEAD];
+    for (int q = 0; q < STREAM_WARPS; ++q) part[q] = reinterpret_cast<const float2*>(warp_ptr(q, L::W_SUM))[a * D2 + jp];
+    float2 tot = part[0];
 #pragma unroll
-      for (int u = 0; u < AHEAD; ++u) v[u] = (u < ng) ? src[u * D2] : make_float2(0.f, 0.f);
-      part[q] = __fadd2_rn(__fadd2_rn(v[0], v[1]), __fadd2_rn(v[2], v[3]));
-      for (int u = AHEAD; u < ng; ++u) part[q] = __fadd2_rn(part[q], src[u * D2]);
-    }
-    return __fadd2_rn(__fadd2_rn(part[0], part[1]), __fadd2_rn(part[2], part[3]));
+    for (int q = 1; q < STREAM_WARPS; ++q) tot = __fadd2_rn(tot, part[q]);
+    return tot;
   };
   auto centre_rows = [&](int a) {
-    int n = 0;
+    float n = 0.f;
 #pragma unroll
-    for (int q = 0; q < STREAM_WARPS; ++q) n += reinterpret_cast<const int*>(warp_ptr(q, L::W_CW))[a];
-    return n;
+    for (int q = 0; q < STREAM_WARPS; ++q) n += reinterpret_cast<const float*>(warp_ptr(q, L::W_CNT))[a];
+    return n;                                                              // whole numbers up to 512: exact
   };
 
   int abort = 0;
-  // A step's samples: the thread's rows of the batch in registers, the tile's shared address for the sums.
+  // A step's samples: the thread's rows of the batch in registers, the tile's place for the sums.
   float2 xv[STREAM_SPT][D2];
-  unsigned xsa = 0;
-  // Gets batch `batch` (the one of step `s`) ready: resets this warp's order and counts, waits for the copy
-  // and loads the thread's rows.  Runs between the two barriers of the step before, beside the update.
+  const unsigned char* xtile = ring;
+  // Gets batch `batch` (the one of step `s`) ready: waits for the copy and loads the thread's rows.  Runs between
+  // the two barriers of the step before, beside the update.
   auto stage_in = [&](long long s, int batch) {
-    {
-      // this warp's order: every entry points at the row of zeros; counts zero
-#pragma unroll
-      for (int e = 0; e < (GCAP * STREAM_GROUP / 4 + 31) / 32; ++e)
-        if (e * 32 + lane < GCAP * STREAM_GROUP / 4) {
-          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(wb + (unsigned)L::W_ORDER + (unsigned)(e * 32 + lane) * 16u), "r"(zrow) : "memory");
-        }
-      if (lane < STREAM_SPT * CWS / 4)
-        asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(wb + (unsigned)L::W_CQ + (unsigned)lane * 16u), "r"(0u) : "memory");
-    }
     unsigned head, bytes;
     const unsigned char* src = tile_src(batch, head, bytes);
-    unsigned char* tile = ring + (size_t)(s & 1) * slot_bytes;
+    unsigned char* tile = ring + (size_t)(s & 1) * L::SLOT;
     if (!mbar_wait_bounded(bars + (s & 1), (unsigned)((s >> 1) & 1), p.wait_limit)) abort = 1;
     if (src + bytes > Xend) {
       // last rows of X: a rounded bulk copy would run past the array, use plain loads
-      const float* g = reinterpret_cast<const float*>(src + head);
+      const float* gx = reinterpret_cast<const float*>(src + head);
       float* sdst = reinterpret_cast<float*>(tile + head);
-      for (int e = tid; e < b * D; e += STREAM_THREADS) sdst[e] = __ldg(g + e);
+      for (int e = tid; e < b * D; e += STREAM_THREADS) sdst[e] = __ldg(gx + e);
       __syncthreads();
     }
-    const float* xs = reinterpret_cast<const float*>(tile + head);
-    xsa = smem_u32(xs);
+    xtile = tile + head;
+    if (warp_on) {
+      const float2* xrow = reinterpret_cast<const float2*>(xtile + (size_t)(wid * STREAM_WARP_SAMPLES + lane) * ROWB);
 #pragma unroll
-    for (int q = 0; q < STREAM_SPT; ++q) {
-      const int r = min(wid * STREAM_WARP_SAMPLES + q * 32 + lane, b - 1);   // rows past the batch re-read its last row
-      const float2* xrow = reinterpret_cast<const float2*>(xs + (size_t)r * D);
+      for (int q = 0; q < STREAM_SPT; ++q)
 #pragma unroll
-      for (int jp = 0; jp < D2; ++jp) xv[q][jp] = xrow[jp];
+        for (int jp = 0; jp < D2; ++jp) xv[q][jp] = xrow[q * 32 * D2 + jp];
     }
   };
   if (steps > 0) stage_in(0, batch_cur);
@@ -327,161 +313,166 @@ asgd_stream_kernel(const Params p, const long long steps) {
     if (tid < p.S) my_seq = ld_relaxed_gpu(p.seq + (size_t)i * p.S + tid);
     const int pos2 = next_pos(pos1);
     const int batch_nn = myperm[pos2];
+    float wmax2 = wmaxs[0];
+#pragma unroll
+    for (int q = 1; q < L::UPD_WARPS; ++q) wmax2 = fmaxf(wmax2, wmaxs[q]);
 
-    // ---- Eq. 8: scores of this thread's samples against every centre ----
-    float s1[STREAM_SPT], s2[STREAM_SPT];
+    if (warp_on) {
+      // ---- Eq. 8: scores of this thread's samples against every centre ----
+      float s1[STREAM_SPT], s2[STREAM_SPT];
 #pragma unroll
-    for (int q = 0; q < STREAM_SPT; ++q) { s1[q] = __int_as_float(0x7f800000); s2[q] = __int_as_float(0x7f800000); }
-    float wmax2 = 0.f;
-    // packed score of centre a for each of the thread's samples
-    auto scores_of = [&](int a, float (&sp)[STREAM_SPT]) {
-      float2 wr[DP / 2];
+      for (int q = 0; q < STREAM_SPT; ++q) { s1[q] = __int_as_float(0x7f800000); s2[q] = __int_as_float(0x7f800000); }
+      // packed score of centre a for each of the thread's samples
+      auto scores_of = [&](int a, float (&sp)[STREAM_SPT]) {
+        float2 wr[DP / 2];
 #pragma unroll
-      for (int j4 = 0; j4 < DP / 4; ++j4) {
-        const float4 v = *reinterpret_cast<const float4*>(wneg2 + a * DP + 4 * j4);
-        wr[2 * j4] = make_float2(v.x, v.y);
-        wr[2 * j4 + 1] = make_float2(v.z, v.w);
-      }
-      const float2 cn = cnorm[a];                       // (||w_a||^2, 0)
-      wmax2 = fmaxf(wmax2, cn.x);
+        for (int j4 = 0; j4 < DP / 4; ++j4) {
+          const float4 v = *reinterpret_cast<const float4*>(wneg2 + a * DP + 4 * j4);
+          wr[2 * j4] = make_float2(v.x, v.y);
+          wr[2 * j4 + 1] = make_float2(v.z, v.w);
+        }
+        const float2 cn = wr[D2];                         // (||w_a||^2, 0)
 #pragma unroll
-      for (int q = 0; q < STREAM_SPT; ++q) {
-        float2 acc = cn;
+        for (int q = 0; q < STREAM_SPT; ++q) {
+          float2 acc = cn;
 #pragma unroll
-        for (int jp = 0; jp < D2; ++jp) acc = __ffma2_rn(xv[q][jp], wr[jp], acc);
-        const float sc = acc.x + acc.y;
-        sp[q] = __uint_as_float((__float_as_uint(sc) & ~L::INDEX_MASK) | (unsigned)a);
-      }
-    };
-    // two centres at a time: with lo <= hi the new pair is  s1' = min(s1, lo),  s2' = min(max(s1, lo), s2, hi)
-#pragma unroll 1
-    for (int a = 0; a + 1 < K; a += 2) {
-      float pa[STREAM_SPT], pb[STREAM_SPT];
-      scores_of(a, pa);
-      scores_of(a + 1, pb);
+          for (int jp = 0; jp < D2; ++jp) acc = __ffma2_rn(xv[q][jp], wr[jp], acc);
+          const float sc = acc.x + acc.y;
+          sp[q] = __uint_as_float((__float_as_uint(sc) & ~L::INDEX_MASK) | (unsigned)a);
+        }
+      };
+      // two centres at a time: with lo <= hi the new pair is  s1' = min(s1, lo),  s2' = min(max(s1, lo), s2, hi)
 #pragma unroll
-      for (int q = 0; q < STREAM_SPT; ++q) {
-        const float lo = fminf(pa[q], pb[q]), hi = fmaxf(pa[q], pb[q]);
-        s2[q] = fmin3(fmaxf(s1[q], lo), s2[q], hi);
-        s1[q] = fminf(s1[q], lo);
-      }
-    }
-    if (K & 1) {
-      float pa[STREAM_SPT];
-      scores_of(K - 1, pa);
+      for (int a = 0; a + 1 < K; a += 2) {
+        asm volatile("" ::: "memory");                     // keep the loads of this pair of centre rows behind the pair before
+        float pa[STREAM_SPT], pb[STREAM_SPT];
+        scores_of(a, pa);
+        scores_of(a + 1, pb);
 #pragma unroll
-      for (int q = 0; q < STREAM_SPT; ++q) {
-        s2[q] = fmaxf(s1[q], fminf(s2[q], pa[q]));
-        s1[q] = fminf(s1[q], pa[q]);
-      }
-    }
-
-    // ---- decide: index from the packed minimum; direct differences when the runner-up is too close ----
-    int best[STREAM_SPT];
-#pragma unroll
-    for (int q = 0; q < STREAM_SPT; ++q) {
-      best[q] = (int)(__float_as_uint(s1[q]) & L::INDEX_MASK);
-      if (K > 1 && (s2[q] - s1[q]) <= tau_scale * (wmax2 + xmax2)) {       // cheap test with the global bound on ||x||^2 first
-        float2 n2 = __fmul2_rn(xv[q][0], xv[q][0]);
-#pragma unroll
-        for (int jp = 1; jp < D2; ++jp) n2 = __ffma2_rn(xv[q][jp], xv[q][jp], n2);
-        if ((s2[q] - s1[q]) <= tau_scale * (wmax2 + (n2.x + n2.y))) {
-          float bd = __int_as_float(0x7f800000);
-          int bb = 0;
-          for (int a = 0; a < K; ++a) {
-            float acc = 0.f;
-#pragma unroll
-            for (int jp = 0; jp < D2; ++jp) {
-              const float d0 = xv[q][jp].x + 0.5f * wneg2[a * DP + 2 * jp];        // -0.5 * (-2w) = w, exact
-              const float d1 = xv[q][jp].y + 0.5f * wneg2[a * DP + 2 * jp + 1];
-              acc = fmaf(d0, d0, acc);
-              acc = fmaf(d1, d1, acc);
-            }
-            if (acc < bd) { bd = acc; bb = a; }          // strict "<": the lowest index keeps a tie
-          }
-          best[q] = bb;
+        for (int q = 0; q < STREAM_SPT; ++q) {
+          const float lo = fminf(pa[q], pb[q]), hi = fmaxf(pa[q], pb[q]);
+          s2[q] = fmin3(fmaxf(s1[q], lo), s2[q], hi);
+          s1[q] = fminf(s1[q], lo);
         }
       }
-      if (wid * STREAM_WARP_SAMPLES + q * 32 + lane >= b) best[q] = K;   // rows past the batch form their own group
-    }
-    if (p.assign_rec) {
+      if (K & 1) {
+        float pa[STREAM_SPT];
+        scores_of(K - 1, pa);
+#pragma unroll
+        for (int q = 0; q < STREAM_SPT; ++q) {
+          s2[q] = fmaxf(s1[q], fminf(s2[q], pa[q]));
+          s1[q] = fminf(s1[q], pa[q]);
+        }
+      }
+
+      // ---- decide: index from the packed minimum; direct differences when the runner-up is too close ----
+      int best[STREAM_SPT];
+      bool close = false;
+      const float thr0 = tau_scale * (wmax2 + xmax2);                        // cheap test with the global bound on ||x||^2 first
 #pragma unroll
       for (int q = 0; q < STREAM_SPT; ++q) {
-        const int r = wid * STREAM_WARP_SAMPLES + q * 32 + lane;
-        if (r < b) p.assign_rec[(size_t)i * b + r] = best[q];
+        best[q] = (int)(__float_as_uint(s1[q]) & L::INDEX_MASK);
+        close |= (s2[q] - s1[q]) <= thr0;
       }
-    }
-    // ---- order: this warp's rows by the centre they chose, in row order inside a centre ----
-    __syncwarp();
-    int rank[STREAM_SPT];
-    unsigned cqa[STREAM_SPT];                                              // address of this row's centre in the block counts
+      if (K > 1 && close) {
 #pragma unroll
-    for (int q = 0; q < STREAM_SPT; ++q) {
-      const unsigned grp = __match_any_sync(0xffffffffu, best[q]);
-      const unsigned below = grp & lane_lt;
-      rank[q] = __popc(below);
-      cqa[q] = wb + (unsigned)L::W_CQ + ((unsigned)best[q] << 2);          // rows past the batch count into the spare column
-      if (q == 0) sts_u32_if<0 * CWS * 4>(cqa[q], (unsigned)__popc(grp), below == 0);
-      if (q == 1) sts_u32_if<1 * CWS * 4>(cqa[q], (unsigned)__popc(grp), below == 0);
-      if (q == 2) sts_u32_if<2 * CWS * 4>(cqa[q], (unsigned)__popc(grp), below == 0);
-      if (q == 3) sts_u32_if<3 * CWS * 4>(cqa[q], (unsigned)__popc(grp), below == 0);
+        for (int q = 0; q < STREAM_SPT; ++q) {
+          if ((s2[q] - s1[q]) <= thr0) {
+            float2 n2 = __fmul2_rn(xv[q][0], xv[q][0]);
+#pragma unroll
+            for (int jp = 1; jp < D2; ++jp) n2 = __ffma2_rn(xv[q][jp], xv[q][jp], n2);
+            if ((s2[q] - s1[q]) <= tau_scale * (wmax2 + (n2.x + n2.y))) {
+              float bd = __int_as_float(0x7f800000);
+              int bb = 0;
+              for (int a = 0; a < K; ++a) {
+                float acc = 0.f;
+#pragma unroll
+                for (int jp = 0; jp < D2; ++jp) {
+                  const float d0 = xv[q][jp].x + 0.5f * wneg2[a * DP + 2 * jp];        // -0.5 * (-2w) = w, exact
+                  const float d1 = xv[q][jp].y + 0.5f * wneg2[a * DP + 2 * jp + 1];
+                  acc = fmaf(d0, d0, acc);
+                  acc = fmaf(d1, d1, acc);
+                }
+                if (acc < bd) { bd = acc; bb = a; }          // strict "<": the lowest index keeps a tie
+              }
+              best[q] = bb;
+            }
+          }
+        }
+      }
+      if ((wid + 1) * STREAM_WARP_SAMPLES > b) {            // the warp that holds the end of the batch: rows past it count for no centre
+#pragma unroll
+        for (int q = 0; q < STREAM_SPT; ++q)
+          if (wid * STREAM_WARP_SAMPLES + q * 32 + lane >= b) best[q] = K;
+      }
+      if (p.assign_rec) {
+#pragma unroll
+        for (int q = 0; q < STREAM_SPT; ++q) {
+          const int r = wid * STREAM_WARP_SAMPLES + q * 32 + lane;
+          if (r < b) p.assign_rec[(size_t)i * b + r] = best[q];
+        }
+      }
+      // ---- Eq. 9 on the tensor cores: S^T[dim][centre] += X^T[dim][row] . onehot[row][centre] over the warp's rows ----
+      __syncwarp();                                        // the table's readers of the step before are done
+#pragma unroll
+      for (int q = 0; q < STREAM_SPT; ++q) best_w[8 * q] = (float)best[q];
+      __syncwarp();
+      float ch[NT][4], cl[NT][4];                          // sums of the hi terms (row d/2: counts), of the lo terms
+      float cc[NT][4];                                     // counts when no result row is spare (d = 16)
+      constexpr bool kSpareRow = D2 < 8;
+      // threads past the dimension pairs read (1, 0) instead of samples: result row d/2 counts the rows of a centre
+      const unsigned char* fa = (g < D2) ? xtile + frag_off : smem_raw + L::ONES;
+      const unsigned ones_a = (g == 0) ? 0x3f800000u : 0u; // d = 16: first operand of the counts, row 0 all ones
+#pragma unroll
+      for (int j2 = 0; j2 < STREAM_KSTEPS / 2; ++j2) {
+        const float4 bq = best_r[j2];                      // best centres of rows (t4, t4 + 4) of two products
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          // product 2*j2 + h takes rows 16*j2 + 2h + {0, 4, 8, 12} (columns t4 = 0..3) and the same rows + 1 (columns 4..7)
+          const float2 xa = *reinterpret_cast<const float2*>(fa + (size_t)(16 * j2 + 2 * h) * ROWB);
+          const float2 xb = *reinterpret_cast<const float2*>(fa + (size_t)(16 * j2 + 2 * h + 1) * ROWB);
+          const unsigned h0 = __float_as_uint(xa.x) & 0xffffe000u, h1 = __float_as_uint(xa.y) & 0xffffe000u;
+          const unsigned h2 = __float_as_uint(xb.x) & 0xffffe000u, h3 = __float_as_uint(xb.y) & 0xffffe000u;
+          const float2 la = __ffma2_rn(make_float2(__uint_as_float(h0), __uint_as_float(h1)), neg1, xa);
+          const float2 lb = __ffma2_rn(make_float2(__uint_as_float(h2), __uint_as_float(h3)), neg1, xb);
+          const float ba = h ? bq.z : bq.x, bb = h ? bq.w : bq.y;
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            const unsigned b0 = onehot_bits(ba, cg[nt]), b1 = onehot_bits(bb, cg[nt]);
+            if (j2 == 0 && h == 0) {
+              mma_tf32_16x8x8_first(ch[nt], h0, h1, h2, h3, b0, b1);
+              mma_tf32_16x8x8_first(cl[nt], __float_as_uint(la.x), __float_as_uint(la.y), __float_as_uint(lb.x), __float_as_uint(lb.y), b0, b1);
+              if (!kSpareRow) mma_tf32_16x8x8_first(cc[nt], ones_a, 0u, ones_a, 0u, b0, b1);
+            } else {
+              mma_tf32_16x8x8(ch[nt], h0, h1, h2, h3, b0, b1);
+              mma_tf32_16x8x8(cl[nt], __float_as_uint(la.x), __float_as_uint(la.y), __float_as_uint(lb.x), __float_as_uint(lb.y), b0, b1);
+              if (!kSpareRow) mma_tf32_16x8x8(cc[nt], ones_a, 0u, ones_a, 0u, b0, b1);
+            }
+          }
+        }
+      }
+      // the warp's sums and counts: thread (g, t4) holds centres 8*nt + 2*t4 (+1), dimensions 2g, 2g+1; the counts sit in
+      // result row d/2 (threads g = d/2), for d = 16 in row 0 of their own product
+      {
+        float2* wsum = reinterpret_cast<float2*>(warp_ptr(wid, L::W_SUM));
+        float* wcnt = reinterpret_cast<float*>(warp_ptr(wid, L::W_CNT));
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+          const int c0 = 8 * nt + 2 * t4;
+          if (g < D2) {
+            if (c0 < K) wsum[c0 * D2 + g] = make_float2(ch[nt][0] + cl[nt][0], ch[nt][2] + cl[nt][2]);
+            if (c0 + 1 < K) wsum[(c0 + 1) * D2 + g] = make_float2(ch[nt][1] + cl[nt][1], ch[nt][3] + cl[nt][3]);
+          }
+          if (kSpareRow ? (g == D2) : (g == 0)) {
+            if (c0 < K) wcnt[c0] = kSpareRow ? ch[nt][0] : cc[nt][0];
+            if (c0 + 1 < K) wcnt[c0 + 1] = kSpareRow ? ch[nt][1] : cc[nt][1];
+          }
+        }
+      }
     }
     if (tid < p.S && my_seq != seen_s[tid]) flags[0] = 1;
-    __syncwarp();
-    int ngroups;
-    {
-      // a row's place inside its centre: the centre's rows in the earlier 32-row blocks, then its rank in its own
-      static_assert(STREAM_SPT == 4, "four 32-row blocks per warp");
-      rank[1] += (int)lds_u32<0>(cqa[1]);
-      rank[2] += (int)(lds_u32<0>(cqa[2]) + lds_u32<CWS * 4>(cqa[2]));
-      rank[3] += (int)(lds_u32<0>(cqa[3]) + lds_u32<CWS * 4>(cqa[3]) + lds_u32<2 * CWS * 4>(cqa[3]));
-      // lane = centre: its rows, its groups, and the first group by a running sum (entry K holds the total)
-      const unsigned ca = wb + (unsigned)L::W_CQ + ((unsigned)lane_c << 2);
-      int n = (int)(lds_u32<0>(ca) + lds_u32<CWS * 4>(ca) + lds_u32<2 * CWS * 4>(ca) + lds_u32<3 * CWS * 4>(ca));
-      n = (lane < K) ? n : 0;
-      sts_u32<(int)(L::W_CW - L::W_CQ)>(ca, (unsigned)n);
-      const int ng = (n + STREAM_GROUP - 1) / STREAM_GROUP;
-      int inc = ng;
-#pragma unroll
-      for (int o = 1; o < K; o <<= 1) inc = scan_step(inc, o);
-      const int first = inc - ng;
-      ngroups = __shfl_sync(0xffffffffu, inc, K - 1);                      // the running sum reaches K - 1 lanes down
-      sts_u32<(int)(L::W_FIRST - L::W_CQ)>(ca, (unsigned)((lane < K) ? first : ngroups));
-#pragma unroll
-      for (int q = 0; q < STREAM_SPT; ++q) {
-        const int f = __shfl_sync(0xffffffffu, first, best[q]);            // best[q] <= K
-        const unsigned at = wb + (unsigned)L::W_ORDER + (((unsigned)f * STREAM_GROUP + (unsigned)rank[q]) << 2);
-        sts_u32_if<0>(at, xsa + row0 + (unsigned)(q * 32 * ROWB), best[q] < K);
-      }
-    }
-    __syncwarp();
 
-    // ---- Eq. 9: lanes (group, dimension pair) add the eight rows of a group (all of one centre) from the tile ----
-    {
-      const int gl = lane / D2, jp = lane - gl * D2;
-      const unsigned jo = (unsigned)jp * 8u;
-      auto group_sum = [&](const uint4& lo, const uint4& hi) {
-        float2 acc0 = lds_f2<0>(lo.x + jo), acc1 = lds_f2<0>(lo.y + jo);
-        acc0 = __fadd2_rn(acc0, lds_f2<0>(lo.z + jo)); acc1 = __fadd2_rn(acc1, lds_f2<0>(lo.w + jo));
-        acc0 = __fadd2_rn(acc0, lds_f2<0>(hi.x + jo)); acc1 = __fadd2_rn(acc1, lds_f2<0>(hi.y + jo));
-        acc0 = __fadd2_rn(acc0, lds_f2<0>(hi.z + jo)); acc1 = __fadd2_rn(acc1, lds_f2<0>(hi.w + jo));
-        return __fadd2_rn(acc0, acc1);
-      };
-      // two groups per lane in flight; groups past the last one hold the row of zeros
-      if (gl < GPR) {
-        for (int g = gl; g < ngroups; g += 2 * GPR) {
-          const unsigned oa = wb + (unsigned)L::W_ORDER + (unsigned)g * (STREAM_GROUP * 4);
-          const uint4 a0 = lds_v4<0>(oa), a1 = lds_v4<16>(oa);
-          const uint4 b0 = lds_v4<GPR * STREAM_GROUP * 4>(oa), b1 = lds_v4<GPR * STREAM_GROUP * 4 + 16>(oa);
-          const float2 sa = group_sum(a0, a1), sb = group_sum(b0, b1);
-          const unsigned ga = wb + (unsigned)L::W_GSUM + (unsigned)g * (D * 4) + jo;
-          sts_f2<0>(ga, sa);
-          sts_f2<GPR * D * 4>(ga, sb);
-        }
-      }
-    }
-
-    // ---- barrier B: group sums and counts complete, the ring slot is free again ----
+    // ---- barrier B: the warps' sums and counts are complete, the ring slot is free again ----
     if (__syncthreads_or(abort)) { abort = 1; break; }
 
     // the slot's rows have been added: start the copy of the batch after the next into it
@@ -494,7 +485,7 @@ asgd_stream_kernel(const Params p, const long long steps) {
       // a message is waiting: totals into SD, then the general tail (which also sends when a put is due)
       for (int e = tid; e < K * D2; e += STREAM_THREADS)
         reinterpret_cast<float2*>(SD)[e] = centre_sum(e / D2, e % D2);
-      if (tid < K) cnt[tid] = centre_rows(tid);
+      if (tid < K) cnt[tid] = (int)centre_rows(tid);
       __syncthreads();
       step_tail<kDet>(p, i, t, w, D, SD, cnt, wglob, ts);
       if (tid < p.S) seen_s[tid] = p.seen[(size_t)i * p.S + tid];
@@ -505,7 +496,13 @@ asgd_stream_kernel(const Params p, const long long steps) {
         float s = 0.f;
 #pragma unroll
         for (int j = 0; j < D; ++j) s = fmaf(w[tid * D + j], w[tid * D + j], s);
-        cnorm[tid] = make_float2(s, 0.f);
+        wneg2[tid * DP + D] = s;
+      }
+      __syncthreads();
+      if (tid < L::UPD_WARPS) {
+        float m = 0.f;
+        for (int a = 0; a < K; ++a) m = fmaxf(m, wneg2[a * DP + D]);
+        wmaxs[tid] = m;
       }
     } else {
       // common case: plain local step  w <- w - eps * D,  D = (n_a w - S) / b.  The first warps update CPW
@@ -516,12 +513,12 @@ asgd_stream_kernel(const Params p, const long long steps) {
         const bool on = (al < L::CPW) && (a < K);
         float sq = 0.f;
         if (on) {
-          const int n = centre_rows(a);
+          const float n = centre_rows(a);
           const float2 ssum = centre_sum(a, jp);
           const float2 ww = *reinterpret_cast<const float2*>(w + a * D + 2 * jp);
           float2 nw;
-          nw.x = ww.x - eps * (((float)n * ww.x - ssum.x) * inv_b);
-          nw.y = ww.y - eps * (((float)n * ww.y - ssum.y) * inv_b);
+          nw.x = ww.x - eps * ((n * ww.x - ssum.x) * inv_b);
+          nw.y = ww.y - eps * ((n * ww.y - ssum.y) * inv_b);
           *reinterpret_cast<float2*>(w + a * D + 2 * jp) = nw;
           *reinterpret_cast<float2*>(wneg2 + a * DP + 2 * jp) = make_float2(-2.f * nw.x, -2.f * nw.y);
           *reinterpret_cast<float2*>(wglob + a * D + 2 * jp) = nw;
@@ -532,7 +529,10 @@ asgd_stream_kernel(const Params p, const long long steps) {
           const float up = __shfl_down_sync(0xffffffffu, sq, o);
           if (jp + o < D2) sq += up;
         }
-        if (on && jp == 0) cnorm[a] = make_float2(sq, 0.f);
+        if (on && jp == 0) wneg2[a * DP + D] = sq;
+        // max ||w_a||^2 over this warp's centres: non-negative floats order like their bit patterns
+        const unsigned mbits = __reduce_max_sync(0xffffffffu, (on && jp == 0) ? __float_as_uint(sq) : 0u);
+        if (lane == 0) wmaxs[wid] = __uint_as_float(mbits);
       }
       unsigned long long n_sent = 0;
       if (put_now) {
