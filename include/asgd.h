@@ -49,8 +49,8 @@ typedef enum asgd_status {
 enum {
   ASGD_PATH_AUTO = 0,
   ASGD_PATH_FP32 = 1,       /* CUDA cores, fp32 (the specialised kernel for the shape, if any) */
-  ASGD_PATH_TC_3XTF32 = 2,  /* tcgen05, three TF32 products per fp32 product                 */
-  ASGD_PATH_TC_BF16 = 3,    /* tcgen05, BF16 operands, fp32 accumulate                       */
+  ASGD_PATH_TC_BF16 = 3,    /* tcgen05, BF16 operands in two terms each (x_hi + x_lo, w_hi + w_lo; */
+                            /* three products per score), fp32 accumulate                    */
   ASGD_PATH_FP32_GENERAL = 4 /* CUDA cores, fp32, the shape-independent kernel                */
 };
 
@@ -84,7 +84,8 @@ int asgd_workspace_bytes(const asgd_config *cfg, size_t *bytes /* HOST out */);
  * receive buffers are emptied, counters zeroed, batch orders drawn.
  *   X_dev        DEVICE [N*d] fp32 row-major, 16-byte aligned.  BORROWED: never written, must stay
  *                alive and unchanged until asgd_destroy().
- *   X_bf16_dev   DEVICE [N*d] bf16 copy of X for ASGD_PATH_TC_BF16, or NULL.
+ *   X_bf16_dev   DEVICE [N*d] bf16 copy of X for ASGD_PATH_TC_BF16 (taken as the leading term x_hi; the
+ *                library forms the residue x_lo itself), or NULL.  BORROWED like X_dev.
  *   w0_dev       DEVICE [k*d] fp32.  COPIED.
  *   workspace    DEVICE, >= asgd_workspace_bytes(), 256-byte aligned.  BORROWED until destroy.
  *   cuda_stream  a cudaStream_t (NULL = default stream).

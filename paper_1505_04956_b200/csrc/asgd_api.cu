@@ -34,7 +34,7 @@ enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2, P_TC_BF16 = 3 };
 
 struct Layout {
   size_t state, mail, seq, seen, arb_win, arb_cnt, mail_rows, rowacc, rowin, stats, perm, status, assign_rec, accept_rec, gsum,
-      eval_partial, tmp_state, xmax, wbf, top2, xbf, total;
+      eval_partial, tmp_state, xmax, wbf, top2, xbf, xbl, xnorm, total;
 };
 
 constexpr size_t kAlign = 256;
@@ -50,7 +50,9 @@ bool config_ok(const asgd_config* c) {
   if (c->comm_interval < 0 || c->fanout < 0 || c->fanout > c->W - 1 || c->fanout > MAX_FANOUT) return false;
   if (c->slots < 1 || c->slots > MAX_SLOTS) return false;
   if (c->partial_rows < 0 || c->partial_rows > c->k) return false;
-  if (c->dist_path < ASGD_PATH_AUTO || c->dist_path > ASGD_PATH_FP32_GENERAL) return false;
+  if (c->dist_path != ASGD_PATH_AUTO && c->dist_path != ASGD_PATH_FP32 && c->dist_path != ASGD_PATH_TC_BF16 &&
+      c->dist_path != ASGD_PATH_FP32_GENERAL)
+    return false;
   if ((long long)c->k * c->d > (1ll << 28)) return false;
   const long long H = c->N / c->W;
   if (H < c->b) return false;
@@ -90,9 +92,11 @@ Layout make_layout(const asgd_config* c) {
   L.tmp_state = take(kd_pad * 4);
   L.xmax = take(64);
   const bool tc = tc_eligible(c) && (c->dist_path == ASGD_PATH_TC_BF16 || c->dist_path == ASGD_PATH_AUTO);
-  L.wbf = take(tc ? W * kd * 2 : 4);
-  L.top2 = take(tc ? W * (size_t)c->b * 8 : 4);
+  L.wbf = take(tc ? 2 * W * kd * 2 : 4);
+  L.top2 = take(tc ? W * (size_t)c->b * 16 : 4);
   L.xbf = take(tc ? (size_t)c->N * c->d * 2 : 4);
+  L.xbl = take(tc ? (size_t)c->N * c->d * 2 : 4);
+  L.xnorm = take(tc ? (size_t)c->N * 4 : 4);
   L.total = off;
   return L;
 }
@@ -115,7 +119,7 @@ struct asgd_ctx {
   int last_cuda;
   int sm_count;
   const void* xbf_user;   // caller's bf16 copy of X, or nullptr
-  CUtensorMap mapX, mapW; // tensor-core path: bf16 samples [N][d], bf16 -2w [W*k][d]
+  CUtensorMap mapXh, mapXl, mapW; // tensor-core path: BF16 terms of the samples [N][d] each, of -2w [2*W*k][d]
 };
 
 namespace {
@@ -221,17 +225,20 @@ int tc_prepare(asgd_ctx* c) {
   CU(c, cudaFuncSetAttribute(asgd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
   p.wbf = c->ws + c->L.wbf;
   p.top2 = (float*)(c->ws + c->L.top2);
-  const void* xbf = c->xbf_user;
-  if (!xbf) {
-    void* dst = c->ws + c->L.xbf;
-    tc_convert_x_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, (__nv_bfloat16*)dst, (size_t)cfg.N * cfg.d);
-    c->launches += 1;
-    CU(c, cudaGetLastError());
-    xbf = dst;
-  }
+  // x = x_hi + x_lo in BF16: x_hi is the caller's copy when one was given, x_lo the rounded residue either way
+  const void* xbf = c->xbf_user ? c->xbf_user : (const void*)(c->ws + c->L.xbf);
+  void* xbl = c->ws + c->L.xbl;
+  tc_split_x_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, (const __nv_bfloat16*)c->xbf_user,
+                                                             c->xbf_user ? nullptr : (__nv_bfloat16*)(c->ws + c->L.xbf),
+                                                             (__nv_bfloat16*)xbl, (size_t)cfg.N * cfg.d);
+  tc_row_norms_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, cfg.N, cfg.d, (float*)(c->ws + c->L.xnorm));
+  c->launches += 2;
+  CU(c, cudaGetLastError());
+  p.xnorm = (const float*)(c->ws + c->L.xnorm);
   { const int rc = compute_xmax2(c); if (rc != ASGD_OK) return rc; }
-  if (!encode_bf16_map(&c->mapX, xbf, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
-  if (!encode_bf16_map(&c->mapW, p.wbf, (unsigned long long)cfg.W * cfg.k, (unsigned long long)cfg.d, TC_N)) return ASGD_ECUDA;
+  if (!encode_bf16_map(&c->mapXh, xbf, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
+  if (!encode_bf16_map(&c->mapXl, xbl, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
+  if (!encode_bf16_map(&c->mapW, p.wbf, 2ull * cfg.W * cfg.k, (unsigned long long)cfg.d, TC_N)) return ASGD_ECUDA;
   return ASGD_OK;
 }
 
@@ -240,9 +247,9 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
   switch (c->path) {
     case P_TC_BF16:
       if (det)
-        asgd_tc_kernel<true><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapX, c->mapW);
+        asgd_tc_kernel<true><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
       else
-        asgd_tc_kernel<false><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapX, c->mapW);
+        asgd_tc_kernel<false><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
       break;
     case P_TILED: {
       int idx = 0;
@@ -271,7 +278,6 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
 
 int resolve_path(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
-  if (cfg.dist_path == ASGD_PATH_TC_3XTF32) return ASGD_EUNSUPPORTED;
   if (cfg.dist_path == ASGD_PATH_TC_BF16 || (cfg.dist_path == ASGD_PATH_AUTO && tc_eligible(&cfg))) {
     if (!tc_eligible(&cfg)) return ASGD_EUNSUPPORTED;
     c->path = P_TC_BF16;
@@ -395,6 +401,7 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   p.withhold_step = -1;
   p.wbf = nullptr;
   p.top2 = nullptr;
+  p.xnorm = nullptr;
 
   int rc = resolve_path(c);
   if (rc != ASGD_OK) { delete c; return rc; }

@@ -35,8 +35,9 @@ struct Params {
   int* accept_rec;         // [W][S] acceptance of the last step
   float* gsum;             // [W][kd_pad] per-worker sums when the state does not fit on chip
   float xmax2;             // max_i ||x_i||^2 over X (error bound of the tensor-core path)
-  void* wbf;               // [W][k][d] bf16 copies of -2w (tensor-core path)
-  float* top2;             // [W][b][2] running (minimum, runner-up) scores (tensor-core path)
+  void* wbf;               // [2][W][k][d] BF16 terms of -2w: w_hi, then w_lo (tensor-core path)
+  float* top2;             // [W][b][4] the three smallest packed squared distances of every row (tensor-core path)
+  const float* xnorm;      // [N] ||x_i||^2 (tensor-core path)
   int rows_m;              // per-centre messages (Section 4.4): centre rows per message, 0 = whole-state messages
   int2* mail_rows;         // [W][S] (first row, number of rows) of the buffer's last message (per-centre mode)
   unsigned* rowacc;        // [W][k] bit s: row accepted from buffer s in the worker's last step (per-centre mode)

@@ -1,19 +1,26 @@
-// Tensor-core path (tcgen05, BF16 operands, FP32 accumulate in tensor memory) for large states
-// (k up to 1024, d a multiple of 64 up to 256): the shapes where the scores of Eq. 8 are a dense
+// Tensor-core path (tcgen05, BF16 operands in two terms each, FP32 accumulate in tensor memory) for large
+// states (k up to 1024, d a multiple of 64 up to 256): the shapes where the scores of Eq. 8 are a dense
 // contraction  -2 X W^T  of a 4096 x 256 mini-batch against a 1024 x 256 centre matrix.
 //
+// Split precision: x = x_hi + x_lo and -2w = w_hi + w_lo with every term a BF16 number (x_lo, w_lo hold the
+// rounding residues), and the score takes three products  x_hi.w_hi + x_lo.w_hi + x_hi.w_lo  into the same
+// accumulator.  What is left out (x_lo.w_lo and the residues of the residues) is below 6 * 2^-18 ||x|| ||w||, so
+// the scores are good to about 16 bits, the Eq. 8 decision falls to the exact fp32 comparison only for a fraction
+// of a percent of the rows, and every such row is decided among ALL centres that the bound cannot rule out.
+//
 // One worker = one thread block = one SM.  Warp roles while the scores are computed:
-//   warp 0   one lane issues the TMA loads: a 128-row sample tile in 128-byte-swizzled K-chunks of 64,
-//            resident while all centre blocks pass, and 256-centre blocks of bf16(-2w) through a
-//            4-slot ring of K-chunks (they come from L2: all workers' bf16 states fit there);
-//   warp 1   allocates tensor memory; one lane issues tcgen05.mma (128 x 256 x 16 per instruction)
-//            into one of two 256-column accumulator stages and commits to mbarriers;
-//   warps 4-7  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread), add
-//            ||w_a||^2 and keep, per sample, the two smallest scores with the centre index packed
+//   warp 0   one lane issues the TMA loads: a 128-row sample tile (hi and lo) in 128-byte-swizzled K-chunks of 64,
+//            resident while all centre blocks pass, and 128-centre blocks of w_hi, w_lo through a ring of
+//            K-chunks (they come from L2);
+//   warp 1   allocates tensor memory; one lane issues tcgen05.mma (128 x 128 x 16 per instruction) into one
+//            of two 128-column accumulator stages and commits to mbarriers;
+//   warps 4-7  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread), add ||w_a||^2 and
+//            ||x||^2 and keep, per sample, the three smallest squared distances with the centre index packed
 //            into the low mantissa bits, carried in registers over the centre blocks.
-// Then all warps: samples whose two best scores are closer than the BF16 error bound are decided
-// between those two centres with fp32 inputs (fp64 sums); rows are grouped by centre and each centre's
-// sum of fp32 master samples, update, bf16(-2w) and ||w_a||^2 come from one pass.  Every wait is bounded.
+// Then all warps: a sample whose runner-up is inside the error bound is decided between its two candidates with
+// fp32 inputs (fp64 sums when still close); one whose third candidate is inside the bound as well is decided
+// over all centres the same way.  Rows are grouped by centre and each centre's sum of fp32 master samples,
+// update, new w_hi, w_lo and ||w_a||^2 come from one pass.  Every wait is bounded.
 #pragma once
 
 #include <cuda.h>
@@ -26,28 +33,28 @@ namespace asgd {
 
 constexpr int TC_THREADS = 256;
 constexpr int TC_WARPS = TC_THREADS / 32;
-constexpr int TC_M = 128, TC_N = 256, TC_KC = 64;        // one MMA's output tile; K chunk = 64 bf16 = one swizzled 128-byte row
-constexpr int TC_MH = 1;                                  // 128-row parts of the resident sample tile (TC_MH * TC_N <= 256 accumulator columns per stage)
-constexpr int TC_A_STAGES = 4;                            // K chunks of the resident sample tile (d <= 256)
-constexpr int TC_B_STAGES = 4;                            // ring slots for the centre blocks
-constexpr int TC_BG = 1;                                  // K chunks per ring slot (one wait and one commit per slot; 2 x 2 was no faster than 4 x 1)
+constexpr int TC_M = 128, TC_N = 128, TC_KC = 64;        // one MMA's output tile; K chunk = 64 bf16 = one swizzled 128-byte row
+constexpr int TC_A_STAGES = 4;                            // K chunks of the resident sample tile (d <= 256), each with a hi and a lo part
+constexpr int TC_B_STAGES = 4;                            // ring slots for the centre blocks (one K chunk of w_hi or of w_lo each)
 constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB per part
-constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;       // 32 KB
+constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;       // 16 KB
+constexpr int TC_TMEM_COLS = 2 * TC_N;                    // two accumulator stages
 constexpr int TC_SUM_ROWS = 4;                            // sample rows a centre's adders keep in flight
-constexpr int TC_MAX_K = 1024, TC_MAX_D = 256, TC_MAX_B = 8192;
+constexpr int TC_MAX_K = 1024, TC_MAX_D = 256, TC_MAX_B = 4096;
 constexpr unsigned TC_INDEX_MASK = 1023u;
+constexpr float TC_FAR = 1e30f;                          // stands for ||w_a||^2 of the padding centres
 
 struct TcSmem {
   size_t B, A, cn, cnt, best, flagged, bars, misc, tail, total;
   __host__ __device__ TcSmem(int k, int d, int b) {
     size_t off = 0;
     auto take = [&](size_t bytes, size_t align) { off = (off + align - 1) / align * align; size_t o = off; off += bytes; return o; };
-    A = take((size_t)TC_A_STAGES * TC_MH * TC_A_STAGE_BYTES, 1024);   // [K chunk][part]
-    B = take((size_t)TC_B_STAGES * TC_BG * TC_B_CHUNK_BYTES, 1024);
+    A = take((size_t)TC_A_STAGES * 2 * TC_A_STAGE_BYTES, 1024);       // [K chunk][hi, lo]; also the scratch of the grouping phase
+    B = take((size_t)TC_B_STAGES * TC_B_CHUNK_BYTES, 1024);
     cn = take((size_t)((k + TC_N - 1) / TC_N) * TC_N * 4, 16);
     cnt = take((size_t)k * 4, 16);
     best = take((size_t)b * 2, 16);
-    flagged = take((size_t)b * 2 + 16, 16);
+    flagged = take((size_t)b * 2 + 16, 16);                          // pairs to settle from the front, rows for the full scan from the back
     bars = take(32 * 8, 16);
     misc = take(64, 16);
     tail = take(sizeof(TailScratch), 16);
@@ -87,13 +94,29 @@ __device__ inline void red_add_v4(float* addr, float4 v) {
   asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
 }
 
-// samples -> bf16 copy (initialisation, when the caller gave none)
-__global__ void tc_convert_x_kernel(const float* __restrict__ X, __nv_bfloat16* __restrict__ out, size_t n) {
-  for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4; e + 3 < n; e += (size_t)gridDim.x * blockDim.x * 4) {
-    const float4 v = *reinterpret_cast<const float4*>(X + e);
-    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-    *reinterpret_cast<__nv_bfloat162*>(out + e) = lo;
-    *reinterpret_cast<__nv_bfloat162*>(out + e + 2) = hi;
+// samples -> BF16 hi and lo terms (initialisation).  hi_in: the caller's BF16 copy, or nullptr (then hi = round(x));
+// lo = round(x - hi) either way, so that hi + lo is x to 16 bits whatever copy the caller brought.
+__global__ void tc_split_x_kernel(const float* __restrict__ X, const __nv_bfloat16* __restrict__ hi_in, __nv_bfloat16* __restrict__ hi_out,
+                                  __nv_bfloat16* __restrict__ lo_out, size_t n) {
+  for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2; e + 1 < n; e += (size_t)gridDim.x * blockDim.x * 2) {
+    const float2 v = *reinterpret_cast<const float2*>(X + e);
+    __nv_bfloat162 h = hi_in ? *reinterpret_cast<const __nv_bfloat162*>(hi_in + e) : __floats2bfloat162_rn(v.x, v.y);
+    if (hi_out) *reinterpret_cast<__nv_bfloat162*>(hi_out + e) = h;
+    const float2 hf = __bfloat1622float2(h);
+    *reinterpret_cast<__nv_bfloat162*>(lo_out + e) = __floats2bfloat162_rn(v.x - hf.x, v.y - hf.y);
+  }
+}
+// ||x_i||^2 of every row (fp32): added to the scores so that the numbers compared are squared distances, whose
+// low mantissa bits (where the centre index rides) are worth far less than those of the raw scores.
+__global__ void tc_row_norms_kernel(const float* __restrict__ X, long long N, int d, float* __restrict__ out) {
+  const int lane = threadIdx.x & 31;
+  for (long long r = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < N; r += ((long long)gridDim.x * blockDim.x) >> 5) {
+    const float* x = X + (size_t)r * d;
+    float s = 0.f;
+    for (int j = lane * 2; j < d; j += 64) { const float2 v = *reinterpret_cast<const float2*>(x + j); s = fmaf(v.x, v.x, s); s = fmaf(v.y, v.y, s); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) out[r] = s;
   }
 }
 
@@ -123,33 +146,43 @@ __device__ inline void tc_add_rows(const float* __restrict__ X, long long row0, 
 enum { TCB_BFULL = 0, TCB_BEMPTY = TC_B_STAGES, TCB_AFULL = 2 * TC_B_STAGES, TCB_AEMPTY = 2 * TC_B_STAGES + TC_A_STAGES,
        TCB_ACCFULL = 2 * TC_B_STAGES + 2 * TC_A_STAGES, TCB_ACCEMPTY = TCB_ACCFULL + 2, TCB_COUNT = TCB_ACCFULL + 4 };
 
+// smallest three of (m1 <= m2 <= m3) and a new value, kept sorted (five min/max)
+__device__ __forceinline__ void tc_top3_insert(float& m1, float& m2, float& m3, float v) {
+  const float hi1 = fmaxf(m1, v);
+  m1 = fminf(m1, v);
+  const float hi2 = fmaxf(m2, hi1);
+  m2 = fminf(m2, hi1);
+  m3 = fminf(m3, hi2);
+}
+
 template <bool kDet>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CUtensorMap mapX,
-               const __grid_constant__ CUtensorMap mapW) {
+asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CUtensorMap mapXh,
+               const __grid_constant__ CUtensorMap mapXl, const __grid_constant__ CUtensorMap mapW) {
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
   unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const int k = p.k, d = p.d, b = p.b;
   const TcSmem map(k, d, b);
   unsigned char* sB = smem + map.B;
   unsigned char* sA = smem + map.A;
-  float* cn = reinterpret_cast<float*>(smem + map.cn);                 // ||w_a||^2, +inf beyond k
+  float* cn = reinterpret_cast<float*>(smem + map.cn);                 // ||w_a||^2; beyond k a large finite number (with index bits
+                                                                       // packed in, an infinity would read as a NaN and upset the min/max chain)
   int* cnt = reinterpret_cast<int*>(smem + map.cnt);
   unsigned short* best = reinterpret_cast<unsigned short*>(smem + map.best);
   unsigned short* flagged = reinterpret_cast<unsigned short*>(smem + map.flagged);
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + map.bars);
-  int* misc = reinterpret_cast<int*>(smem + map.misc);                 // [0] tmem base, [1] flagged count, [2] abort, [3] wmax2 bits
+  int* misc = reinterpret_cast<int*>(smem + map.misc);                 // [0] tmem base, [1] pairs to settle, [2] abort, [4] news, [5] rows for the full scan
   TailScratch* ts = reinterpret_cast<TailScratch*>(smem + map.tail);
 
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int i = blockIdx.x;
   const int nkc = d / TC_KC;                                           // K chunks per tile
-  const int ngr = (nkc + TC_BG - 1) / TC_BG;                           // ring slots a centre block passes through
-  const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_MH * TC_M - 1) / (TC_MH * TC_M);
+  const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_M - 1) / TC_M;
   float* wglob = p.state + (size_t)i * p.kd_pad;
   float* gsum = p.gsum + (size_t)i * p.kd_pad;
-  __nv_bfloat16* wbf = reinterpret_cast<__nv_bfloat16*>(p.wbf) + (size_t)i * k * d;
-  float2* top2 = reinterpret_cast<float2*>(p.top2) + (size_t)i * b;        // per row: (minimum, runner-up)
+  __nv_bfloat16* wbf = reinterpret_cast<__nv_bfloat16*>(p.wbf) + (size_t)i * k * d;          // w_hi of this worker
+  __nv_bfloat16* wbl = wbf + (size_t)p.W * k * d;                                            // w_lo: second half of the array
+  float4* top3 = reinterpret_cast<float4*>(p.top2) + (size_t)i * b;        // per row: three smallest packed squared distances
   const float INF = __int_as_float(0x7f800000);
   const float inv_b = 1.0f / (float)b;
 
@@ -161,24 +194,48 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     misc[2] = 0;
   }
   if (wid == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(misc)) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(misc)), "n"(TC_TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // prologue: bf16(-2w), ||w_a||^2 from the fp32 state (a warp per centre, lane = dl dimensions)
-  for (int a = wid; a < n_tiles * TC_N; a += TC_WARPS) {
-    float s = 0.f;
-    if (a < k) {
-      for (int j = lane * 2; j < d; j += 64) {
-        const float2 v = *reinterpret_cast<const float2*>(wglob + (size_t)a * d + j);
-        s = fmaf(v.x, v.x, s); s = fmaf(v.y, v.y, s);
-        *reinterpret_cast<__nv_bfloat162*>(wbf + (size_t)a * d + j) = __floats2bfloat162_rn(-2.f * v.x, -2.f * v.y);
+  // -2w as two BF16 terms and ||w_a||^2 of one centre held by eight lanes (lane l8: dimensions 4*l8 + 32*q)
+  const int sub = lane >> 3, l8 = lane & 7;
+  const int nq = d / 32;
+  auto refresh = [&](int a, const float4 (&w4)[TC_MAX_D / 32]) {
+    float sq = 0.f;
+#pragma unroll
+    for (int q = 0; q < TC_MAX_D / 32; ++q) {
+      if (q < nq) {
+        sq = fmaf(w4[q].x, w4[q].x, sq); sq = fmaf(w4[q].y, w4[q].y, sq); sq = fmaf(w4[q].z, w4[q].z, sq); sq = fmaf(w4[q].w, w4[q].w, sq);
+        const size_t o = (size_t)a * d + 4 * l8 + 32 * q;
+        const float v[4] = {-2.f * w4[q].x, -2.f * w4[q].y, -2.f * w4[q].z, -2.f * w4[q].w};     // exact
+        const __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
+        const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+        *reinterpret_cast<__nv_bfloat162*>(wbf + o) = h01;
+        *reinterpret_cast<__nv_bfloat162*>(wbf + o + 2) = h23;
+        *reinterpret_cast<__nv_bfloat162*>(wbl + o) = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y);
+        *reinterpret_cast<__nv_bfloat162*>(wbl + o + 2) = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+      }
+    }
+    return sq;
+  };
+  auto refresh_all = [&]() {                                            // every centre from the fp32 state in HBM
+    for (int a0 = wid * 4; a0 < n_tiles * TC_N; a0 += TC_WARPS * 4) {
+      const int a = a0 + sub;
+      float sq = 0.f;
+      if (a < k) {
+        float4 w4[TC_MAX_D / 32];
+#pragma unroll
+        for (int q = 0; q < TC_MAX_D / 32; ++q)
+          if (q < nq) w4[q] = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q);
+        sq = refresh(a, w4);
       }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+      for (int o = 1; o < 8; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      if (l8 == 0) cn[a] = (a < k) ? sq : TC_FAR;
     }
-    if (lane == 0) cn[a] = (a < k) ? s : INF;
-  }
-  asm volatile("fence.proxy.async;" ::: "memory");                      // bf16(-2w) written above is read by TMA
+  };
+  refresh_all();
+  asm volatile("fence.proxy.async;" ::: "memory");                      // the BF16 terms written above are read by TMA
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -193,33 +250,31 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     const long long batch = p.perm[(size_t)i * p.B + (size_t)(t % (unsigned long long)p.B)];
     const long long row0 = (long long)i * p.H + batch * b;
 
-    // ================= scores: -2 X W^T + ||w||^2, two best per sample =================
-    // A sample tile (TC_MH parts of 128 rows, nkc K-chunks each) stays in shared memory while the centre blocks stream
-    // past it through the ring (the bf16 states of all workers fit in L2; the samples are read from HBM once).
+    // ================= scores: three BF16 products per K chunk, three best per sample =================
+    // A sample tile (128 rows, nkc K-chunks of x_hi and x_lo) stays in shared memory while the centre blocks stream
+    // past it through the ring, w_hi then w_lo of every K chunk; the samples are read from HBM once.
     if (wid == 0) {
       if (lane == 0) {
         unsigned um = it_m, ibc = it_bc;
         bool ok = true;
         for (int m = 0; m < m_tiles && ok; ++m, ++um) {
-          const int halves = min(TC_MH, (b - m * TC_MH * TC_M + TC_M - 1) / TC_M);
           for (int kc = 0; kc < nkc && ok; ++kc) {
             if (um > 0) ok = mbar_wait_bounded(bars + TCB_AEMPTY + kc, (um - 1) & 1, p.wait_limit);     // last use of the chunk by the previous tile
             if (!ok) break;
-            mbar_expect_tx(bars + TCB_AFULL + kc, (unsigned)(halves * TC_A_STAGE_BYTES));
+            mbar_expect_tx(bars + TCB_AFULL + kc, (unsigned)(2 * TC_A_STAGE_BYTES));
             const bool withheld = (m == 0 && kc == 0 && step == p.withhold_step);   // failure drill: announced, never copied
-            for (int h = 0; h < halves && !withheld; ++h)
-              tma_load_2d(sA + (size_t)(kc * TC_MH + h) * TC_A_STAGE_BYTES, &mapX, kc * TC_KC,
-                          (int)(row0 + (long long)(m * TC_MH + h) * TC_M), bars + TCB_AFULL + kc);
+            if (!withheld) {
+              tma_load_2d(sA + (size_t)(kc * 2 + 0) * TC_A_STAGE_BYTES, &mapXh, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc);
+              tma_load_2d(sA + (size_t)(kc * 2 + 1) * TC_A_STAGE_BYTES, &mapXl, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc);
+            }
           }
           for (int n = 0; n < n_tiles && ok; ++n) {
-            for (int g = 0; g < ngr; ++g, ++ibc) {
+            for (int g = 0; g < 2 * nkc; ++g, ++ibc) {                 // g = 2 * K chunk + (0: w_hi, 1: w_lo)
               const int st = ibc % TC_B_STAGES;
               if (ibc >= TC_B_STAGES) ok = mbar_wait_bounded(bars + TCB_BEMPTY + st, ((ibc / TC_B_STAGES) - 1) & 1, p.wait_limit);
               if (!ok) break;
-              const int cnt_kc = min(TC_BG, nkc - g * TC_BG);
-              mbar_expect_tx(bars + TCB_BFULL + st, (unsigned)(cnt_kc * TC_B_CHUNK_BYTES));
-              for (int c = 0; c < cnt_kc; ++c)
-                tma_load_2d(sB + (size_t)(st * TC_BG + c) * TC_B_CHUNK_BYTES, &mapW, (g * TC_BG + c) * TC_KC, i * k + n * TC_N, bars + TCB_BFULL + st);
+              mbar_expect_tx(bars + TCB_BFULL + st, (unsigned)TC_B_CHUNK_BYTES);
+              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, (g >> 1) * TC_KC, (g & 1) * p.W * k + i * k + n * TC_N, bars + TCB_BFULL + st);
             }
           }
         }
@@ -231,36 +286,34 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         bool ok = true;
         const unsigned long long dA0 = tc_smem_desc(sA, 0), dB0 = tc_smem_desc(sB, 0);
         for (int m = 0; m < m_tiles && ok; ++m, ++um) {
-          const int halves = min(TC_MH, (b - m * TC_MH * TC_M + TC_M - 1) / TC_M);
           for (int n = 0; n < n_tiles && ok; ++n, ++iacc) {
             const int buf = iacc & 1;
             if (iacc >= 2) ok = mbar_wait_bounded(bars + TCB_ACCEMPTY + buf, ((iacc >> 1) - 1) & 1, p.wait_limit);
             if (!ok) break;
             tc_fence_after();
-            for (int g = 0; g < ngr && ok; ++g, ++ibc) {
+            const unsigned acc_col = tmem + (unsigned)(buf * TC_N);
+            for (int g = 0; g < 2 * nkc && ok; ++g, ++ibc) {
               const int st = ibc % TC_B_STAGES;
-              const int cnt_kc = min(TC_BG, nkc - g * TC_BG);
-              if (n == 0)
-                for (int c = 0; c < cnt_kc && ok; ++c) ok = mbar_wait_bounded(bars + TCB_AFULL + g * TC_BG + c, um & 1, p.wait_limit);
+              const int kc = g >> 1, lo_w = g & 1;
+              if (n == 0 && lo_w == 0) ok = mbar_wait_bounded(bars + TCB_AFULL + kc, um & 1, p.wait_limit);
               if (ok) ok = mbar_wait_bounded(bars + TCB_BFULL + st, (ibc / TC_B_STAGES) & 1, p.wait_limit);
               if (!ok) break;
               tc_fence_after();
-              for (int c = 0; c < cnt_kc; ++c) {
-                const int kc = g * TC_BG + c;
-                // operand descriptors: the base descriptor plus the chunk's offset in 16-byte units (the address field
-                // holds address >> 4 and shared memory is below 256 KB, so the sum stays inside the field)
-                const unsigned long long db = dB0 + (unsigned long long)((st * TC_BG + c) * (TC_B_CHUNK_BYTES >> 4));
-                for (int h = 0; h < halves; ++h) {
-                  const unsigned long long da = dA0 + (unsigned long long)((kc * TC_MH + h) * (TC_A_STAGE_BYTES >> 4));
+              // operand descriptors: the base descriptor plus the chunk's offset in 16-byte units (the address field
+              // holds address >> 4 and shared memory is below 256 KB, so the sum stays inside the field)
+              const unsigned long long db = dB0 + (unsigned long long)(st * (TC_B_CHUNK_BYTES >> 4));
+              const unsigned long long dah = dA0 + (unsigned long long)((kc * 2 + 0) * (TC_A_STAGE_BYTES >> 4));
+              const unsigned long long dal = dA0 + (unsigned long long)((kc * 2 + 1) * (TC_A_STAGE_BYTES >> 4));
 #pragma unroll
-                  for (int k4 = 0; k4 < TC_KC / 16; ++k4)
-                    tc_mma_bf16(tmem + (unsigned)((buf * TC_MH + h) * TC_N), da + (unsigned long long)(2 * k4), db + (unsigned long long)(2 * k4),
-                                idesc, (kc | k4) != 0);
-                }
+              for (int k4 = 0; k4 < TC_KC / 16; ++k4)                   // x_hi . w_hi  or  x_hi . w_lo
+                tc_mma_bf16(acc_col, dah + (unsigned long long)(2 * k4), db + (unsigned long long)(2 * k4), idesc, (g | k4) != 0);
+              if (lo_w == 0) {
+#pragma unroll
+                for (int k4 = 0; k4 < TC_KC / 16; ++k4)                 // x_lo . w_hi
+                  tc_mma_bf16(acc_col, dal + (unsigned long long)(2 * k4), db + (unsigned long long)(2 * k4), idesc, true);
               }
               tc_commit(bars + TCB_BEMPTY + st);                        // the ring slot is free when these MMAs have read it
-              if (n == n_tiles - 1)                                     // and so are the sample chunks after their last centre block
-                for (int c = 0; c < cnt_kc; ++c) tc_commit(bars + TCB_AEMPTY + g * TC_BG + c);
+              if (n == n_tiles - 1 && lo_w == 1) tc_commit(bars + TCB_AEMPTY + kc);   // and so is the sample chunk after its last centre block
             }
             tc_commit(bars + TCB_ACCFULL + buf);                        // the accumulator stage is complete
           }
@@ -268,15 +321,15 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         if (!ok) atomicExch(&misc[2], 1);
       }
     } else if (wid >= 4) {
-      // four warps read the accumulators: warp q of them owns TMEM lanes 32q .. 32q+31, i.e. one row of each part per thread
+      // four warps read the accumulators: warp q of them owns TMEM lanes 32q .. 32q+31, i.e. one row per thread
       const int quarter = wid & 3;
       unsigned iacc = it_acc;
       bool ok = true;
       for (int m = 0; m < m_tiles; ++m) {
-        const int r0 = m * TC_MH * TC_M + quarter * 32 + lane;     // the thread's row of part 0; part h is h * TC_M further
-        float m1[TC_MH][2], m2[TC_MH][2];                           // per row two independent (minimum, runner-up) pairs, kept over the centre blocks
-#pragma unroll
-        for (int h = 0; h < TC_MH; ++h) { m1[h][0] = m1[h][1] = INF; m2[h][0] = m2[h][1] = INF; }
+        const int r = m * TC_M + quarter * 32 + lane;              // the thread's row of the batch
+        const float xn = (r < b) ? __ldg(p.xnorm + row0 + r) : 0.f;
+        float m1[2], m2[2], m3[2];                                  // two independent sorted triples, kept over the centre blocks
+        m1[0] = m1[1] = m2[0] = m2[1] = m3[0] = m3[1] = INF;
         for (int n = 0; n < n_tiles; ++n, ++iacc) {
           const int buf = iacc & 1;
           if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bars + TCB_ACCFULL + buf, (iacc >> 1) & 1, p.wait_limit));
@@ -284,18 +337,15 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           tc_fence_after();
 #pragma unroll 1
           for (int c0 = 0; c0 < TC_N; c0 += 32) {
-            unsigned v[TC_MH][32];
-#pragma unroll
-            for (int h = 0; h < TC_MH; ++h) {
-              const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)((buf * TC_MH + h) * TC_N + c0);
-              asm volatile(
-                  "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                  : "=r"(v[h][0]), "=r"(v[h][1]), "=r"(v[h][2]), "=r"(v[h][3]), "=r"(v[h][4]), "=r"(v[h][5]), "=r"(v[h][6]), "=r"(v[h][7]),
-                    "=r"(v[h][8]), "=r"(v[h][9]), "=r"(v[h][10]), "=r"(v[h][11]), "=r"(v[h][12]), "=r"(v[h][13]), "=r"(v[h][14]), "=r"(v[h][15]),
-                    "=r"(v[h][16]), "=r"(v[h][17]), "=r"(v[h][18]), "=r"(v[h][19]), "=r"(v[h][20]), "=r"(v[h][21]), "=r"(v[h][22]), "=r"(v[h][23]),
-                    "=r"(v[h][24]), "=r"(v[h][25]), "=r"(v[h][26]), "=r"(v[h][27]), "=r"(v[h][28]), "=r"(v[h][29]), "=r"(v[h][30]), "=r"(v[h][31])
-                  : "r"(taddr) : "memory");
-            }
+            unsigned v[32];
+            const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)(buf * TC_N + c0);
+            asm volatile(
+                "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                  "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                  "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                  "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                : "r"(taddr) : "memory");
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             if (c0 + 32 == TC_N) {                        // last read of this accumulator stage: hand it back
               tc_fence_before();
@@ -309,34 +359,31 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
               const float cv[4] = {cn4.x, cn4.y, cn4.z, cn4.w};
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
-#pragma unroll
-                for (int h = 0; h < TC_MH; ++h) {
-                  const float sc = __uint_as_float(v[h][c + u]) + cv[u];
-                  // one logic op: the score's high bits, the block's and the column's index bits below them
-                  // (where both masks are set take the score, elsewhere the OR of the two index words)
-                  unsigned spb;
-                  asm("lop3.b32 %0, %1, %2, %3, 0xE6;" : "=r"(spb) : "r"(__float_as_uint(sc)), "r"(hi_or_base), "r"(~TC_INDEX_MASK | (unsigned)(c + u)));
-                  const float sp = __uint_as_float(spb);
-                  m2[h][u & 1] = fmaxf(m1[h][u & 1], fminf(m2[h][u & 1], sp));
-                  m1[h][u & 1] = fminf(m1[h][u & 1], sp);
-                }
+                // squared distance ||x||^2 - 2 x.w_a + ||w_a||^2 (fp32 adds), then one logic op: the value's high
+                // bits, the block's and the column's index bits below them
+                const float d2 = (__uint_as_float(v[c + u]) + cv[u]) + xn;
+                unsigned spb;
+                asm("lop3.b32 %0, %1, %2, %3, 0xE6;" : "=r"(spb) : "r"(__float_as_uint(d2)), "r"(hi_or_base), "r"(~TC_INDEX_MASK | (unsigned)(c + u)));
+                tc_top3_insert(m1[u & 1], m2[u & 1], m3[u & 1], __uint_as_float(spb));
               }
             }
           }
         }
-#pragma unroll
-        for (int h = 0; h < TC_MH; ++h) {
-          const int r = r0 + h * TC_M;
-          if (ok && r < b)
-            __stcg(top2 + r, make_float2(fminf(m1[h][0], m1[h][1]), fminf(fmaxf(m1[h][0], m1[h][1]), fminf(m2[h][0], m2[h][1]))));
+        if (ok && r < b) {
+          // merge the two sorted triples: the three smallest of the six
+          float a1 = m1[0], a2 = m2[0], a3 = m3[0];
+          tc_top3_insert(a1, a2, a3, m1[1]);
+          tc_top3_insert(a1, a2, a3, m2[1]);
+          tc_top3_insert(a1, a2, a3, m3[1]);
+          __stcg(top3 + r, make_float4(a1, a2, a3, 0.f));
         }
       }
       if (!ok && lane == 0) atomicExch(&misc[2], 1);
     }
     it_m += (unsigned)m_tiles;
-    it_bc += (unsigned)(m_tiles * n_tiles * ngr);
+    it_bc += (unsigned)(m_tiles * n_tiles * 2 * nkc);
     it_acc += (unsigned)(n_tiles * m_tiles);
-    if (tid == 0) misc[1] = 0;
+    if (tid == 0) { misc[1] = 0; misc[5] = 0; }
     for (int a = tid; a < k; a += TC_THREADS) cnt[a] = 0;
     tc_fence_before();
     __syncthreads();
@@ -348,33 +395,38 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     for (int a = lane; a < k; a += 32) wmax2 = fmaxf(wmax2, cn[a]);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) wmax2 = fmaxf(wmax2, __shfl_xor_sync(0xffffffffu, wmax2, o));
-    // BF16 rounding (2^-8 relative) of both operands: |error of -2 x.w| <= 2 * 2^-7 * 1.004 * ||x|| ||w||; index bits: 2^10 ulp of the score
+    // Error of a computed squared distance (see the file header and the tolerance note of the library):
+    //   terms left out of the split product          6 * 2^-18 ||x|| ||w||
+    //   fp32 accumulation of 3 d / 16 partial sums    (3 d / 16 + 1) * 2^-22 ||x|| ||w||     (each step at most one ulp of a sum <= 2 ||x|| ||w||)
+    //   the two fp32 adds of the norms                3 * 2^-24 (||x||^2 + ||w||^2 + 2 ||x|| ||w||)
+    // with a quarter on top; the index bits cost 2^10 ulp <= 2^-13 of the value itself, applied relative to the values compared.
     const float xw = sqrtf(p.xmax2 * wmax2);
-    const float tau = 2.f * (0.0157f * xw + 2.45e-4f * (wmax2 + 2.f * xw));
+    const float err = 1.25f * ((2.289e-5f + (float)(3 * d / 16 + 1) * 2.384e-7f) * xw + 1.79e-7f * (p.xmax2 + wmax2 + 2.f * xw));
+    auto inside = [&](float lo, float hi_) { return (hi_ - lo) <= 2.f * err + 2.4415e-4f * fmaxf(fabsf(lo), fabsf(hi_)); };
     // Scratch for the rest of the step lives in the sample ring, which is idle until the next step's loads.
     int* wcnt = reinterpret_cast<int*>(sA);                                   // [TC_WARPS][k] rows of a centre in a warp's row block
     unsigned short* lrank = reinterpret_cast<unsigned short*>(sA + (size_t)TC_WARPS * k * 4);   // [b] rank of a row among its warp's rows of the centre
     unsigned short* order = flagged;                                          // [b] rows grouped by centre, ascending inside a group
-    const int sub = lane >> 3, l8 = lane & 7;                                 // eight lanes share a row or a centre
-    const int nq = d / 32;
 
-    // ---- decide: rows whose two best scores are closer than the bound go on a list; the others take the minimum ----
+    // ---- decide: the minimum, unless the runner-up lies inside the bound (settle the pair) or the third does too (scan all) ----
     for (int e = tid; e < TC_WARPS * k; e += TC_THREADS) wcnt[e] = 0;
     for (int r = tid; r < b; r += TC_THREADS) {
-      const float2 s = __ldcg(top2 + r);
-      const int i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK);
-      best[r] = (unsigned short)i1;
-      if (k > 1 && (s.y - s.x) <= tau) order[atomicAdd(&misc[1], 1)] = (unsigned short)r;
+      const float4 s = __ldcg(top3 + r);
+      best[r] = (unsigned short)(__float_as_uint(s.x) & TC_INDEX_MASK);
+      if (k > 1 && inside(s.x, s.y)) {
+        if (k > 2 && inside(s.x, s.z)) order[b - 1 - atomicAdd(&misc[5], 1)] = (unsigned short)r;
+        else order[atomicAdd(&misc[1], 1)] = (unsigned short)r;
+      }
     }
     __syncthreads();
-    // ---- listed rows are settled between their two candidates with fp32 inputs and fp64 sums: eight lanes per
+    // ---- listed pairs are settled between their two candidates with fp32 inputs and fp64 sums: eight lanes per
     //      row (lane l8 holds dimensions 4*l8 + 32*q), a warp settles four rows at a time ----
     {
       const int nflag = misc[1];
       auto settle_load = [&](int f, float4 (&xv)[TC_MAX_D / 32], float4 (&a1)[TC_MAX_D / 32], float4 (&a2)[TC_MAX_D / 32], int& r,
                              int& i1, int& i2) {
         r = (f < nflag) ? (int)order[f] : -1;
-        const float2 s = (r >= 0) ? __ldcg(top2 + r) : make_float2(0.f, 0.f);
+        const float4 s = (r >= 0) ? __ldcg(top3 + r) : make_float4(0.f, 0.f, 0.f, 0.f);
         i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK);
         i2 = (int)(__float_as_uint(s.y) & TC_INDEX_MASK);
         const float* x = p.X + (size_t)(row0 + max(r, 0)) * d + 4 * l8;
@@ -431,6 +483,59 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         int ra, ia1, ia2;
         settle_load(f0, xa, pa, qa, ra, ia1, ia2);
         settle_finish(xa, pa, qa, ra, ia1, ia2);
+      }
+    }
+    // ---- rows with three or more candidates: a warp per row looks at every centre, lanes over centres, direct
+    //      differences in fp32; if the two smallest are still within rounding of each other, again in fp64 ----
+    {
+      const int nwide = misc[5];
+      for (int f = wid; f < nwide; f += TC_WARPS) {            // warp-uniform trip count
+        const int r = (int)order[b - 1 - f];
+        const float* xr = p.X + (size_t)(row0 + r) * d;
+        float fd1 = INF, fd2 = INF;
+        int fi = 0x7fffffff;
+        for (int a = lane; a < k; a += 32) {
+          const float* wa = wglob + (size_t)a * d;
+          float sacc = 0.f;
+          for (int j = 0; j < d; j += 4) {
+            const float4 xv4 = __ldg(reinterpret_cast<const float4*>(xr + j));
+            const float4 wv4 = *reinterpret_cast<const float4*>(wa + j);
+            float u;
+            u = xv4.x - wv4.x; sacc = fmaf(u, u, sacc); u = xv4.y - wv4.y; sacc = fmaf(u, u, sacc);
+            u = xv4.z - wv4.z; sacc = fmaf(u, u, sacc); u = xv4.w - wv4.w; sacc = fmaf(u, u, sacc);
+          }
+          if (sacc < fd1) { fd2 = fd1; fd1 = sacc; fi = a; } else if (sacc < fd2) { fd2 = sacc; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const float o1 = __shfl_xor_sync(0xffffffffu, fd1, o);
+          const float o2 = __shfl_xor_sync(0xffffffffu, fd2, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, fi, o);
+          const bool take = (o1 < fd1) || (o1 == fd1 && oi < fi);
+          fd2 = fminf(take ? fd1 : o1, fminf(fd2, o2));
+          if (take) { fd1 = o1; fi = oi; }
+        }
+        int bi = fi;
+        if (fd2 - fd1 <= (float)(4 * TC_MAX_D + 16) * 5.9604645e-8f * fd2) {
+          double bd = 1e300;
+          bi = 0x7fffffff;
+          for (int a = lane; a < k; a += 32) {
+            const float* wa = wglob + (size_t)a * d;
+            double sacc = 0.0;
+            for (int j = 0; j < d; ++j) {
+              const double u = (double)__ldg(xr + j) - (double)wa[j];
+              sacc = fma(u, u, sacc);
+            }
+            if (sacc < bd) { bd = sacc; bi = a; }                // ascending a: the lowest index keeps a tie
+          }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const double od = __shfl_xor_sync(0xffffffffu, bd, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (od < bd || (od == bd && oi < bi)) { bd = od; bi = oi; }
+          }
+        }
+        if (lane == 0) best[r] = (unsigned short)bi;
       }
     }
     __syncthreads();
@@ -502,19 +607,6 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
 
     // ---- Eq. 9 and the update: eight lanes per centre add its rows (fp32 master, ascending row order);
     //      plain step: w <- w - eps (n w - S) / b at once; otherwise S goes to the sum buffer for the general tail ----
-    auto refresh = [&](int a, const float4 (&w4)[TC_MAX_D / 32]) {           // bf16(-2w), ||w||^2 of one centre
-      float sq = 0.f;
-#pragma unroll
-      for (int q = 0; q < TC_MAX_D / 32; ++q) {
-        if (q < nq) {
-          sq = fmaf(w4[q].x, w4[q].x, sq); sq = fmaf(w4[q].y, w4[q].y, sq); sq = fmaf(w4[q].z, w4[q].z, sq); sq = fmaf(w4[q].w, w4[q].w, sq);
-          __nv_bfloat16* o = wbf + (size_t)a * d + 4 * l8 + 32 * q;
-          *reinterpret_cast<__nv_bfloat162*>(o) = __floats2bfloat162_rn(-2.f * w4[q].x, -2.f * w4[q].y);
-          *reinterpret_cast<__nv_bfloat162*>(o + 2) = __floats2bfloat162_rn(-2.f * w4[q].z, -2.f * w4[q].w);
-        }
-      }
-      return sq;
-    };
     {
       const int* start = reinterpret_cast<const int*>(sB);
       for (int a0 = (wid * 4) ; a0 < k; a0 += TC_WARPS * 4) {
@@ -560,20 +652,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       __syncthreads();
       step_tail<kDet>(p, i, t, wglob, d, gsum, cnt, nullptr, ts, false);
       __syncthreads();
-      for (int a0 = wid * 4; a0 < k; a0 += TC_WARPS * 4) {
-        const int a = a0 + sub;
-        float sq = 0.f;
-        if (a < k) {
-          float4 w4[TC_MAX_D / 32];
-#pragma unroll
-          for (int q = 0; q < TC_MAX_D / 32; ++q)
-            if (q < nq) w4[q] = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q);
-          sq = refresh(a, w4);
-        }
-#pragma unroll
-        for (int o = 1; o < 8; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-        if (a < k && l8 == 0) cn[a] = sq;
-      }
+      refresh_all();
     } else {
       unsigned long long n_sent = 0;
       if (put_now) {
@@ -590,7 +669,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         if (n_sent) atomicAdd(st + ST_SENT, n_sent);
       }
     }
-    asm volatile("fence.proxy.async;" ::: "memory");      // the refreshed bf16(-2w) is read by the next step's TMA
+    asm volatile("fence.proxy.async;" ::: "memory");      // the refreshed w_hi, w_lo are read by the next step's TMA
     __syncthreads();
   }
 
@@ -602,7 +681,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   }
   tc_fence_before();
   __syncthreads();
-  if (wid == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  if (wid == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TC_TMEM_COLS) : "memory");
 }
 
 }  // namespace asgd

@@ -12,7 +12,7 @@ import torch
 import paper_1505_04956_b200 as pkg
 from paper_1505_04956_b200 import inputs
 from oracle import asgd_oracle as orc
-from tests.gpu_util import CENTRE_TOL, CENTRE_TOL_BF16, decided
+from tests.gpu_util import CENTRE_TOL, decided
 
 pytestmark = pytest.mark.gpu
 
@@ -51,11 +51,24 @@ def test_first_rounds_at_full_size_match_the_oracle(name):
     cpu = orc.Oracle(Xc, w0.cpu().numpy(), W=wl.W, b=wl.b, eps=wl.eps, comm_interval=wl.comm_interval, fanout=wl.fanout,
                      shuffle=0, seed=wl.seed, threads=orc.max_threads())
     assert cpu.H == rounds * wl.b
-    ctx.step(rounds)
+    # all rounds but the last on both sides; then the last round from the oracle's states, so that the rounding
+    # differences of the earlier rounds cannot move a sample across a bisecting plane and the assignments of the
+    # last round compare exactly (the receive buffers keep their own rounding: it only enters the centres)
+    if rounds > 1:
+        ctx.step(rounds - 1)
+        ctx.sync()
+        cpu.rounds(rounds - 1)
+        worst = 0.0
+        for i in range(wl.W):
+            g = ctx.get_state(i).cpu().numpy().astype(np.float64)
+            c = cpu.state(i).astype(np.float64)
+            worst = max(worst, float(np.linalg.norm(g - c) / np.linalg.norm(c)))
+        assert worst < CENTRE_TOL, (name, "before the last round", worst)
+        for i in range(wl.W):
+            ctx.set_state(i, torch.from_numpy(cpu.state(i)).to(X.device))
+    ctx.step(1)
     ctx.sync()
-    cpu.rounds(rounds)
-    bf16 = ctx.path_name() == "tcgen05-bf16"
-    tol = CENTRE_TOL_BF16 if bf16 else CENTRE_TOL
+    cpu.rounds(1)
     got_assign = ctx.get_assign().cpu().numpy()
     sample = np.unique(np.linspace(0, wl.W - 1, 64).astype(int))
     worst = 0.0
@@ -63,20 +76,15 @@ def test_first_rounds_at_full_size_match_the_oracle(name):
         g = ctx.get_state(i).cpu().numpy().astype(np.float64)
         c = cpu.state(i).astype(np.float64)
         worst = max(worst, float(np.linalg.norm(g - c) / np.linalg.norm(c)))
-    assert worst < tol, (name, worst)
+    assert worst < CENTRE_TOL, (name, worst)
     for i in sample:
         gs, cs = ctx.get_stats(int(i)), cpu.stats(int(i))
         for key in ("steps", "sent", "received", "overwritten"):
             assert gs[key] == cs[key], (name, i, key, gs, cs)
         tr = cpu.last_step(int(i))
         ok = decided(tr["d1"], tr["d2"])
-        agree = (got_assign[i] == tr["assign"]) | ~ok
-        if bf16 or rounds > 1:
-            # after more than one round the states differ by rounding, BF16 scores by their error bound:
-            # a handful of samples close to a bisecting plane may fall on the other side
-            assert agree.mean() > 0.995, (name, i, agree.mean())
-        else:
-            assert agree.all(), (name, i)
+        assert (got_assign[i][ok] == tr["assign"][ok]).all(), (name, i)
+        assert ok.mean() > 0.99
     ctx.destroy()
 
 

@@ -7,7 +7,7 @@ import torch
 
 import paper_1505_04956_b200 as pkg
 from oracle import asgd_oracle as orc
-from tests.gpu_util import CENTRE_TOL, CENTRE_TOL_BF16, PARITY_WORKLOADS, Pair, decided, scaled
+from tests.gpu_util import CENTRE_TOL, PARITY_WORKLOADS, Pair, decided, scaled
 
 pytestmark = pytest.mark.gpu
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
@@ -72,27 +72,17 @@ def test_single_step_assignments_bit_exact(name):
     pr.rounds(1)
     pr.gpu.sync()
     got = pr.gpu.get_assign().cpu().numpy()
-    bf16 = pr.gpu.path_name() == "tcgen05-bf16"
     checked = 0
     for i in range(wl.W):
         tr = pr.cpu.last_step(i)
         ok = decided(tr["d1"], tr["d2"])
-        if bf16:
-            # BF16 operands: a score is off by at most 2 * 2^-7 * 1.004 * ||x|| ||w|| (+ index bits); the kernel settles
-            # the two best exactly, so only samples with a third centre inside that bound may differ
-            w = pr.cpu.state(i).astype(np.float64)
-            xw = np.sqrt((pr.Xh.astype(np.float64) ** 2).sum(1).max() * (w ** 2).sum(1).max())
-            tau = 2 * (0.0157 * xw + 2.45e-4 * ((w ** 2).sum(1).max() + 2 * xw))
-            wrong = ok & (got[i] != tr["assign"])
-            assert wrong.mean() < 0.01, (name, i, wrong.mean())
-            assert ((tr["d2"] - tr["d1"])[wrong] <= tau).all()
-        else:
-            assert (got[i][ok] == tr["assign"][ok]).all(), (name, i)
-            # counts n_k of Eq. 9: equal to the oracle's per centre, up to the undecided rows either side gave it
-            und = ~ok
-            slack = np.bincount(got[i][und], minlength=wl.k) + np.bincount(tr["assign"][und], minlength=wl.k)
-            diff = np.abs(np.bincount(got[i], minlength=wl.k) - tr["counts"])
-            assert (diff <= slack).all(), (name, i, diff, slack)
+        # every path, the split-precision tensor-core one included: the nearest centre of Eq. 8, exactly
+        assert (got[i][ok] == tr["assign"][ok]).all(), (name, i)
+        # counts n_k of Eq. 9: equal to the oracle's per centre, up to the undecided rows either side gave it
+        und = ~ok
+        slack = np.bincount(got[i][und], minlength=wl.k) + np.bincount(tr["assign"][und], minlength=wl.k)
+        diff = np.abs(np.bincount(got[i], minlength=wl.k) - tr["counts"])
+        assert (diff <= slack).all(), (name, i, diff, slack)
         checked += int(ok.sum())
     assert checked >= 0.99 * wl.W * wl.b
     assert pr.max_rel_l2() < pr.centre_tol()
