@@ -273,7 +273,7 @@ def main():
                         "traffic": None, "peak_kind": "SMs x 128 fp32 lanes x 2 x max SM clock", "kernel": ctx.path_name(),
                         "launch_ms": launch_ms, "algorithmic_flops_per_launch": flops,
                         "hbm_GBs": achieved}
-    elif ctx.path_name() == "tcgen05-bf16":
+    elif ctx.path_name().startswith("tcgen05"):
         # bound by the tensor pipe: the 2*k*d flops per sample of the -2 X W^T contraction against the measured
         # sustained BF16 rate (the kernel is timed inside a long launch)
         tpeak, tkind = 1400.0, "fallback (sustained)"

@@ -49,8 +49,12 @@ typedef enum asgd_status {
 enum {
   ASGD_PATH_AUTO = 0,
   ASGD_PATH_FP32 = 1,       /* CUDA cores, fp32 (the specialised kernel for the shape, if any) */
-  ASGD_PATH_TC_BF16 = 3,    /* tcgen05, BF16 operands in two terms each (x_hi + x_lo, w_hi + w_lo; */
-                            /* three products per score), fp32 accumulate                    */
+  ASGD_PATH_TC_FP16 = 2,    /* tcgen05, FP16 operands, fp32 accumulate; rows the rounding bound cannot   */
+                            /* decide are decided exactly afterwards.  Needs 8 max ||x|| < 65504       */
+                            /* (ASGD_EUNSUPPORTED otherwise; AUTO then takes an fp32 path)              */
+  ASGD_PATH_TC_BF16 = 3,    /* tcgen05, BF16 operands in two terms each (x_hi + x_lo, w_hi + w_lo;     */
+                            /* three products per score), fp32 accumulate: any fp32 range, same exact  */
+                            /* decisions, three times the tensor work                                  */
   ASGD_PATH_FP32_GENERAL = 4 /* CUDA cores, fp32, the shape-independent kernel                */
 };
 

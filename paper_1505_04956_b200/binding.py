@@ -12,7 +12,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libasgd.so")
 
 ASGD_OK, ASGD_EINVAL, ASGD_ENOMEM, ASGD_ECUDA, ASGD_EUNSUPPORTED, ASGD_ETIMEOUT = 0, -1, -2, -3, -4, -5
-PATH_AUTO, PATH_FP32, PATH_TC_BF16, PATH_FP32_GENERAL = 0, 1, 3, 4
+PATH_AUTO, PATH_FP32, PATH_TC_FP16, PATH_TC_BF16, PATH_FP32_GENERAL = 0, 1, 2, 3, 4
 
 EXPORTS = (
     "asgd_workspace_bytes", "asgd_init", "asgd_step", "asgd_run", "asgd_get_state", "asgd_set_state",

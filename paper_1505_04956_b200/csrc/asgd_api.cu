@@ -21,7 +21,7 @@ using namespace asgd;
 
 namespace {
 
-enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2, P_TC_BF16 = 3 };
+enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2, P_TC_BF16 = 3, P_TC_FP16 = 4 };
 
 // (d, k) shapes the streaming path is compiled for
 #define ASGD_STREAM_SHAPES(X) X(10, 10) X(16, 16) X(4, 5) X(2, 3)
@@ -50,9 +50,7 @@ bool config_ok(const asgd_config* c) {
   if (c->comm_interval < 0 || c->fanout < 0 || c->fanout > c->W - 1 || c->fanout > MAX_FANOUT) return false;
   if (c->slots < 1 || c->slots > MAX_SLOTS) return false;
   if (c->partial_rows < 0 || c->partial_rows > c->k) return false;
-  if (c->dist_path != ASGD_PATH_AUTO && c->dist_path != ASGD_PATH_FP32 && c->dist_path != ASGD_PATH_TC_BF16 &&
-      c->dist_path != ASGD_PATH_FP32_GENERAL)
-    return false;
+  if (c->dist_path < ASGD_PATH_AUTO || c->dist_path > ASGD_PATH_FP32_GENERAL) return false;
   if ((long long)c->k * c->d > (1ll << 28)) return false;
   const long long H = c->N / c->W;
   if (H < c->b) return false;
@@ -63,7 +61,7 @@ bool config_ok(const asgd_config* c) {
 // shapes the tensor-core path takes: d a multiple of 64 up to 256, more centres than the tiled path holds
 bool tc_eligible(const asgd_config* c) {
   return c->d % TC_KC == 0 && c->d <= TC_MAX_D && c->k > 128 && c->k <= TC_MAX_K && c->b >= TC_M && c->b <= TC_MAX_B &&
-         tc_smem_bytes(c->k, c->d, c->b) <= kMaxDynSmem;
+         tc_smem_bytes(c->k, c->d, c->b, 1) <= kMaxDynSmem && tc_smem_bytes(c->k, c->d, c->b, 3) <= kMaxDynSmem;
 }
 
 Layout make_layout(const asgd_config* c) {
@@ -91,11 +89,14 @@ Layout make_layout(const asgd_config* c) {
   L.eval_partial = take((size_t)kEvalBlocks * 8);
   L.tmp_state = take(kd_pad * 4);
   L.xmax = take(64);
-  const bool tc = tc_eligible(c) && (c->dist_path == ASGD_PATH_TC_BF16 || c->dist_path == ASGD_PATH_AUTO);
-  L.wbf = take(tc ? 2 * W * kd * 2 : 4);
+  // tensor-core path: 16-bit copies of -2w and of the samples (one FP16 term, or the two BF16 terms), the three
+  // best per row, the row norms
+  const bool tc = tc_eligible(c) && (c->dist_path == ASGD_PATH_TC_BF16 || c->dist_path == ASGD_PATH_TC_FP16 || c->dist_path == ASGD_PATH_AUTO);
+  const bool two_terms = tc && c->dist_path == ASGD_PATH_TC_BF16;
+  L.wbf = take(tc ? (two_terms ? 2 : 1) * W * kd * 2 : 4);
   L.top2 = take(tc ? W * (size_t)c->b * 16 : 4);
   L.xbf = take(tc ? (size_t)c->N * c->d * 2 : 4);
-  L.xbl = take(tc ? (size_t)c->N * c->d * 2 : 4);
+  L.xbl = take(two_terms ? (size_t)c->N * c->d * 2 : 4);
   L.xnorm = take(tc ? (size_t)c->N * 4 : 4);
   L.total = off;
   return L;
@@ -119,6 +120,7 @@ struct asgd_ctx {
   int last_cuda;
   int sm_count;
   const void* xbf_user;   // caller's bf16 copy of X, or nullptr
+  int no_tc;              // AUTO: the samples do not fit FP16, take an fp32 path
   CUtensorMap mapXh, mapXl, mapW; // tensor-core path: BF16 terms of the samples [N][d] each, of -2w [2*W*k][d]
 };
 
@@ -183,7 +185,7 @@ void tiled_launch(asgd_ctx* c, bool det, long long steps) {
     asgd_tiled_kernel<D, KP, WS, WK, MINB, false><<<c->grid, 32 * WS * WK, c->smem_bytes, c->stream>>>(c->p, steps);
 }
 
-bool encode_bf16_map(CUtensorMap* map, const void* base, unsigned long long rows, unsigned long long cols, unsigned box_rows) {
+bool encode_16bit_map(CUtensorMap* map, bool fp16, const void* base, unsigned long long rows, unsigned long long cols, unsigned box_rows) {
   static PFN_cuTensorMapEncodeTiled encode = nullptr;
   if (!encode) {
     void* fn = nullptr;
@@ -195,7 +197,7 @@ bool encode_bf16_map(CUtensorMap* map, const void* base, unsigned long long rows
   cuuint64_t strides[1] = {cols * 2};
   cuuint32_t box[2] = {(cuuint32_t)TC_KC, box_rows};
   cuuint32_t estr[2] = {1, 1};
-  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  return encode(map, fp16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -217,28 +219,45 @@ int compute_xmax2(asgd_ctx* c) {
   return ASGD_OK;
 }
 
+// Tensor-core path set-up: 16-bit copies of X, row norms, max ||x||^2, tensor maps.  Returns ASGD_EUNSUPPORTED when
+// the one-term FP16 format was asked for and the samples do not fit FP16's range.
 int tc_prepare(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
   Params& p = c->p;
-  c->smem_bytes = tc_smem_bytes(cfg.k, cfg.d, cfg.b);
-  CU(c, cudaFuncSetAttribute(asgd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
-  CU(c, cudaFuncSetAttribute(asgd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  const bool fp16 = (c->path == P_TC_FP16);
+  c->smem_bytes = tc_smem_bytes(cfg.k, cfg.d, cfg.b, fp16 ? 1 : 3);
+  if (fp16) {
+    CU(c, cudaFuncSetAttribute(asgd_tc_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+    CU(c, cudaFuncSetAttribute(asgd_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  } else {
+    CU(c, cudaFuncSetAttribute(asgd_tc_kernel<true, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+    CU(c, cudaFuncSetAttribute(asgd_tc_kernel<false, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  }
   p.wbf = c->ws + c->L.wbf;
   p.top2 = (float*)(c->ws + c->L.top2);
-  // x = x_hi + x_lo in BF16: x_hi is the caller's copy when one was given, x_lo the rounded residue either way
-  const void* xbf = c->xbf_user ? c->xbf_user : (const void*)(c->ws + c->L.xbf);
-  void* xbl = c->ws + c->L.xbl;
-  tc_split_x_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, (const __nv_bfloat16*)c->xbf_user,
-                                                             c->xbf_user ? nullptr : (__nv_bfloat16*)(c->ws + c->L.xbf),
-                                                             (__nv_bfloat16*)xbl, (size_t)cfg.N * cfg.d);
+  { const int rc = compute_xmax2(c); if (rc != ASGD_OK) return rc; }
+  // |x_j| <= ||x||, and a centre stays inside the hull of the samples and the initial state: keep a factor 4 of room
+  if (fp16 && !(8.f * sqrtf(p.xmax2) < 65504.f)) return ASGD_EUNSUPPORTED;
+  const void* xh = nullptr;
+  const void* xl = nullptr;
+  if (fp16) {
+    tc_half_x_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, (__half*)(c->ws + c->L.xbf), (size_t)cfg.N * cfg.d);
+    xh = xl = c->ws + c->L.xbf;
+  } else {
+    // x = x_hi + x_lo in BF16: x_hi is the caller's copy when one was given, x_lo the rounded residue either way
+    xh = c->xbf_user ? c->xbf_user : (const void*)(c->ws + c->L.xbf);
+    xl = c->ws + c->L.xbl;
+    tc_split_x_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, (const __nv_bfloat16*)c->xbf_user,
+                                                               c->xbf_user ? nullptr : (__nv_bfloat16*)(c->ws + c->L.xbf),
+                                                               (__nv_bfloat16*)(c->ws + c->L.xbl), (size_t)cfg.N * cfg.d);
+  }
   tc_row_norms_kernel<<<c->sm_count * 8, 256, 0, c->stream>>>(p.X, cfg.N, cfg.d, (float*)(c->ws + c->L.xnorm));
   c->launches += 2;
   CU(c, cudaGetLastError());
   p.xnorm = (const float*)(c->ws + c->L.xnorm);
-  { const int rc = compute_xmax2(c); if (rc != ASGD_OK) return rc; }
-  if (!encode_bf16_map(&c->mapXh, xbf, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
-  if (!encode_bf16_map(&c->mapXl, xbl, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
-  if (!encode_bf16_map(&c->mapW, p.wbf, 2ull * cfg.W * cfg.k, (unsigned long long)cfg.d, TC_N)) return ASGD_ECUDA;
+  if (!encode_16bit_map(&c->mapXh, fp16, xh, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
+  if (!encode_16bit_map(&c->mapXl, fp16, xl, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
+  if (!encode_16bit_map(&c->mapW, fp16, p.wbf, (fp16 ? 1ull : 2ull) * cfg.W * cfg.k, (unsigned long long)cfg.d, (unsigned)tc_block_n(fp16 ? 1 : 3))) return ASGD_ECUDA;
   return ASGD_OK;
 }
 
@@ -247,9 +266,15 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
   switch (c->path) {
     case P_TC_BF16:
       if (det)
-        asgd_tc_kernel<true><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
+        asgd_tc_kernel<true, 3><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
       else
-        asgd_tc_kernel<false><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
+        asgd_tc_kernel<false, 3><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
+      break;
+    case P_TC_FP16:
+      if (det)
+        asgd_tc_kernel<true, 1><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
+      else
+        asgd_tc_kernel<false, 1><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
       break;
     case P_TILED: {
       int idx = 0;
@@ -278,9 +303,10 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
 
 int resolve_path(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
-  if (cfg.dist_path == ASGD_PATH_TC_BF16 || (cfg.dist_path == ASGD_PATH_AUTO && tc_eligible(&cfg))) {
+  if (cfg.dist_path == ASGD_PATH_TC_BF16 || cfg.dist_path == ASGD_PATH_TC_FP16 ||
+      (cfg.dist_path == ASGD_PATH_AUTO && tc_eligible(&cfg) && !c->no_tc)) {
     if (!tc_eligible(&cfg)) return ASGD_EUNSUPPORTED;
-    c->path = P_TC_BF16;
+    c->path = (cfg.dist_path == ASGD_PATH_TC_BF16) ? P_TC_BF16 : P_TC_FP16;
     c->state_on_chip = 0;
     return ASGD_OK;                       // device-side set-up (tc_prepare) runs once the workspace is cleared
   }
@@ -373,6 +399,7 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   c->last_cuda = 0;
   c->sm_count = prop.multiProcessorCount;
   c->xbf_user = X_bf16_dev;
+  c->no_tc = 0;
 
   Params& p = c->p;
   p.X = X_dev; p.N = cfg->N; p.d = cfg->d; p.k = cfg->k; p.W = cfg->W; p.b = cfg->b; p.eps = cfg->eps;
@@ -412,8 +439,13 @@ int asgd_init(asgd_ctx** out, const asgd_config* cfg, const float* X_dev, const 
   if (e != cudaSuccess) { delete c; return ASGD_ECUDA; }
   broadcast_state_kernel<<<256, 256, 0, c->stream>>>(p.state, w0_dev, p.W, p.kd, p.kd_pad);
   c->launches += 1;
-  if (c->path == P_TC_BF16) {
+  if (c->path == P_TC_BF16 || c->path == P_TC_FP16) {
     rc = tc_prepare(c);
+    if (rc == ASGD_EUNSUPPORTED && cfg->dist_path == ASGD_PATH_AUTO) {      // samples outside FP16's range: an fp32 path instead
+      c->no_tc = 1;
+      rc = resolve_path(c);
+      if (rc == ASGD_OK && (c->path == P_STREAM || c->path == P_TILED)) rc = compute_xmax2(c);
+    }
     if (rc != ASGD_OK) { delete c; return rc; }
   } else if (c->path == P_STREAM || c->path == P_TILED) {
     rc = compute_xmax2(c);
@@ -600,7 +632,8 @@ const char* asgd_path_name(const asgd_ctx* c) {
     case P_GENERIC: return c->state_on_chip ? "fp32-generic" : "fp32-generic-offchip";
     case P_STREAM: return "fp32-stream";
     case P_TILED: return "fp32-tiled";
-    case P_TC_BF16: return "tcgen05-bf16";
+    case P_TC_BF16: return "tcgen05-bf16x3";
+    case P_TC_FP16: return "tcgen05-fp16";
     default: return "unknown";
   }
 }

@@ -8,6 +8,13 @@
 // the scores are good to about 16 bits, the Eq. 8 decision falls to the exact fp32 comparison only for a fraction
 // of a percent of the rows, and every such row is decided among ALL centres that the bound cannot rule out.
 //
+// Two operand formats (template parameter kTerms):
+//   1  FP16, one term per operand: x and -2w rounded to FP16 (11 significant bits), one product.  A score is good to
+//      2^-10 ||x|| ||w||; the rows whose candidates lie closer than that (a few per cent) are decided exactly afterwards.
+//      Needs |x|, |2w| inside FP16's range.
+//   3  BF16, two terms per operand, three products as above (about 16 bits): any fp32 range, three times the tensor work
+//      and twice the operand bytes.
+//
 // One worker = one thread block = one SM.  Warp roles while the scores are computed:
 //   warp 0   one lane issues the TMA loads: a 128-row sample tile (hi and lo) in 128-byte-swizzled K-chunks of 64,
 //            resident while all centre blocks pass, and 128-centre blocks of w_hi, w_lo through a ring of
@@ -25,6 +32,7 @@
 
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "asgd_step_tail.cuh"
 #include "asgd_stream.cuh"   // mbarrier helpers
@@ -33,25 +41,27 @@ namespace asgd {
 
 constexpr int TC_THREADS = 256;
 constexpr int TC_WARPS = TC_THREADS / 32;
-constexpr int TC_M = 128, TC_N = 128, TC_KC = 64;        // one MMA's output tile; K chunk = 64 bf16 = one swizzled 128-byte row
+constexpr int TC_M = 128, TC_KC = 64;                    // rows of an MMA's output tile; K chunk = 64 16-bit numbers = one swizzled 128-byte row
+// centres per block (the MMA's N): 256 with one term per operand, 128 with two (the sample tile then takes twice the room)
+__host__ __device__ constexpr int tc_block_n(int terms) { return terms == 1 ? 256 : 128; }
 constexpr int TC_A_STAGES = 4;                            // K chunks of the resident sample tile (d <= 256), each with a hi and a lo part
 constexpr int TC_B_STAGES = 4;                            // ring slots for the centre blocks (one K chunk of w_hi or of w_lo each)
 constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB per part
-constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;       // 16 KB
-constexpr int TC_TMEM_COLS = 2 * TC_N;                    // two accumulator stages
 constexpr int TC_SUM_ROWS = 4;                            // sample rows a centre's adders keep in flight
 constexpr int TC_MAX_K = 1024, TC_MAX_D = 256, TC_MAX_B = 4096;
 constexpr unsigned TC_INDEX_MASK = 1023u;
+constexpr int TC_SCAN_ROWS = 16;                          // rows the full scan measures at a time
 constexpr float TC_FAR = 1e30f;                          // stands for ||w_a||^2 of the padding centres
 
 struct TcSmem {
   size_t B, A, cn, cnt, best, flagged, bars, misc, tail, total;
-  __host__ __device__ TcSmem(int k, int d, int b) {
+  __host__ __device__ TcSmem(int k, int d, int b, int terms) {
+    const int nb = tc_block_n(terms);
     size_t off = 0;
     auto take = [&](size_t bytes, size_t align) { off = (off + align - 1) / align * align; size_t o = off; off += bytes; return o; };
-    A = take((size_t)TC_A_STAGES * 2 * TC_A_STAGE_BYTES, 1024);       // [K chunk][hi, lo]; also the scratch of the grouping phase
-    B = take((size_t)TC_B_STAGES * TC_B_CHUNK_BYTES, 1024);
-    cn = take((size_t)((k + TC_N - 1) / TC_N) * TC_N * 4, 16);
+    A = take((size_t)TC_A_STAGES * (terms == 3 ? 2 : 1) * TC_A_STAGE_BYTES, 1024);   // [K chunk][hi, lo]; also the scratch of the grouping phase (<= 40 KB)
+    B = take((size_t)TC_B_STAGES * nb * TC_KC * 2, 1024);
+    cn = take((size_t)((k + nb - 1) / nb) * nb * 4, 16);
     cnt = take((size_t)k * 4, 16);
     best = take((size_t)b * 2, 16);
     flagged = take((size_t)b * 2 + 16, 16);                          // pairs to settle from the front, rows for the full scan from the back
@@ -61,7 +71,7 @@ struct TcSmem {
     total = off + 1024;          // room to align the base to 1024 bytes
   }
 };
-inline size_t tc_smem_bytes(int k, int d, int b) { return TcSmem(k, d, b).total; }
+inline size_t tc_smem_bytes(int k, int d, int b, int terms) { return TcSmem(k, d, b, terms).total; }
 
 __device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -104,6 +114,13 @@ __global__ void tc_split_x_kernel(const float* __restrict__ X, const __nv_bfloat
     if (hi_out) *reinterpret_cast<__nv_bfloat162*>(hi_out + e) = h;
     const float2 hf = __bfloat1622float2(h);
     *reinterpret_cast<__nv_bfloat162*>(lo_out + e) = __floats2bfloat162_rn(v.x - hf.x, v.y - hf.y);
+  }
+}
+// samples -> FP16 (initialisation, one-term format)
+__global__ void tc_half_x_kernel(const float* __restrict__ X, __half* __restrict__ out, size_t n) {
+  for (size_t e = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 2; e + 1 < n; e += (size_t)gridDim.x * blockDim.x * 2) {
+    const float2 v = *reinterpret_cast<const float2*>(X + e);
+    *reinterpret_cast<__half2*>(out + e) = __floats2half2_rn(v.x, v.y);
   }
 }
 // ||x_i||^2 of every row (fp32): added to the scores so that the numbers compared are squared distances, whose
@@ -155,14 +172,14 @@ __device__ __forceinline__ void tc_top3_insert(float& m1, float& m2, float& m3, 
   m3 = fminf(m3, hi2);
 }
 
-template <bool kDet>
+template <bool kDet, int kTerms>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CUtensorMap mapXh,
                const __grid_constant__ CUtensorMap mapXl, const __grid_constant__ CUtensorMap mapW) {
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
   unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const int k = p.k, d = p.d, b = p.b;
-  const TcSmem map(k, d, b);
+  const TcSmem map(k, d, b, kTerms);
   unsigned char* sB = smem + map.B;
   unsigned char* sA = smem + map.A;
   float* cn = reinterpret_cast<float*>(smem + map.cn);                 // ||w_a||^2; beyond k a large finite number (with index bits
@@ -174,14 +191,19 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   int* misc = reinterpret_cast<int*>(smem + map.misc);                 // [0] tmem base, [1] pairs to settle, [2] abort, [4] news, [5] rows for the full scan
   TailScratch* ts = reinterpret_cast<TailScratch*>(smem + map.tail);
 
+  static_assert(kTerms == 1 || kTerms == 3, "one FP16 term or two BF16 terms per operand");
+  constexpr int PPK = (kTerms == 3) ? 2 : 1;                            // parts (hi, lo) per K chunk of an operand
+  constexpr int TC_N = tc_block_n(kTerms);                              // centres per block
+  constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;                    // a ring slot: one K chunk of a centre block
+  constexpr int TC_TMEM_COLS = 2 * TC_N;                                // two accumulator stages
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int i = blockIdx.x;
   const int nkc = d / TC_KC;                                           // K chunks per tile
   const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_M - 1) / TC_M;
   float* wglob = p.state + (size_t)i * p.kd_pad;
   float* gsum = p.gsum + (size_t)i * p.kd_pad;
-  __nv_bfloat16* wbf = reinterpret_cast<__nv_bfloat16*>(p.wbf) + (size_t)i * k * d;          // w_hi of this worker
-  __nv_bfloat16* wbl = wbf + (size_t)p.W * k * d;                                            // w_lo: second half of the array
+  unsigned short* wbf = reinterpret_cast<unsigned short*>(p.wbf) + (size_t)i * k * d;        // 16-bit -2w (w_hi) of this worker
+  unsigned short* wbl = wbf + (size_t)p.W * k * d;                                           // w_lo: second half of the array (two-term format)
   float4* top3 = reinterpret_cast<float4*>(p.top2) + (size_t)i * b;        // per row: three smallest packed squared distances
   const float INF = __int_as_float(0x7f800000);
   const float inv_b = 1.0f / (float)b;
@@ -208,12 +230,17 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         sq = fmaf(w4[q].x, w4[q].x, sq); sq = fmaf(w4[q].y, w4[q].y, sq); sq = fmaf(w4[q].z, w4[q].z, sq); sq = fmaf(w4[q].w, w4[q].w, sq);
         const size_t o = (size_t)a * d + 4 * l8 + 32 * q;
         const float v[4] = {-2.f * w4[q].x, -2.f * w4[q].y, -2.f * w4[q].z, -2.f * w4[q].w};     // exact
-        const __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
-        const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
-        *reinterpret_cast<__nv_bfloat162*>(wbf + o) = h01;
-        *reinterpret_cast<__nv_bfloat162*>(wbf + o + 2) = h23;
-        *reinterpret_cast<__nv_bfloat162*>(wbl + o) = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y);
-        *reinterpret_cast<__nv_bfloat162*>(wbl + o + 2) = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+        if (kTerms == 1) {
+          *reinterpret_cast<__half2*>(wbf + o) = __floats2half2_rn(v[0], v[1]);
+          *reinterpret_cast<__half2*>(wbf + o + 2) = __floats2half2_rn(v[2], v[3]);
+        } else {
+          const __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
+          const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+          *reinterpret_cast<__nv_bfloat162*>(wbf + o) = h01;
+          *reinterpret_cast<__nv_bfloat162*>(wbf + o + 2) = h23;
+          *reinterpret_cast<__nv_bfloat162*>(wbl + o) = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y);
+          *reinterpret_cast<__nv_bfloat162*>(wbl + o + 2) = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+        }
       }
     }
     return sq;
@@ -240,7 +267,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const unsigned tmem = (unsigned)misc[0];
-  const unsigned idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(TC_N >> 3) << 17) | ((unsigned)(TC_M >> 4) << 24);
+  // instruction descriptor: fp32 accumulate, operand format (0 = FP16, 1 = BF16) for both operands, N / 8, M / 16
+  const unsigned fmt = (kTerms == 3) ? 1u : 0u;
+  const unsigned idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(TC_N >> 3) << 17) | ((unsigned)(TC_M >> 4) << 24);
 
   unsigned long long t = p.stats[(size_t)i * ST_STRIDE + ST_STEPS];
   // running phase counters of the pipelines (each role keeps its own copies in step)
@@ -261,20 +290,21 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           for (int kc = 0; kc < nkc && ok; ++kc) {
             if (um > 0) ok = mbar_wait_bounded(bars + TCB_AEMPTY + kc, (um - 1) & 1, p.wait_limit);     // last use of the chunk by the previous tile
             if (!ok) break;
-            mbar_expect_tx(bars + TCB_AFULL + kc, (unsigned)(2 * TC_A_STAGE_BYTES));
+            mbar_expect_tx(bars + TCB_AFULL + kc, (unsigned)(PPK * TC_A_STAGE_BYTES));
             const bool withheld = (m == 0 && kc == 0 && step == p.withhold_step);   // failure drill: announced, never copied
             if (!withheld) {
-              tma_load_2d(sA + (size_t)(kc * 2 + 0) * TC_A_STAGE_BYTES, &mapXh, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc);
-              tma_load_2d(sA + (size_t)(kc * 2 + 1) * TC_A_STAGE_BYTES, &mapXl, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc);
+              tma_load_2d(sA + (size_t)(kc * PPK + 0) * TC_A_STAGE_BYTES, &mapXh, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc);
+              if (kTerms == 3)
+                tma_load_2d(sA + (size_t)(kc * PPK + 1) * TC_A_STAGE_BYTES, &mapXl, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc);
             }
           }
           for (int n = 0; n < n_tiles && ok; ++n) {
-            for (int g = 0; g < 2 * nkc; ++g, ++ibc) {                 // g = 2 * K chunk + (0: w_hi, 1: w_lo)
+            for (int g = 0; g < PPK * nkc; ++g, ++ibc) {               // g = PPK * K chunk + (0: w_hi, 1: w_lo)
               const int st = ibc % TC_B_STAGES;
               if (ibc >= TC_B_STAGES) ok = mbar_wait_bounded(bars + TCB_BEMPTY + st, ((ibc / TC_B_STAGES) - 1) & 1, p.wait_limit);
               if (!ok) break;
               mbar_expect_tx(bars + TCB_BFULL + st, (unsigned)TC_B_CHUNK_BYTES);
-              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, (g >> 1) * TC_KC, (g & 1) * p.W * k + i * k + n * TC_N, bars + TCB_BFULL + st);
+              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, (g / PPK) * TC_KC, (g % PPK) * p.W * k + i * k + n * TC_N, bars + TCB_BFULL + st);
             }
           }
         }
@@ -292,9 +322,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             if (!ok) break;
             tc_fence_after();
             const unsigned acc_col = tmem + (unsigned)(buf * TC_N);
-            for (int g = 0; g < 2 * nkc && ok; ++g, ++ibc) {
+            for (int g = 0; g < PPK * nkc && ok; ++g, ++ibc) {
               const int st = ibc % TC_B_STAGES;
-              const int kc = g >> 1, lo_w = g & 1;
+              const int kc = g / PPK, lo_w = g % PPK;
               if (n == 0 && lo_w == 0) ok = mbar_wait_bounded(bars + TCB_AFULL + kc, um & 1, p.wait_limit);
               if (ok) ok = mbar_wait_bounded(bars + TCB_BFULL + st, (ibc / TC_B_STAGES) & 1, p.wait_limit);
               if (!ok) break;
@@ -302,18 +332,18 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
               // operand descriptors: the base descriptor plus the chunk's offset in 16-byte units (the address field
               // holds address >> 4 and shared memory is below 256 KB, so the sum stays inside the field)
               const unsigned long long db = dB0 + (unsigned long long)(st * (TC_B_CHUNK_BYTES >> 4));
-              const unsigned long long dah = dA0 + (unsigned long long)((kc * 2 + 0) * (TC_A_STAGE_BYTES >> 4));
-              const unsigned long long dal = dA0 + (unsigned long long)((kc * 2 + 1) * (TC_A_STAGE_BYTES >> 4));
+              const unsigned long long dah = dA0 + (unsigned long long)((kc * PPK + 0) * (TC_A_STAGE_BYTES >> 4));
+              const unsigned long long dal = dA0 + (unsigned long long)((kc * PPK + 1) * (TC_A_STAGE_BYTES >> 4));
 #pragma unroll
               for (int k4 = 0; k4 < TC_KC / 16; ++k4)                   // x_hi . w_hi  or  x_hi . w_lo
                 tc_mma_bf16(acc_col, dah + (unsigned long long)(2 * k4), db + (unsigned long long)(2 * k4), idesc, (g | k4) != 0);
-              if (lo_w == 0) {
+              if (kTerms == 3 && lo_w == 0) {
 #pragma unroll
                 for (int k4 = 0; k4 < TC_KC / 16; ++k4)                 // x_lo . w_hi
                   tc_mma_bf16(acc_col, dal + (unsigned long long)(2 * k4), db + (unsigned long long)(2 * k4), idesc, true);
               }
               tc_commit(bars + TCB_BEMPTY + st);                        // the ring slot is free when these MMAs have read it
-              if (n == n_tiles - 1 && lo_w == 1) tc_commit(bars + TCB_AEMPTY + kc);   // and so is the sample chunk after its last centre block
+              if (n == n_tiles - 1 && lo_w == PPK - 1) tc_commit(bars + TCB_AEMPTY + kc);   // and so is the sample chunk after its last centre block
             }
             tc_commit(bars + TCB_ACCFULL + buf);                        // the accumulator stage is complete
           }
@@ -381,7 +411,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       if (!ok && lane == 0) atomicExch(&misc[2], 1);
     }
     it_m += (unsigned)m_tiles;
-    it_bc += (unsigned)(m_tiles * n_tiles * 2 * nkc);
+    it_bc += (unsigned)(m_tiles * n_tiles * PPK * nkc);
     it_acc += (unsigned)(n_tiles * m_tiles);
     if (tid == 0) { misc[1] = 0; misc[5] = 0; }
     for (int a = tid; a < k; a += TC_THREADS) cnt[a] = 0;
@@ -400,8 +430,14 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     //   fp32 accumulation of 3 d / 16 partial sums    (3 d / 16 + 1) * 2^-22 ||x|| ||w||     (each step at most one ulp of a sum <= 2 ||x|| ||w||)
     //   the two fp32 adds of the norms                3 * 2^-24 (||x||^2 + ||w||^2 + 2 ||x|| ||w||)
     // with a quarter on top; the index bits cost 2^10 ulp <= 2^-13 of the value itself, applied relative to the values compared.
+    // One FP16 term per operand: both factors of a product are off by 2^-12 relative, the sum of |x_j| |2 w_j| is at
+    // most 2 ||x|| ||w||: 2^-10 ||x|| ||w||; d / 16 partial sums; inputs below FP16's normal range (6.1e-5) lose at
+    // most 2^-25 each in absolute terms: 2^-24 sqrt(d) (||x|| + 2 ||w||) in all.
     const float xw = sqrtf(p.xmax2 * wmax2);
-    const float err = 1.25f * ((2.289e-5f + (float)(3 * d / 16 + 1) * 2.384e-7f) * xw + 1.79e-7f * (p.xmax2 + wmax2 + 2.f * xw));
+    const float err = (kTerms == 3)
+        ? 1.25f * ((2.289e-5f + (float)(3 * d / 16 + 1) * 2.384e-7f) * xw + 1.79e-7f * (p.xmax2 + wmax2 + 2.f * xw))
+        : 1.25f * ((9.766e-4f + (float)(d / 16 + 1) * 2.384e-7f) * xw + 1.79e-7f * (p.xmax2 + wmax2 + 2.f * xw) +
+                   5.96e-8f * sqrtf((float)d) * (sqrtf(p.xmax2) + 2.f * sqrtf(wmax2)));
     auto inside = [&](float lo, float hi_) { return (hi_ - lo) <= 2.f * err + 2.4415e-4f * fmaxf(fabsf(lo), fabsf(hi_)); };
     // Scratch for the rest of the step lives in the sample ring, which is idle until the next step's loads.
     int* wcnt = reinterpret_cast<int*>(sA);                                   // [TC_WARPS][k] rows of a centre in a warp's row block
@@ -485,57 +521,132 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         settle_finish(xa, pa, qa, ra, ia1, ia2);
       }
     }
-    // ---- rows with three or more candidates: a warp per row looks at every centre, lanes over centres, direct
-    //      differences in fp32; if the two smallest are still within rounding of each other, again in fp64 ----
+    // ---- rows with three or more candidates are decided over all centres, TC_SCAN_ROWS rows at a time: the rows wait
+    //      in shared memory (the idle centre ring), every warp walks its share of the centres (a centre row is one
+    //      coalesced read, lanes over the dimensions, the next centre's row already on its way) and measures it against
+    //      every waiting row with direct differences in fp32; the lanes' partial sums of all rows are added up by a
+    //      halving exchange (lanes 2j, 2j+1 end with row j's distance), and lane 2j keeps row j's two smallest.  A row
+    //      whose two smallest are still within rounding of each other is measured once more in fp64. ----
     {
+      __syncthreads();                                         // the pairs' readers of `order` and `top3` are done; the ring is idle
+      constexpr int RB = TC_SCAN_ROWS;
       const int nwide = misc[5];
-      for (int f = wid; f < nwide; f += TC_WARPS) {            // warp-uniform trip count
-        const int r = (int)order[b - 1 - f];
-        const float* xr = p.X + (size_t)(row0 + r) * d;
-        float fd1 = INF, fd2 = INF;
-        int fi = 0x7fffffff;
-        for (int a = lane; a < k; a += 32) {
-          const float* wa = wglob + (size_t)a * d;
-          float sacc = 0.f;
-          for (int j = 0; j < d; j += 4) {
-            const float4 xv4 = __ldg(reinterpret_cast<const float4*>(xr + j));
-            const float4 wv4 = *reinterpret_cast<const float4*>(wa + j);
-            float u;
-            u = xv4.x - wv4.x; sacc = fmaf(u, u, sacc); u = xv4.y - wv4.y; sacc = fmaf(u, u, sacc);
-            u = xv4.z - wv4.z; sacc = fmaf(u, u, sacc); u = xv4.w - wv4.w; sacc = fmaf(u, u, sacc);
-          }
-          if (sacc < fd1) { fd2 = fd1; fd1 = sacc; fi = a; } else if (sacc < fd2) { fd2 = sacc; }
+      const int d4 = d / 4;
+      float4* xs4 = reinterpret_cast<float4*>(sB);             // [RB][d / 4] waiting rows
+      float* res = reinterpret_cast<float*>(sB) + RB * d;      // [TC_WARPS][RB][5] per warp and row: the three smallest, indices of the first two
+      int* need64 = reinterpret_cast<int*>(res + TC_WARPS * RB * 5);      // [RB][3]: 0 decided, 1 compare two in fp64, 2 scan all in fp64; the two indices
+      const bool on0 = lane < d4, on1 = 32 + lane < d4;
+      const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int base = 0; base < nwide; base += RB) {           // block-uniform trip count
+        const int R = min(RB, nwide - base);
+        for (int e = tid; e < RB * d4; e += TC_THREADS) {
+          const int j = e / d4, c4 = e - j * d4;
+          xs4[e] = (j < R) ? __ldg(reinterpret_cast<const float4*>(p.X + (size_t)(row0 + (int)order[b - 1 - (base + j)]) * d) + c4) : z4;
         }
+        __syncthreads();
+        float bd1 = INF, bd2 = INF, bd3 = INF;                 // lane 2j: row j over this warp's centres
+        int bi1 = 0x7fffffff, bi2 = 0x7fffffff;
+        const float4* wa = reinterpret_cast<const float4*>(wglob + (size_t)wid * d);
+        float4 w0v = (wid < k && on0) ? wa[lane] : z4, w1v = (wid < k && on1) ? wa[32 + lane] : z4;
+        for (int a = wid; a < k; a += TC_WARPS) {              // ascending inside a warp: a strict "<" keeps the lowest index of a tie
+          const float4* wn = reinterpret_cast<const float4*>(wglob + (size_t)min(a + TC_WARPS, k - 1) * d);
+          const float4 n0 = on0 ? wn[lane] : z4, n1 = on1 ? wn[32 + lane] : z4;      // the next centre's row
+          float part[RB];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          const float o1 = __shfl_xor_sync(0xffffffffu, fd1, o);
-          const float o2 = __shfl_xor_sync(0xffffffffu, fd2, o);
-          const int oi = __shfl_xor_sync(0xffffffffu, fi, o);
-          const bool take = (o1 < fd1) || (o1 == fd1 && oi < fi);
-          fd2 = fminf(take ? fd1 : o1, fminf(fd2, o2));
-          if (take) { fd1 = o1; fi = oi; }
-        }
-        int bi = fi;
-        if (fd2 - fd1 <= (float)(4 * TC_MAX_D + 16) * 5.9604645e-8f * fd2) {
-          double bd = 1e300;
-          bi = 0x7fffffff;
-          for (int a = lane; a < k; a += 32) {
-            const float* wa = wglob + (size_t)a * d;
-            double sacc = 0.0;
-            for (int j = 0; j < d; ++j) {
-              const double u = (double)__ldg(xr + j) - (double)wa[j];
-              sacc = fma(u, u, sacc);
+          for (int j = 0; j < RB; ++j) {
+            const float4 x0 = on0 ? xs4[j * d4 + lane] : z4;
+            const float4 x1 = on1 ? xs4[j * d4 + 32 + lane] : z4;
+            float s0 = 0.f, s1 = 0.f, e;
+            e = x0.x - w0v.x; s0 = fmaf(e, e, s0); e = x0.y - w0v.y; s1 = fmaf(e, e, s1);
+            e = x0.z - w0v.z; s0 = fmaf(e, e, s0); e = x0.w - w0v.w; s1 = fmaf(e, e, s1);
+            e = x1.x - w1v.x; s0 = fmaf(e, e, s0); e = x1.y - w1v.y; s1 = fmaf(e, e, s1);
+            e = x1.z - w1v.z; s0 = fmaf(e, e, s0); e = x1.w - w1v.w; s1 = fmaf(e, e, s1);
+            part[j] = s0 + s1;
+          }
+          // halving exchange: at offset o the lanes with that bit clear keep the lower half of the rows still held
+#pragma unroll
+          for (int o = 16, n = RB / 2; n >= 1; o >>= 1, n >>= 1) {
+            const bool up = (lane & o) != 0;
+#pragma unroll
+            for (int j = 0; j < n; ++j) {
+              const float send = up ? part[j] : part[j + n];
+              const float keep = up ? part[j + n] : part[j];
+              part[j] = keep + __shfl_xor_sync(0xffffffffu, send, o);
             }
-            if (sacc < bd) { bd = sacc; bi = a; }                // ascending a: the lowest index keeps a tie
           }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const double od = __shfl_xor_sync(0xffffffffu, bd, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (od < bd || (od == bd && oi < bi)) { bd = od; bi = oi; }
+          const float tot = part[0] + __shfl_xor_sync(0xffffffffu, part[0], 1);      // lanes 2j and 2j+1: row j
+          if ((lane & 1) == 0) {
+            if (tot < bd1) { bd3 = bd2; bd2 = bd1; bi2 = bi1; bd1 = tot; bi1 = a; }
+            else if (tot < bd2) { bd3 = bd2; bd2 = tot; bi2 = a; }
+            else if (tot < bd3) { bd3 = tot; }
           }
+          w0v = n0; w1v = n1;
         }
-        if (lane == 0) best[r] = (unsigned short)bi;
+        if ((lane & 1) == 0) {
+          const int j = lane >> 1;
+          float* o = res + (wid * RB + j) * 5;
+          o[0] = bd1; o[1] = bd2; o[2] = bd3; o[3] = __int_as_float(bi1); o[4] = __int_as_float(bi2);
+        }
+        __syncthreads();
+        if (tid < RB) {
+          // the warps' shares merged: three smallest distances, the first two with their centres (equal distances: lowest index first)
+          float fd1 = INF, fd2 = INF, fd3 = INF;
+          int fi1 = 0x7fffffff, fi2 = 0x7fffffff;
+          auto put = [&](float v, int idx) {
+            if (v < fd1 || (v == fd1 && idx < fi1)) { fd3 = fd2; fd2 = fd1; fi2 = fi1; fd1 = v; fi1 = idx; }
+            else if (v < fd2 || (v == fd2 && idx < fi2)) { fd3 = fd2; fd2 = v; fi2 = idx; }
+            else if (v < fd3) { fd3 = v; }
+          };
+          for (int q = 0; q < TC_WARPS; ++q) {
+            const float* o = res + (q * RB + tid) * 5;
+            put(o[0], __float_as_int(o[3]));
+            put(o[1], __float_as_int(o[4]));
+            put(o[2], 0x7fffffff);
+          }
+          // fp32 distances are off by at most (d + 2) u relative: a gap above (4 d + 16) u of the larger one decides
+          const float tol = (float)(4 * TC_MAX_D + 16) * 5.9604645e-8f;
+          int how = 0;
+          if (tid < R && fd2 - fd1 <= tol * fd2) how = (fd3 - fd1 <= tol * fd3) ? 2 : 1;
+          need64[tid * 3 + 0] = how;
+          need64[tid * 3 + 1] = fi1;
+          need64[tid * 3 + 2] = fi2;
+          if (tid < R && how == 0) best[order[b - 1 - (base + tid)]] = (unsigned short)fi1;
+        }
+        __syncthreads();
+        for (int j = wid; j < R; j += TC_WARPS) {              // warp-uniform: need64[j] is the same for every lane
+          const int how = need64[j * 3 + 0];
+          if (how == 0) continue;
+          const float4 x0 = on0 ? xs4[j * d4 + lane] : z4;
+          const float4 x1 = on1 ? xs4[j * d4 + 32 + lane] : z4;
+          auto dist64 = [&](int a) {                           // fp64 squared distance to centre a (the same value in every lane)
+            const float4* wr = reinterpret_cast<const float4*>(wglob + (size_t)a * d);
+            const float4 u0 = on0 ? wr[lane] : z4;
+            const float4 u1 = on1 ? wr[32 + lane] : z4;
+            double sacc = 0.0, e;
+            e = (double)x0.x - (double)u0.x; sacc = fma(e, e, sacc); e = (double)x0.y - (double)u0.y; sacc = fma(e, e, sacc);
+            e = (double)x0.z - (double)u0.z; sacc = fma(e, e, sacc); e = (double)x0.w - (double)u0.w; sacc = fma(e, e, sacc);
+            e = (double)x1.x - (double)u1.x; sacc = fma(e, e, sacc); e = (double)x1.y - (double)u1.y; sacc = fma(e, e, sacc);
+            e = (double)x1.z - (double)u1.z; sacc = fma(e, e, sacc); e = (double)x1.w - (double)u1.w; sacc = fma(e, e, sacc);
+#pragma unroll
+            for (int sh = 16; sh > 0; sh >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, sh);
+            return sacc;
+          };
+          int bi;
+          if (how == 1) {                                      // two candidates: the closer one, the lower index on a tie
+            const int i1 = need64[j * 3 + 1], i2 = need64[j * 3 + 2];
+            const double e1 = dist64(i1), e2 = dist64(i2);
+            bi = (e2 < e1 || (e2 == e1 && i2 < i1)) ? i2 : i1;
+          } else {                                             // three or more within rounding: every centre once more
+            double bd = 1e300;
+            bi = 0;
+            for (int a = 0; a < k; ++a) {
+              const double e1 = dist64(a);
+              if (e1 < bd) { bd = e1; bi = a; }                  // ascending a: the lowest index keeps a tie
+            }
+          }
+          if (lane == 0) best[order[b - 1 - (base + j)]] = (unsigned short)bi;
+        }
+        __syncthreads();                                       // before the next rows overwrite the waiting area
       }
     }
     __syncthreads();

@@ -89,6 +89,50 @@ def test_single_step_assignments_bit_exact(name):
     pr.close()
 
 
+@pytest.mark.parametrize("name", ["dense", "codebook"])
+@pytest.mark.parametrize("fmt", ["fp16", "bf16x3"])
+def test_tensor_core_formats_decide_exactly(name, fmt):
+    """Both operand formats of the tensor-core path (one FP16 term; two BF16 terms) against the oracle: the
+    trajectory within the centre tolerance, the assignments of a round started from the oracle's states exactly."""
+    wl, rounds = PARITY_WORKLOADS[name]
+    pr = Pair(wl, dist_path=pkg.PATH_TC_FP16 if fmt == "fp16" else pkg.PATH_TC_BF16)
+    assert pr.gpu.path_name() == "tcgen05-" + fmt
+    pr.rounds(rounds)
+    pr.gpu.sync()
+    assert pr.max_rel_l2() < CENTRE_TOL, (name, fmt, pr.max_rel_l2())
+    pr.load_oracle_states_into_gpu()
+    pr.rounds(1)
+    pr.gpu.sync()
+    got = pr.gpu.get_assign().cpu().numpy()
+    for i in range(wl.W):
+        tr = pr.cpu.last_step(i)
+        ok = decided(tr["d1"], tr["d2"])
+        assert (got[i][ok] == tr["assign"][ok]).all(), (name, fmt, i)
+        assert ok.mean() > 0.99
+    _compare_stats(pr, exact_accept=False)
+    pr.close()
+
+
+def test_fp16_format_refuses_samples_outside_its_range():
+    wl = scaled("dense", N=2 * 256 * 3, W=2, b=256, k=200, d=64, comm_interval=1)
+    X = np.random.default_rng(3).standard_normal((wl.N, wl.d)).astype(np.float32) * 3.0e4      # ||x|| far beyond 65504 / 8
+    with pytest.raises(pkg.AsgdError) as err:
+        Pair(wl, X=X, oracle=False, dist_path=pkg.PATH_TC_FP16)
+    assert err.value.status == pkg.binding.ASGD_EUNSUPPORTED
+    pr = Pair(wl, X=X, dist_path=pkg.PATH_AUTO)                   # AUTO: an fp32 path takes over
+    assert pr.gpu.path_name().startswith("fp32")
+    pr.rounds(2)
+    pr.gpu.sync()
+    assert pr.max_rel_l2() < CENTRE_TOL
+    pr.close()
+    pr = Pair(wl, X=X, dist_path=pkg.PATH_TC_BF16)                # the two-term BF16 format has fp32's range
+    assert pr.gpu.path_name() == "tcgen05-bf16x3"
+    pr.rounds(2)
+    pr.gpu.sync()
+    assert pr.max_rel_l2() < CENTRE_TOL
+    pr.close()
+
+
 def test_parzen_hand_cases_on_gpu():
     for line in open(os.path.join(GOLD, "parzen_1d_cases.txt")):
         if line.startswith("#") or not line.strip():

@@ -44,7 +44,7 @@ def test_random_configuration_matches_oracle(family, seed):
     over, slots, parzen, rows, batches = _draw(family, seed)
     wl = scaled("tiny", **over)
     pr = Pair(wl, parzen=parzen, slots=slots, partial_rows=rows, shuffle=int(seed % 2))
-    want = {"stream": "fp32-stream", "tiled": "fp32-tiled", "tensor": "tcgen05-bf16", "general": "fp32-generic"}[family]
+    want = {"stream": "fp32-stream", "tiled": "fp32-tiled", "tensor": "tcgen05-fp16", "general": "fp32-generic"}[family]
     assert pr.gpu.path_name() == want, (family, seed, over, pr.gpu.path_name())
     rounds = 2 * batches + 1
     pr.rounds(rounds)

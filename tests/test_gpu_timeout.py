@@ -17,14 +17,16 @@ CASES = {
     # kernel: (workload, path name)
     "stream": (scaled("tiny", N=4 * 100 * 6, comm_interval=2), "fp32-stream"),
     "tiled": (scaled("sweep", N=6 * 256 * 5 + 3, W=6, comm_interval=2), "fp32-tiled"),
-    "tensor": (scaled("dense", N=2 * 512 * 5 + 1, W=2, b=512, comm_interval=2), "tcgen05-bf16"),
+    "tensor": (scaled("dense", N=2 * 512 * 5 + 1, W=2, b=512, comm_interval=2), "tcgen05-fp16"),
+    "tensor_two_terms": (scaled("dense", N=2 * 512 * 5 + 1, W=2, b=512, comm_interval=2), "tcgen05-bf16x3"),
 }
 
 
 @pytest.mark.parametrize("kernel", list(CASES))
 def test_a_wait_that_runs_out_is_reported_and_the_device_stays_usable(kernel):
     wl, path = CASES[kernel]
-    pr = Pair(wl, oracle=False, record_assign=0)
+    dist_path = pkg.PATH_TC_BF16 if kernel == "tensor_two_terms" else pkg.PATH_AUTO
+    pr = Pair(wl, oracle=False, record_assign=0, dist_path=dist_path)
     assert pr.gpu.path_name().startswith(path)
     pr.gpu.run(2)
     pr.gpu.sync()                                     # nothing wrong so far
@@ -38,7 +40,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_device_stays_usable(kernel):
     pr.close()
 
     # a fresh context on the same device: the kernel left nothing behind (shared memory, tensor memory, status)
-    again = Pair(wl)
+    again = Pair(wl, dist_path=dist_path)
     again.rounds(3)
     again.gpu.sync()
     assert again.max_rel_l2() < again.centre_tol()
