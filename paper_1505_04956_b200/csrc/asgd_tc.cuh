@@ -433,12 +433,15 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     // One FP16 term per operand: both factors of a product are off by 2^-12 relative, the sum of |x_j| |2 w_j| is at
     // most 2 ||x|| ||w||: 2^-10 ||x|| ||w||; d / 16 partial sums; inputs below FP16's normal range (6.1e-5) lose at
     // most 2^-25 each in absolute terms: 2^-24 sqrt(d) (||x|| + 2 ||w||) in all.
-    const float xw = sqrtf(p.xmax2 * wmax2);
-    const float err = (kTerms == 3)
-        ? 1.25f * ((2.289e-5f + (float)(3 * d / 16 + 1) * 2.384e-7f) * xw + 1.79e-7f * (p.xmax2 + wmax2 + 2.f * xw))
-        : 1.25f * ((9.766e-4f + (float)(d / 16 + 1) * 2.384e-7f) * xw + 1.79e-7f * (p.xmax2 + wmax2 + 2.f * xw) +
-                   5.96e-8f * sqrtf((float)d) * (sqrtf(p.xmax2) + 2.f * sqrtf(wmax2)));
-    auto inside = [&](float lo, float hi_) { return (hi_ - lo) <= 2.f * err + 2.4415e-4f * fmaxf(fabsf(lo), fabsf(hi_)); };
+    // The bound is taken per row, with the row's own ||x||^2 (and the largest ||w_a||^2).
+    auto row_err = [&](float xn) {
+      const float xw = sqrtf(xn * wmax2);
+      return (kTerms == 3)
+          ? 1.25f * ((2.289e-5f + (float)(3 * d / 16 + 1) * 2.384e-7f) * xw + 1.79e-7f * (xn + wmax2 + 2.f * xw))
+          : 1.25f * ((9.766e-4f + (float)(d / 16 + 1) * 2.384e-7f) * xw + 1.79e-7f * (xn + wmax2 + 2.f * xw) +
+                     5.96e-8f * sqrtf((float)d) * (sqrtf(xn) + 2.f * sqrtf(wmax2)));
+    };
+    auto inside = [&](float lo, float hi_, float err) { return (hi_ - lo) <= 2.f * err + 2.4415e-4f * fmaxf(fabsf(lo), fabsf(hi_)); };
     // Scratch for the rest of the step lives in the sample ring, which is idle until the next step's loads.
     int* wcnt = reinterpret_cast<int*>(sA);                                   // [TC_WARPS][k] rows of a centre in a warp's row block
     unsigned short* lrank = reinterpret_cast<unsigned short*>(sA + (size_t)TC_WARPS * k * 4);   // [b] rank of a row among its warp's rows of the centre
@@ -449,8 +452,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     for (int r = tid; r < b; r += TC_THREADS) {
       const float4 s = __ldcg(top3 + r);
       best[r] = (unsigned short)(__float_as_uint(s.x) & TC_INDEX_MASK);
-      if (k > 1 && inside(s.x, s.y)) {
-        if (k > 2 && inside(s.x, s.z)) order[b - 1 - atomicAdd(&misc[5], 1)] = (unsigned short)r;
+      const float err = row_err(__ldg(p.xnorm + row0 + r));
+      if (k > 1 && inside(s.x, s.y, err)) {
+        if (k > 2 && inside(s.x, s.z, err)) order[b - 1 - atomicAdd(&misc[5], 1)] = (unsigned short)r;
         else order[atomicAdd(&misc[1], 1)] = (unsigned short)r;
       }
     }
@@ -521,10 +525,10 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         settle_finish(xa, pa, qa, ra, ia1, ia2);
       }
     }
-    // ---- rows with three or more candidates are decided over all centres, TC_SCAN_ROWS rows at a time: the rows wait
-    //      in shared memory (the idle centre ring), every warp walks its share of the centres (a centre row is one
-    //      coalesced read, lanes over the dimensions, the next centre's row already on its way) and measures it against
-    //      every waiting row with direct differences in fp32; the lanes' partial sums of all rows are added up by a
+    // ---- rows with three or more candidates are decided over all centres, TC_SCAN_ROWS rows at a time: every lane
+    //      holds its dimensions of all the rows in registers, every warp walks its share of the centres (a centre row is
+    //      one coalesced read, lanes over the dimensions, the next centre's row already on its way) and measures it
+    //      against every row with direct differences in fp32; the lanes' partial sums of all rows are added up by a
     //      halving exchange (lanes 2j, 2j+1 end with row j's distance), and lane 2j keeps row j's two smallest.  A row
     //      whose two smallest are still within rounding of each other is measured once more in fp64. ----
     {
@@ -532,18 +536,19 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       constexpr int RB = TC_SCAN_ROWS;
       const int nwide = misc[5];
       const int d4 = d / 4;
-      float4* xs4 = reinterpret_cast<float4*>(sB);             // [RB][d / 4] waiting rows
-      float* res = reinterpret_cast<float*>(sB) + RB * d;      // [TC_WARPS][RB][5] per warp and row: the three smallest, indices of the first two
+      float* res = reinterpret_cast<float*>(sB);               // [TC_WARPS][RB][5] per warp and row: the three smallest, indices of the first two
       int* need64 = reinterpret_cast<int*>(res + TC_WARPS * RB * 5);      // [RB][3]: 0 decided, 1 compare two in fp64, 2 scan all in fp64; the two indices
       const bool on0 = lane < d4, on1 = 32 + lane < d4;
       const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
       for (int base = 0; base < nwide; base += RB) {           // block-uniform trip count
         const int R = min(RB, nwide - base);
-        for (int e = tid; e < RB * d4; e += TC_THREADS) {
-          const int j = e / d4, c4 = e - j * d4;
-          xs4[e] = (j < R) ? __ldg(reinterpret_cast<const float4*>(p.X + (size_t)(row0 + (int)order[b - 1 - (base + j)]) * d) + c4) : z4;
+        float4 xr0[RB], xr1[RB];                               // this lane's dimensions of the rows (zeros past the last row)
+#pragma unroll
+        for (int j = 0; j < RB; ++j) {
+          const float4* xrow = reinterpret_cast<const float4*>(p.X + (size_t)(row0 + (int)order[b - 1 - (base + min(j, R - 1))]) * d);
+          xr0[j] = (j < R && on0) ? __ldg(xrow + lane) : z4;
+          xr1[j] = (j < R && on1) ? __ldg(xrow + 32 + lane) : z4;
         }
-        __syncthreads();
         float bd1 = INF, bd2 = INF, bd3 = INF;                 // lane 2j: row j over this warp's centres
         int bi1 = 0x7fffffff, bi2 = 0x7fffffff;
         const float4* wa = reinterpret_cast<const float4*>(wglob + (size_t)wid * d);
@@ -554,8 +559,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           float part[RB];
 #pragma unroll
           for (int j = 0; j < RB; ++j) {
-            const float4 x0 = on0 ? xs4[j * d4 + lane] : z4;
-            const float4 x1 = on1 ? xs4[j * d4 + 32 + lane] : z4;
+            const float4 x0 = xr0[j], x1 = xr1[j];
             float s0 = 0.f, s1 = 0.f, e;
             e = x0.x - w0v.x; s0 = fmaf(e, e, s0); e = x0.y - w0v.y; s1 = fmaf(e, e, s1);
             e = x0.z - w0v.z; s0 = fmaf(e, e, s0); e = x0.w - w0v.w; s1 = fmaf(e, e, s1);
@@ -616,8 +620,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         for (int j = wid; j < R; j += TC_WARPS) {              // warp-uniform: need64[j] is the same for every lane
           const int how = need64[j * 3 + 0];
           if (how == 0) continue;
-          const float4 x0 = on0 ? xs4[j * d4 + lane] : z4;
-          const float4 x1 = on1 ? xs4[j * d4 + 32 + lane] : z4;
+          const float4* xrow = reinterpret_cast<const float4*>(p.X + (size_t)(row0 + (int)order[b - 1 - (base + j)]) * d);
+          const float4 x0 = on0 ? __ldg(xrow + lane) : z4;
+          const float4 x1 = on1 ? __ldg(xrow + 32 + lane) : z4;
           auto dist64 = [&](int a) {                           // fp64 squared distance to centre a (the same value in every lane)
             const float4* wr = reinterpret_cast<const float4*>(wglob + (size_t)a * d);
             const float4 u0 = on0 ? wr[lane] : z4;
