@@ -172,6 +172,16 @@ __device__ __forceinline__ void tc_top3_insert(float& m1, float& m2, float& m3, 
   m3 = fminf(m3, hi2);
 }
 
+// the same for two new values at once (eight min/max, three of them three-input): with lo <= hi the new triple is
+//   min(m1, lo),  min(max(m1, lo), m2, hi),  min(m3, max(m2, lo), max(m1, hi))
+__device__ __forceinline__ void tc_top3_insert2(float& m1, float& m2, float& m3, float v, float u) {
+  const float lo = fminf(v, u), hi = fmaxf(v, u);
+  const float a = fmaxf(m1, lo), b2 = fmaxf(m2, lo), c = fmaxf(m1, hi);
+  m3 = fmin3(m3, b2, c);
+  m2 = fmin3(a, m2, hi);
+  m1 = fminf(m1, lo);
+}
+
 template <bool kDet, int kTerms>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CUtensorMap mapXh,
@@ -387,6 +397,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             for (int c = 0; c < 32; c += 4) {
               const float4 cn4 = *reinterpret_cast<const float4*>(cn + abase + c);
               const float cv[4] = {cn4.x, cn4.y, cn4.z, cn4.w};
+              float sp[4];
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
                 // squared distance ||x||^2 - 2 x.w_a + ||w_a||^2 (fp32 adds), then one logic op: the value's high
@@ -394,8 +405,10 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
                 const float d2 = (__uint_as_float(v[c + u]) + cv[u]) + xn;
                 unsigned spb;
                 asm("lop3.b32 %0, %1, %2, %3, 0xE6;" : "=r"(spb) : "r"(__float_as_uint(d2)), "r"(hi_or_base), "r"(~TC_INDEX_MASK | (unsigned)(c + u)));
-                tc_top3_insert(m1[u & 1], m2[u & 1], m3[u & 1], __uint_as_float(spb));
+                sp[u] = __uint_as_float(spb);
               }
+              tc_top3_insert2(m1[0], m2[0], m3[0], sp[0], sp[1]);
+              tc_top3_insert2(m1[1], m2[1], m3[1], sp[2], sp[3]);
             }
           }
         }
