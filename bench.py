@@ -23,22 +23,50 @@ if ROOT not in sys.path:
 
 METRIC = "K-Means ASGD samples/s"
 UNIT = "samples/s"
-CPU_SAMPLE_ROWS = 1 << 25          # prefix of the workload the CPU baseline runs on
+CPU_SAMPLE_ROWS = 1 << 25          # prefix of the workload the CPU baseline runs on (all cores)
+CPU_SAMPLE_ROWS_ONE_CORE = 1 << 22 # and on one core
 NOMINAL_HBM_GBS = 8000.0
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the stream kernel per algorithmic byte, from one ncu
-# capture of a 2^24-row case (profiles/asgd_stream_kernel__stream_workload.md); it grows in proportion to the rows
-# a launch processes.  Valid only for the kernel sources it was taken on (stream_kernel_sha1()).
-TRAFFIC_CAPTURE = {"kernel_sha1": "3dee0be9b006", "traffic_per_algorithmic_byte": 670.41 / 663.51}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the worker kernel per algorithmic byte, each from one
+# small-case ncu capture of that kernel (a few hundred MB of samples, more than L2 holds; the traffic grows in
+# proportion to the rows a launch processes).  A record is valid only for the kernel sources it was taken on.
+KERNEL_SOURCES = {
+    "fp32-stream": ("asgd_common.cuh", "asgd_step_tail.cuh", "asgd_stream.cuh"),
+    "fp32-tiled": ("asgd_common.cuh", "asgd_step_tail.cuh", "asgd_stream.cuh", "asgd_tiled.cuh"),
+    "tcgen05-fp16": ("asgd_common.cuh", "asgd_step_tail.cuh", "asgd_stream.cuh", "asgd_tc.cuh"),
+    "tcgen05-bf16x3": ("asgd_common.cuh", "asgd_step_tail.cuh", "asgd_stream.cuh", "asgd_tc.cuh"),
+}
+TRAFFIC_CAPTURES = {
+    # (kernel, workload): source key at capture time, captured DRAM bytes / algorithmic bytes
+    ("fp32-stream", "stream"): {"kernel_sha1": "738aaa8084ba", "traffic_per_algorithmic_byte": 671.51 / 663.51},
+    ("fp32-tiled", "mid"): {"kernel_sha1": "ff7195b109a9", "traffic_per_algorithmic_byte": 1198.54 / 1060.86},
+    ("fp32-tiled", "sweep"): {"kernel_sha1": "ff7195b109a9", "traffic_per_algorithmic_byte": 1092.2 / 1091.17},
+    ("tcgen05-fp16", "dense"): {"kernel_sha1": "0d400020dff1", "traffic_per_algorithmic_byte": 3502.74 / 1241.51},
+    ("tcgen05-fp16", "codebook"): {"kernel_sha1": "0d400020dff1", "traffic_per_algorithmic_byte": 2531.6 / 620.76},
+}
 
 
-def stream_kernel_sha1():
-    """First 12 hex digits of the SHA-1 over the sources the streaming kernel is compiled from."""
+def kernel_sha1(kernel):
+    """First 12 hex digits of the SHA-1 over the sources a worker kernel is compiled from."""
     import hashlib
     h = hashlib.sha1()
-    for name in ("asgd_common.cuh", "asgd_step_tail.cuh", "asgd_stream.cuh"):
+    for name in KERNEL_SOURCES.get(kernel, ()):
         with open(os.path.join(ROOT, "paper_1505_04956_b200", "csrc", name), "rb") as f:
             h.update(f.read())
     return h.hexdigest()[:12]
+
+
+def stream_kernel_sha1():
+    return kernel_sha1("fp32-stream")
+
+
+def captured_traffic(kernel, workload, algorithmic_bytes):
+    """(bytes, how) of the DRAM traffic of one launch scaled from the stored capture, or (None, why not)."""
+    rec = TRAFFIC_CAPTURES.get((kernel, workload))
+    if rec is None:
+        return None, "no capture of this kernel on this workload"
+    if rec["kernel_sha1"] != kernel_sha1(kernel):
+        return None, "the kernel has changed since its counters were taken"
+    return algorithmic_bytes * rec["traffic_per_algorithmic_byte"], "scaled from a small-case ncu capture by the rows processed"
 
 
 def env_int(name, default):
@@ -175,51 +203,18 @@ def run_reference(args):
     return 0
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="stream")
-    ap.add_argument("--rows", type=int, default=0, help="use only the first ROWS rows (profiling of a small case)")
-    ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--reference-rows", type=int, default=1 << 23)
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    # points of the worker / communication sweep and the ablations (the defaults are the workload's own values)
-    ap.add_argument("--workers", type=int, default=0, help="W")
-    ap.add_argument("--comm-interval", type=int, default=-1, help="c; 0 = silent (no puts)")
-    ap.add_argument("--no-parzen", action="store_true", help="accept every non-empty message (Eq. 3 without Eq. 4)")
-    ap.add_argument("--partial-rows", type=int, default=0, help="centre rows per message (Section 4.4); 0 = whole state")
-    args = ap.parse_args()
-    if args.impl == "reference":
-        return run_reference(args)
-
+def measure(args, wl, dev, rank, world, dist, keep=False):
+    """The timed region for one workload on this rank: W untimed passes, K timed passes (one asgd_run launch each)."""
     import torch
     import paper_1505_04956_b200 as pkg
-    from paper_1505_04956_b200 import dist, inputs
-
-    args.warmup = max(args.warmup, 3)
-    rank, world, local = dist.init_from_env(backend="nccl")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    pkg.load()
-
-    wl = inputs.WORKLOADS[args.workload]
-    if args.rows:
-        wl = wl.scaled(N=args.rows)
-    if args.workers:
-        wl = wl.scaled(W=args.workers)
-    if args.comm_interval >= 0:
-        wl = wl.scaled(comm_interval=args.comm_interval)
+    from paper_1505_04956_b200 import inputs, metrics
     # each rank owns an independent group of W workers on its own seeded shard (no cross-GPU exchange)
     wl_rank = wl.scaled(seed=dist.shard_seed(wl.seed, rank, world))
     X, mu = inputs.make_samples(wl_rank, device=dev)
     w0 = inputs.initial_centres(wl_rank, X)
     cfg = pkg.make_config(N=wl.N, d=wl.d, k=wl.k, W=wl.W, b=wl.b, eps=wl.eps, comm_interval=wl.comm_interval,
                           fanout=wl.fanout, seed=wl_rank.seed, parzen=0 if args.no_parzen else 1,
-                          partial_rows=args.partial_rows)
+                          partial_rows=args.partial_rows, dist_path=args.dist_path)
     ctx = pkg.Asgd(cfg, X, w0)
     steps = wl.B                                   # one pass
     samples_per_pass = wl.W * steps * wl.b
@@ -227,7 +222,7 @@ def main():
     for _ in range(args.warmup):
         ctx.run(steps)
     ctx.sync()
-    sampler = ClockSampler(local)
+    sampler = ClockSampler(dev.index)
     l0 = ctx.launch_count()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     dist.barrier()
@@ -247,7 +242,6 @@ def main():
     value = world * samples_per_pass * args.steps / (total_ms * 1e-3)
     E_final = ctx.eval(0)
     E_mean = ctx.eval(-1)
-    from paper_1505_04956_b200 import metrics
     centre_err, _ = metrics.generator_centre_error(mu.cpu().numpy(), ctx.get_state(0).cpu().numpy())
     msgs = {"sent": 0, "received": 0, "accepted": 0, "overwritten": 0}
     for i in range(wl.W):
@@ -256,41 +250,115 @@ def main():
             msgs[key] += st[key]
 
     # roofline of the dominant kernel (the persistent worker kernel: one launch per bench step)
-    peak, peak_kind = measured_peaks()
+    kernel = ctx.path_name()
+    hbm_peak, peak_kind = measured_peaks()
     launch_ms = statistics.mean(per_launch_ms)
     bytes_per_launch = algorithmic_bytes_per_pass(wl, steps, args.partial_rows)
-    achieved = bytes_per_launch / (launch_ms * 1e-3) / 1e9
-    traffic = None
-    if ctx.path_name() == "fp32-stream" and stream_kernel_sha1() == TRAFFIC_CAPTURE["kernel_sha1"]:
-        traffic = bytes_per_launch * TRAFFIC_CAPTURE["traffic_per_algorithmic_byte"]
-    if ctx.path_name() in ("fp32-tiled",):
+    hbm_gbs = bytes_per_launch / (launch_ms * 1e-3) / 1e9
+    traffic, traffic_kind = captured_traffic(kernel, wl.name, bytes_per_launch)
+    flops = 2.0 * wl.k * wl.d * samples_per_pass
+    common = {"traffic": traffic, "traffic_kind": traffic_kind, "kernel": kernel, "launch_ms": launch_ms,
+              "algorithmic_bytes_per_launch": bytes_per_launch}
+    dtype = "f32"
+    if kernel == "fp32-tiled":
         # bound by the fp32 pipe: 2*k*d flops per sample against SMs x 128 lanes x 2 x max SM clock
         props = torch.cuda.get_device_properties(dev)
         alu_peak = props.multi_processor_count * 128 * 2 * (clocks.get("sm_max_mhz") or 1965.0) * 1e6 / 1e12
-        flops = 2.0 * wl.k * wl.d * samples_per_pass
         ach = flops / (launch_ms * 1e-3) / 1e12
-        roofline_alu = {"bound": "alu", "achieved": ach, "peak": alu_peak, "unit": "TFLOP/s", "frac": ach / alu_peak,
-                        "traffic": None, "peak_kind": "SMs x 128 fp32 lanes x 2 x max SM clock", "kernel": ctx.path_name(),
-                        "launch_ms": launch_ms, "algorithmic_flops_per_launch": flops,
-                        "hbm_GBs": achieved}
-    elif ctx.path_name().startswith("tcgen05"):
-        # bound by the tensor pipe: the 2*k*d flops per sample of the -2 X W^T contraction against the measured
-        # sustained BF16 rate (the kernel is timed inside a long launch)
+        roofline = dict(common, bound="alu", achieved=ach, peak=alu_peak, unit="TFLOP/s", frac=ach / alu_peak,
+                        peak_kind="SMs x 128 fp32 lanes x 2 x max SM clock", algorithmic_flops_per_launch=flops, hbm_GBs=hbm_gbs)
+    elif kernel.startswith("tcgen05"):
+        # bound by the tensor pipe: the 2*k*d flops per sample of the -2 X W^T contraction against the measured sustained
+        # BF16 rate (FP16 and BF16 share one nominal rate; the kernel is timed inside a long launch)
         tpeak, tkind = 1400.0, "fallback (sustained)"
         ppath = os.path.join(ROOT, "MEASURED_PEAKS.json")
         if os.path.exists(ppath):
             with open(ppath) as f:
                 tpeak, tkind = float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
-        flops = 2.0 * wl.k * wl.d * samples_per_pass
         ach = flops / (launch_ms * 1e-3) / 1e12
-        roofline_alu = {"bound": "tensor", "achieved": ach, "peak": tpeak, "unit": "TFLOP/s", "frac": ach / tpeak,
-                        "traffic": None, "peak_kind": "of " + tkind, "kernel": ctx.path_name(), "launch_ms": launch_ms,
-                        "algorithmic_flops_per_launch": flops, "hbm_GBs": achieved}
+        roofline = dict(common, bound="tensor", achieved=ach, peak=tpeak, unit="TFLOP/s", frac=ach / tpeak,
+                        peak_kind="of " + tkind, algorithmic_flops_per_launch=flops, hbm_GBs=hbm_gbs)
+        dtype = "f16" if kernel.endswith("fp16") else "bf16"
     else:
-        roofline_alu = None
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": traffic, "peak_kind": "of " + peak_kind, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "kernel": ctx.path_name(), "launch_ms": launch_ms, "algorithmic_bytes_per_launch": bytes_per_launch}
+        roofline = dict(common, bound="hbm", achieved=hbm_gbs, peak=hbm_peak, unit="GB/s", frac=hbm_gbs / hbm_peak,
+                        peak_kind="of " + peak_kind, frac_of_nominal_8TBs=hbm_gbs / NOMINAL_HBM_GBS)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": dtype, "data": "synthetic",
+        "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "k": wl.k, "W": wl.W, "b": wl.b, "eps": wl.eps,
+                   "comm_interval": wl.comm_interval, "fanout": wl.fanout, "parzen": 0 if args.no_parzen else 1,
+                   "partial_rows": args.partial_rows, "mode": "free-running",
+                   "steps_per_worker_per_bench_step": steps, "parallelism": "dp%d" % world,
+                   "l2": "inputs larger than L2 (%.2f GB per pass)" % (bytes_per_launch / 1e9)},
+        "roofline": roofline, "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
+        "quantization_error_worker0": E_final, "quantization_error_mean_state": E_mean,
+        "generator_centre_error_worker0": centre_err, "messages": msgs, "messages_over_passes": args.warmup + args.steps,
+    }
+    if keep:
+        return line, (ctx, cfg, X, w0, steps, samples_per_pass)
+    ctx.destroy()
+    del ctx, X
+    torch.cuda.empty_cache()
+    return line, None
+
+
+# workloads other than the headline one: (name, overrides) in the order of the table they make
+OTHER_WORKLOADS = [("mid", {})] + \
+    [("sweep", {"W": W, "comm_interval": c}) for W in (148, 296, 592, 1184, 2368) for c in (1, 10, 100)] + \
+    [("dense", {}), ("codebook", {})]
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="stream")
+    ap.add_argument("--all-workloads", action="store_true",
+                    help="one line per other workload (mid, the W x c grid of sweep, dense, codebook) instead of the headline line")
+    ap.add_argument("--rows", type=int, default=0, help="use only the first ROWS rows (profiling of a small case)")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--reference-rows", type=int, default=1 << 23)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    # points of the worker / communication sweep and the ablations (the defaults are the workload's own values)
+    ap.add_argument("--workers", type=int, default=0, help="W")
+    ap.add_argument("--comm-interval", type=int, default=-1, help="c; 0 = silent (no puts)")
+    ap.add_argument("--no-parzen", action="store_true", help="accept every non-empty message (Eq. 3 without Eq. 4)")
+    ap.add_argument("--partial-rows", type=int, default=0, help="centre rows per message (Section 4.4); 0 = whole state")
+    ap.add_argument("--dist-path", type=int, default=0, help="ASGD_PATH_* (0 = the library's choice)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import paper_1505_04956_b200 as pkg
+    from paper_1505_04956_b200 import dist, inputs
+
+    args.warmup = max(args.warmup, 3)
+    rank, world, local = dist.init_from_env(backend="nccl")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    pkg.load()
+
+    if args.all_workloads:
+        for name, over in OTHER_WORKLOADS:
+            line, _ = measure(args, inputs.WORKLOADS[name].scaled(**over), dev, rank, world, dist)
+            if rank == 0:
+                print(json.dumps(line), flush=True)
+        dist.shutdown()
+        return 0
+
+    wl = inputs.WORKLOADS[args.workload]
+    if args.rows:
+        wl = wl.scaled(N=args.rows)
+    if args.workers:
+        wl = wl.scaled(W=args.workers)
+    if args.comm_interval >= 0:
+        wl = wl.scaled(comm_interval=args.comm_interval)
+    line, (ctx, cfg, X, w0, steps, samples_per_pass) = measure(args, wl, dev, rank, world, dist, keep=True)
 
     # end to end through the host-buffer entry point: H2D of X and w0, the pass, D2H of w^1
     e2e = None
@@ -324,21 +392,13 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, desc, th = cpu_baseline(wl, CPU_SAMPLE_ROWS, min_seconds=2.0)
-        cpu = {"value": v, "unit": UNIT, "cores": th, "kind": "oracle", "sample": desc}
+        v1, desc1, _ = cpu_baseline(wl, CPU_SAMPLE_ROWS_ONE_CORE, threads=1, min_seconds=2.0)
+        cpu = {"value": v, "unit": UNIT, "cores": th, "kind": "oracle", "sample": desc,
+               "single_core": {"value": v1, "unit": UNIT, "cores": 1, "sample": desc1}}
 
     if rank == 0:
-        line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": wl.name, "N": wl.N, "d": wl.d, "k": wl.k, "W": wl.W, "b": wl.b, "eps": wl.eps,
-                       "comm_interval": wl.comm_interval, "fanout": wl.fanout, "parzen": 0 if args.no_parzen else 1,
-                       "partial_rows": args.partial_rows, "mode": "free-running",
-                       "steps_per_worker_per_bench_step": steps, "parallelism": "dp%d" % world,
-                       "l2": "inputs larger than L2 (%.2f GB per pass)" % (bytes_per_launch / 1e9)},
-            "roofline": roofline_alu or roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
-            "quantization_error_worker0": E_final, "quantization_error_mean_state": E_mean, "generator_centre_error_worker0": centre_err, "messages": msgs, "messages_over_passes": args.warmup + args.steps,
-        }
+        line["e2e"] = e2e
+        line["cpu_baseline"] = cpu
         print(json.dumps(line), flush=True)
     dist.shutdown()
     return 0

@@ -27,9 +27,15 @@ def test_algorithmic_bytes_of_the_stream_workload():
     assert bench.algorithmic_bytes_per_pass(wl.scaled(comm_interval=0), wl.B) == samples
 
 
-def test_traffic_record_is_keyed_on_the_kernel_sources():
+def test_traffic_records_are_keyed_on_the_kernel_sources():
     bench = _bench()
-    key = bench.stream_kernel_sha1()
-    assert re.fullmatch(r"[0-9a-f]{12}", key)
-    assert re.fullmatch(r"[0-9a-f]{12}", bench.TRAFFIC_CAPTURE["kernel_sha1"])
-    assert 1.0 <= bench.TRAFFIC_CAPTURE["traffic_per_algorithmic_byte"] < 1.05
+    for (kernel, workload), rec in bench.TRAFFIC_CAPTURES.items():
+        assert kernel in bench.KERNEL_SOURCES
+        assert re.fullmatch(r"[0-9a-f]{12}", bench.kernel_sha1(kernel))
+        assert 0.5 <= rec["traffic_per_algorithmic_byte"] < 8.0
+    # a record taken on other sources is not used
+    bench.TRAFFIC_CAPTURES[("fp32-stream", "stream")] = {"kernel_sha1": "000000000000", "traffic_per_algorithmic_byte": 1.0}
+    assert bench.captured_traffic("fp32-stream", "stream", 1000)[0] is None
+    bench.TRAFFIC_CAPTURES[("fp32-stream", "stream")]["kernel_sha1"] = bench.kernel_sha1("fp32-stream")
+    assert bench.captured_traffic("fp32-stream", "stream", 1000)[0] == 1000
+    assert bench.captured_traffic("fp32-generic", "tiny", 1000)[0] is None
