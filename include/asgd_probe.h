@@ -1,0 +1,32 @@
+/*
+ * libasgd_probe -- issue-rate probes for sm_100a (a measuring aid of the K-Means ASGD library; the paper has no
+ * counterpart).  The notes on the worker kernels quote what an instruction kind costs in issue slots on a B200;
+ * this entry point measures those numbers on the GPU at hand.
+ */
+#ifndef ASGD_PROBE_H_
+#define ASGD_PROBE_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/*
+ * Cycles one of an SM's four schedulers spends per warp instruction (clock64 around unrolled loops, one block of
+ * 16 warps per SM) for thirteen instruction streams, in this order:
+ *   0 FFMA with two immediate operands      1 FFMA acc = x * w + acc (three registers)
+ *   2 the packed two-wide FMA in that form  3 the packed two-wide add
+ *   4 LOP3    5 FMNMX    6 FSET    7 IMAD   8 mma.sync m16n8k8 TF32 (the legacy tensor-core product)
+ *   9 LOP3 and FFMA alternating            10 LOP3 and the packed FMA alternating
+ *  11 one tensor-core product with six FFMA                12 one tensor-core product with four LOP3
+ *   out_host     HOST [n_out], n_out >= 13 (written)
+ *   scratch_dev  DEVICE, at least 4 * (1 + sms * 512) bytes, caller's; overwritten
+ *   sms          blocks to launch (the GPU's SM count)
+ * Launches on the default stream and synchronises.  Returns 0; -1 for a NULL pointer, n_out < 13 or sms < 1
+ * (nothing is launched); -3 when a CUDA call failed.
+ */
+int asgd_probe_issue_rates(float *out_host, int n_out, float *scratch_dev, int sms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ASGD_PROBE_H_ */

@@ -42,5 +42,24 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+PROBE_LIB = os.path.join(PKG, "libasgd_probe.so")
+
+
+def build_probe(force: bool = False) -> str:
+    """Compile the issue-rate probes (csrc/asgd_probe.cu) into their own library; return its path."""
+    src = os.path.join(CSRC, "asgd_probe.cu")
+    if not force and os.path.exists(PROBE_LIB) and os.path.getmtime(PROBE_LIB) >= os.path.getmtime(src):
+        return PROBE_LIB
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    tmp = PROBE_LIB + ".%d.tmp" % os.getpid()
+    res = subprocess.run([nvcc] + NVCC_FLAGS + [src, "-o", tmp], stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout)
+        raise RuntimeError("nvcc failed building libasgd_probe.so")
+    os.replace(tmp, PROBE_LIB)
+    return PROBE_LIB
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build_probe(force="--force" in sys.argv))

@@ -155,7 +155,7 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
       if (fresh) {
         const float* __restrict__ v = p.mail + si * (size_t)p.kd_pad;
         double dot = 0.0, dd = 0.0, nv = 0.0;
-#pragma unroll 4
+#pragma unroll 8
         for (int q = tid; q < nvec; q += nt) {
           const int e = q * V;
           const TailVec<V> vv = tail_ldcg<V>(v + e);
@@ -225,7 +225,7 @@ __device__ inline void step_tail_impl(const Params& p, int i, unsigned long long
 
   // Eq. 6: Dbar = w - (w + sum_s a_s v_s) / (1 + sum_s a_s) + D ;  w <- w - eps * Dbar   (a_s per row in per-centre mode)
   const float inv_m1_whole = 1.0f / (float)(1 + m);
-#pragma unroll 4
+#pragma unroll 8
   for (int q = tid; q < nvec; q += nt) {
     const int e = q * V;
     const unsigned bits = by_rows ? rowacc[e / d] : whole_bits;

@@ -240,16 +240,16 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         sq = fmaf(w4[q].x, w4[q].x, sq); sq = fmaf(w4[q].y, w4[q].y, sq); sq = fmaf(w4[q].z, w4[q].z, sq); sq = fmaf(w4[q].w, w4[q].w, sq);
         const size_t o = (size_t)a * d + 4 * l8 + 32 * q;
         const float v[4] = {-2.f * w4[q].x, -2.f * w4[q].y, -2.f * w4[q].z, -2.f * w4[q].w};     // exact
+        // four 16-bit numbers per store (8 bytes; o is a multiple of 4)
         if (kTerms == 1) {
-          *reinterpret_cast<__half2*>(wbf + o) = __floats2half2_rn(v[0], v[1]);
-          *reinterpret_cast<__half2*>(wbf + o + 2) = __floats2half2_rn(v[2], v[3]);
+          const __half2 h01 = __floats2half2_rn(v[0], v[1]), h23 = __floats2half2_rn(v[2], v[3]);
+          *reinterpret_cast<uint2*>(wbf + o) = make_uint2(*reinterpret_cast<const unsigned*>(&h01), *reinterpret_cast<const unsigned*>(&h23));
         } else {
           const __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
           const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
-          *reinterpret_cast<__nv_bfloat162*>(wbf + o) = h01;
-          *reinterpret_cast<__nv_bfloat162*>(wbf + o + 2) = h23;
-          *reinterpret_cast<__nv_bfloat162*>(wbl + o) = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y);
-          *reinterpret_cast<__nv_bfloat162*>(wbl + o + 2) = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+          const __nv_bfloat162 l01 = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y), l23 = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+          *reinterpret_cast<uint2*>(wbf + o) = make_uint2(*reinterpret_cast<const unsigned*>(&h01), *reinterpret_cast<const unsigned*>(&h23));
+          *reinterpret_cast<uint2*>(wbl + o) = make_uint2(*reinterpret_cast<const unsigned*>(&l01), *reinterpret_cast<const unsigned*>(&l23));
         }
       }
     }

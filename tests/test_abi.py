@@ -25,6 +25,18 @@ def test_library_builds_and_exports_every_declared_symbol():
     assert set(names) == set(pkg.EXPORTS)
 
 
+def test_probe_library_builds_and_exports_its_entry_point():
+    text = open(os.path.join(ROOT, "include", "asgd_probe.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = sorted(set(re.findall(r"\b(asgd_[a-z0-9_]+)\s*\(", text)))
+    assert names == ["asgd_probe_issue_rates"]
+    lib = C.CDLL(libbuild.build_probe())
+    for n in names:
+        assert hasattr(lib, n), n
+    lib.asgd_probe_issue_rates.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int]
+    assert lib.asgd_probe_issue_rates(None, 13, None, 148) == -1           # argument check, nothing launched
+
+
 def test_argument_checks_need_no_gpu():
     L = pkg.load()
     cfg = pkg.make_config(N=1000, d=4, k=3, W=2, b=10, eps=0.1, comm_interval=1, fanout=1)

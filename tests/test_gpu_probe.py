@@ -1,0 +1,15 @@
+"""The issue-rate probes run and give numbers of the expected kind (a B200 is assumed, not particular values)."""
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+def test_issue_rates_are_plausible():
+    from paper_1505_04956_b200 import peaks
+    r = dict(zip(peaks.NAMES, peaks.issue_rates()))
+    assert len(r) == 13
+    for name, v in r.items():
+        assert 0.4 < v < 40.0, (name, v)
+    # a scalar FMA issues about every cycle; the half-rate kinds take about two
+    assert r["FFMA (two immediates)"] < 1.5
+    assert r["LOP3"] > 1.5 * r["FFMA (two immediates)"]
