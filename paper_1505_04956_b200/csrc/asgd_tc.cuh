@@ -752,14 +752,18 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           if (plain) {
             float4 w4[TC_MAX_D / 32];
             const float fn = (float)n;
+            // all of the centre's row first, then the stores: a store between two loads from the same array would keep
+            // the second load behind it (they might alias), one L2 round trip per piece instead of one per row
+#pragma unroll
+            for (int q = 0; q < TC_MAX_D / 32; ++q)
+              if (q < nq) w4[q] = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q);
 #pragma unroll
             for (int q = 0; q < TC_MAX_D / 32; ++q) {
               if (q < nq) {
-                float* wp = wglob + (size_t)a * d + 4 * l8 + 32 * q;
-                float4 u = *reinterpret_cast<const float4*>(wp);
+                float4 u = w4[q];
                 u.x -= p.eps * ((fn * u.x - S4[q].x) * inv_b); u.y -= p.eps * ((fn * u.y - S4[q].y) * inv_b);
                 u.z -= p.eps * ((fn * u.z - S4[q].z) * inv_b); u.w -= p.eps * ((fn * u.w - S4[q].w) * inv_b);
-                *reinterpret_cast<float4*>(wp) = u;
+                *reinterpret_cast<float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q) = u;
                 w4[q] = u;
               }
             }
