@@ -198,7 +198,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   unsigned short* best = reinterpret_cast<unsigned short*>(smem + map.best);
   unsigned short* flagged = reinterpret_cast<unsigned short*>(smem + map.flagged);
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + map.bars);
-  int* misc = reinterpret_cast<int*>(smem + map.misc);                 // [0] tmem base, [1] pairs to settle, [2] abort, [4] news, [5] rows for the full scan
+  int* misc = reinterpret_cast<int*>(smem + map.misc);                 // [0] tmem base, [1] pairs to settle, [2] abort, [4] news, [5] rows for the full scan, [6] rows with three candidates
   TailScratch* ts = reinterpret_cast<TailScratch*>(smem + map.tail);
 
   static_assert(kTerms == 1 || kTerms == 3, "one FP16 term or two BF16 terms per operand");
@@ -368,8 +368,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       for (int m = 0; m < m_tiles; ++m) {
         const int r = m * TC_M + quarter * 32 + lane;              // the thread's row of the batch
         const float xn = (r < b) ? __ldg(p.xnorm + row0 + r) : 0.f;
-        float m1[2], m2[2], m3[2];                                  // two independent sorted triples, kept over the centre blocks
-        m1[0] = m1[1] = m2[0] = m2[1] = m3[0] = m3[1] = INF;
+        float m1[4], m2[4], m3[4];                                  // four independent sorted triples, kept over the centre blocks
+#pragma unroll
+        for (int q = 0; q < 4; ++q) m1[q] = m2[q] = m3[q] = INF;
         for (int n = 0; n < n_tiles; ++n, ++iacc) {
           const int buf = iacc & 1;
           if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bars + TCB_ACCFULL + buf, (iacc >> 1) & 1, p.wait_limit));
@@ -407,18 +408,27 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
                 asm("lop3.b32 %0, %1, %2, %3, 0xE6;" : "=r"(spb) : "r"(__float_as_uint(d2)), "r"(hi_or_base), "r"(~TC_INDEX_MASK | (unsigned)(c + u)));
                 sp[u] = __uint_as_float(spb);
               }
-              tc_top3_insert2(m1[0], m2[0], m3[0], sp[0], sp[1]);
-              tc_top3_insert2(m1[1], m2[1], m3[1], sp[2], sp[3]);
+              const int sq = (c >> 1) & 2;                        // columns 0-3 of every eight feed triples 0 and 1, columns 4-7 triples 2 and 3
+              tc_top3_insert2(m1[sq], m2[sq], m3[sq], sp[0], sp[1]);
+              tc_top3_insert2(m1[sq + 1], m2[sq + 1], m3[sq + 1], sp[2], sp[3]);
             }
           }
         }
         if (ok && r < b) {
-          // merge the two sorted triples: the three smallest of the six
-          float a1 = m1[0], a2 = m2[0], a3 = m3[0];
-          tc_top3_insert(a1, a2, a3, m1[1]);
-          tc_top3_insert(a1, a2, a3, m2[1]);
-          tc_top3_insert(a1, a2, a3, m3[1]);
-          __stcg(top3 + r, make_float4(a1, a2, a3, 0.f));
+          // the four smallest of the twelve kept values.  Every value that was not kept is at least the largest of its
+          // triple, so the fourth smallest of ALL values is at least min(fourth smallest kept, smallest of the four
+          // triples' largest): a floor under the fourth candidate that costs nothing in the loop above
+          float a1 = INF, a2 = INF, a3 = INF, a4 = INF;
+          auto put4 = [&](float v) {
+            const float h1 = fmaxf(a1, v); a1 = fminf(a1, v);
+            const float h2 = fmaxf(a2, h1); a2 = fminf(a2, h1);
+            const float h3 = fmaxf(a3, h2); a3 = fminf(a3, h2);
+            a4 = fminf(a4, h3);
+          };
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { put4(m1[q]); put4(m2[q]); put4(m3[q]); }
+          const float floor4 = fminf(a4, fminf(fminf(m3[0], m3[1]), fminf(m3[2], m3[3])));
+          __stcg(top3 + r, make_float4(a1, a2, a3, floor4));
         }
       }
       if (!ok && lane == 0) atomicExch(&misc[2], 1);
@@ -426,7 +436,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     it_m += (unsigned)m_tiles;
     it_bc += (unsigned)(m_tiles * n_tiles * PPK * nkc);
     it_acc += (unsigned)(n_tiles * m_tiles);
-    if (tid == 0) { misc[1] = 0; misc[5] = 0; }
+    if (tid == 0) { misc[1] = 0; misc[5] = 0; misc[6] = 0; }
     for (int a = tid; a < k; a += TC_THREADS) cnt[a] = 0;
     tc_fence_before();
     __syncthreads();
@@ -459,6 +469,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     int* wcnt = reinterpret_cast<int*>(sA);                                   // [TC_WARPS][k] rows of a centre in a warp's row block
     unsigned short* lrank = reinterpret_cast<unsigned short*>(sA + (size_t)TC_WARPS * k * 4);   // [b] rank of a row among its warp's rows of the centre
     unsigned short* order = flagged;                                          // [b] rows grouped by centre, ascending inside a group
+    unsigned short* triples = lrank;                                          // until the grouping: rows with exactly three candidates
 
     // ---- decide: the minimum, unless the runner-up lies inside the bound (settle the pair) or the third does too (scan all) ----
     for (int e = tid; e < TC_WARPS * k; e += TC_THREADS) wcnt[e] = 0;
@@ -467,75 +478,92 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       best[r] = (unsigned short)(__float_as_uint(s.x) & TC_INDEX_MASK);
       const float err = row_err(__ldg(p.xnorm + row0 + r));
       if (k > 1 && inside(s.x, s.y, err)) {
-        if (k > 2 && inside(s.x, s.z, err)) order[b - 1 - atomicAdd(&misc[5], 1)] = (unsigned short)r;
-        else order[atomicAdd(&misc[1], 1)] = (unsigned short)r;
+        if (k > 2 && inside(s.x, s.z, err)) {
+          if (k > 3 && inside(s.x, s.w, err)) order[b - 1 - atomicAdd(&misc[5], 1)] = (unsigned short)r;   // a fourth may be inside: all centres
+          else triples[atomicAdd(&misc[6], 1)] = (unsigned short)r;                                         // exactly three candidates
+        } else {
+          order[atomicAdd(&misc[1], 1)] = (unsigned short)r;
+        }
       }
     }
     __syncthreads();
-    // ---- listed pairs are settled between their two candidates with fp32 inputs and fp64 sums: eight lanes per
-    //      row (lane l8 holds dimensions 4*l8 + 32*q), a warp settles four rows at a time ----
+    // ---- listed rows are settled among their two or three candidates with fp32 inputs (direct differences; fp64 sums
+    //      when the two smallest fp32 distances are within rounding of each other): eight lanes per row (lane l8 holds
+    //      dimensions 4*l8 + 32*q), a warp settles four rows at a time ----
     {
-      const int nflag = misc[1];
-      auto settle_load = [&](int f, float4 (&xv)[TC_MAX_D / 32], float4 (&a1)[TC_MAX_D / 32], float4 (&a2)[TC_MAX_D / 32], int& r,
-                             int& i1, int& i2) {
-        r = (f < nflag) ? (int)order[f] : -1;
+      const int npair = misc[1], ntrip = misc[6];
+      const int groups = TC_WARPS * 4;
+      for (int fb = wid * 4; fb < npair + ntrip; fb += groups) {   // the same trip count for all lanes of a warp (shuffles inside)
+        const int f = fb + sub;
+        const bool have = f < npair + ntrip;
+        const bool three = f >= npair;
+        const int r = have ? (int)(three ? triples[f - npair] : order[f]) : -1;
         const float4 s = (r >= 0) ? __ldcg(top3 + r) : make_float4(0.f, 0.f, 0.f, 0.f);
-        i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK);
-        i2 = (int)(__float_as_uint(s.y) & TC_INDEX_MASK);
+        const int i1 = (int)(__float_as_uint(s.x) & TC_INDEX_MASK), i2 = (int)(__float_as_uint(s.y) & TC_INDEX_MASK);
+        const int i3 = (have && three) ? (int)(__float_as_uint(s.z) & TC_INDEX_MASK) : i2;
         const float* x = p.X + (size_t)(row0 + max(r, 0)) * d + 4 * l8;
         const float* w1 = wglob + (size_t)i1 * d + 4 * l8;
         const float* w2 = wglob + (size_t)i2 * d + 4 * l8;
+        const float* w3 = wglob + (size_t)i3 * d + 4 * l8;
+        float4 xv[TC_MAX_D / 32], c1[TC_MAX_D / 32], c2[TC_MAX_D / 32], c3[TC_MAX_D / 32];
 #pragma unroll
         for (int q = 0; q < TC_MAX_D / 32; ++q) {
           if (q < nq && r >= 0) {
             xv[q] = __ldg(reinterpret_cast<const float4*>(x + 32 * q));
-            a1[q] = *reinterpret_cast<const float4*>(w1 + 32 * q);
-            a2[q] = *reinterpret_cast<const float4*>(w2 + 32 * q);
+            c1[q] = *reinterpret_cast<const float4*>(w1 + 32 * q);
+            c2[q] = *reinterpret_cast<const float4*>(w2 + 32 * q);
+            c3[q] = *reinterpret_cast<const float4*>(w3 + 32 * q);
           } else {
-            xv[q] = a1[q] = a2[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            xv[q] = c1[q] = c2[q] = c3[q] = make_float4(0.f, 0.f, 0.f, 0.f);
           }
         }
-      };
-      auto settle_finish = [&](const float4 (&xv)[TC_MAX_D / 32], const float4 (&a1)[TC_MAX_D / 32], const float4 (&a2)[TC_MAX_D / 32],
-                               int r, int i1, int i2) {
         // direct differences in fp32 first: each squared distance is off by at most (d + 2) u relative, so a gap
         // above (4 d + 16) u of the larger one decides; only rows closer than that are summed again in fp64
-        float f1 = 0.f, f2 = 0.f;
+        float f1 = 0.f, f2 = 0.f, f3 = 0.f;
 #pragma unroll
         for (int q = 0; q < TC_MAX_D / 32; ++q) {
           float u;
-          u = xv[q].x - a1[q].x; f1 = fmaf(u, u, f1); u = xv[q].y - a1[q].y; f1 = fmaf(u, u, f1);
-          u = xv[q].z - a1[q].z; f1 = fmaf(u, u, f1); u = xv[q].w - a1[q].w; f1 = fmaf(u, u, f1);
-          u = xv[q].x - a2[q].x; f2 = fmaf(u, u, f2); u = xv[q].y - a2[q].y; f2 = fmaf(u, u, f2);
-          u = xv[q].z - a2[q].z; f2 = fmaf(u, u, f2); u = xv[q].w - a2[q].w; f2 = fmaf(u, u, f2);
+          u = xv[q].x - c1[q].x; f1 = fmaf(u, u, f1); u = xv[q].y - c1[q].y; f1 = fmaf(u, u, f1);
+          u = xv[q].z - c1[q].z; f1 = fmaf(u, u, f1); u = xv[q].w - c1[q].w; f1 = fmaf(u, u, f1);
+          u = xv[q].x - c2[q].x; f2 = fmaf(u, u, f2); u = xv[q].y - c2[q].y; f2 = fmaf(u, u, f2);
+          u = xv[q].z - c2[q].z; f2 = fmaf(u, u, f2); u = xv[q].w - c2[q].w; f2 = fmaf(u, u, f2);
+          u = xv[q].x - c3[q].x; f3 = fmaf(u, u, f3); u = xv[q].y - c3[q].y; f3 = fmaf(u, u, f3);
+          u = xv[q].z - c3[q].z; f3 = fmaf(u, u, f3); u = xv[q].w - c3[q].w; f3 = fmaf(u, u, f3);
         }
 #pragma unroll
-        for (int o = 1; o < 8; o <<= 1) { f1 += __shfl_xor_sync(0xffffffffu, f1, o); f2 += __shfl_xor_sync(0xffffffffu, f2, o); }
-        bool second = f2 < f1;
-        const bool close = fabsf(f1 - f2) <= (float)(4 * TC_MAX_D + 16) * 5.9604645e-8f * fmaxf(f1, f2);
+        for (int o = 1; o < 8; o <<= 1) {
+          f1 += __shfl_xor_sync(0xffffffffu, f1, o); f2 += __shfl_xor_sync(0xffffffffu, f2, o); f3 += __shfl_xor_sync(0xffffffffu, f3, o);
+        }
+        if (!three) f3 = INF;                                                    // a pair has no third candidate
+        const float lo = fminf(f1, fminf(f2, f3));
+        const float mid = fmaxf(fminf(f1, f2), fminf(fmaxf(f1, f2), f3));       // the second smallest
+        int pick = (f1 == lo) ? i1 : (f2 == lo) ? i2 : i3;
+        const bool close = (mid - lo) <= (float)(4 * TC_MAX_D + 16) * 5.9604645e-8f * mid;
         if (__any_sync(0xffffffffu, close && r >= 0)) {       // warp-uniform: the shuffles below need every lane
-          double d1 = 0.0, d2 = 0.0;
+          double d1 = 0.0, d2 = 0.0, d3 = 0.0;
 #pragma unroll
           for (int q = 0; q < TC_MAX_D / 32; ++q) {
             double u;
-            u = (double)xv[q].x - (double)a1[q].x; d1 = fma(u, u, d1); u = (double)xv[q].y - (double)a1[q].y; d1 = fma(u, u, d1);
-            u = (double)xv[q].z - (double)a1[q].z; d1 = fma(u, u, d1); u = (double)xv[q].w - (double)a1[q].w; d1 = fma(u, u, d1);
-            u = (double)xv[q].x - (double)a2[q].x; d2 = fma(u, u, d2); u = (double)xv[q].y - (double)a2[q].y; d2 = fma(u, u, d2);
-            u = (double)xv[q].z - (double)a2[q].z; d2 = fma(u, u, d2); u = (double)xv[q].w - (double)a2[q].w; d2 = fma(u, u, d2);
+            u = (double)xv[q].x - (double)c1[q].x; d1 = fma(u, u, d1); u = (double)xv[q].y - (double)c1[q].y; d1 = fma(u, u, d1);
+            u = (double)xv[q].z - (double)c1[q].z; d1 = fma(u, u, d1); u = (double)xv[q].w - (double)c1[q].w; d1 = fma(u, u, d1);
+            u = (double)xv[q].x - (double)c2[q].x; d2 = fma(u, u, d2); u = (double)xv[q].y - (double)c2[q].y; d2 = fma(u, u, d2);
+            u = (double)xv[q].z - (double)c2[q].z; d2 = fma(u, u, d2); u = (double)xv[q].w - (double)c2[q].w; d2 = fma(u, u, d2);
+            u = (double)xv[q].x - (double)c3[q].x; d3 = fma(u, u, d3); u = (double)xv[q].y - (double)c3[q].y; d3 = fma(u, u, d3);
+            u = (double)xv[q].z - (double)c3[q].z; d3 = fma(u, u, d3); u = (double)xv[q].w - (double)c3[q].w; d3 = fma(u, u, d3);
           }
 #pragma unroll
-          for (int o = 1; o < 8; o <<= 1) { d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); }
-          if (close) second = (d2 < d1 || (d2 == d1 && i2 < i1));
+          for (int o = 1; o < 8; o <<= 1) {
+            d1 += __shfl_xor_sync(0xffffffffu, d1, o); d2 += __shfl_xor_sync(0xffffffffu, d2, o); d3 += __shfl_xor_sync(0xffffffffu, d3, o);
+          }
+          if (!three) d3 = 1e300;
+          if (close) {                                        // the smallest, the lowest index among equals
+            pick = i1;
+            double bd = d1;
+            if (d2 < bd || (d2 == bd && i2 < pick)) { bd = d2; pick = i2; }
+            if (d3 < bd || (d3 == bd && i3 < pick)) { bd = d3; pick = i3; }
+          }
         }
-        if (r >= 0 && l8 == 0 && second) best[r] = (unsigned short)i2;
-      };
-      const int groups = TC_WARPS * 4;
-      for (int fb = wid * 4; fb < nflag; fb += groups) {       // the same trip count for all lanes of a warp (shuffles inside)
-        const int f0 = fb + sub;
-        float4 xa[TC_MAX_D / 32], pa[TC_MAX_D / 32], qa[TC_MAX_D / 32];
-        int ra, ia1, ia2;
-        settle_load(f0, xa, pa, qa, ra, ia1, ia2);
-        settle_finish(xa, pa, qa, ra, ia1, ia2);
+        if (r >= 0 && l8 == 0) best[r] = (unsigned short)pick;
       }
     }
     // ---- rows with three or more candidates are decided over all centres, TC_SCAN_ROWS rows at a time: every lane
