@@ -34,6 +34,8 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "asgd_step_tail.cuh"
 #include "asgd_stream.cuh"   // mbarrier helpers
 
@@ -570,19 +572,20 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     //      holds its dimensions of all the rows in registers, every warp walks its share of the centres (a centre row is
     //      one coalesced read, lanes over the dimensions, the next centre's row already on its way) and measures it
     //      against every row with direct differences in fp32; the lanes' partial sums of all rows are added up by a
-    //      halving exchange (lanes 2j, 2j+1 end with row j's distance), and lane 2j keeps row j's two smallest.  A row
+    //      halving exchange (a run of lanes ends with row j's distance), and the first lane of the run keeps row j's three smallest.  A row
     //      whose two smallest are still within rounding of each other is measured once more in fp64. ----
     {
       __syncthreads();                                         // the pairs' readers of `order` and `top3` are done; the ring is idle
-      constexpr int RB = TC_SCAN_ROWS;
       const int nwide = misc[5];
       const int d4 = d / 4;
-      float* res = reinterpret_cast<float*>(sB);               // [TC_WARPS][RB][5] per warp and row: the three smallest, indices of the first two
-      int* need64 = reinterpret_cast<int*>(res + TC_WARPS * RB * 5);      // [RB][3]: 0 decided, 1 compare two in fp64, 2 scan all in fp64; the two indices
       const bool on0 = lane < d4, on1 = 32 + lane < d4;
       const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
-      for (int base = 0; base < nwide; base += RB) {           // block-uniform trip count
-        const int R = min(RB, nwide - base);
+      // one batch of R <= RB rows (RB = 16, or 4 for the usual handful: a quarter of the arithmetic per centre)
+      auto scan_batch = [&](auto rb_tag, const int base, const int R) {
+        constexpr int RB = decltype(rb_tag)::value;
+        constexpr int LPR = 32 / RB;                           // lanes that end up with the same row: LPR * j .. LPR * j + LPR - 1
+        float* res = reinterpret_cast<float*>(sB);             // [TC_WARPS][RB][5] per warp and row: the three smallest, indices of the first two
+        int* need64 = reinterpret_cast<int*>(res + TC_WARPS * RB * 5);    // [RB][3]: 0 decided, 1 compare two in fp64, 2 scan all in fp64; the two indices
         float4 xr0[RB], xr1[RB];                               // this lane's dimensions of the rows (zeros past the last row)
 #pragma unroll
         for (int j = 0; j < RB; ++j) {
@@ -590,7 +593,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           xr0[j] = (j < R && on0) ? __ldg(xrow + lane) : z4;
           xr1[j] = (j < R && on1) ? __ldg(xrow + 32 + lane) : z4;
         }
-        float bd1 = INF, bd2 = INF, bd3 = INF;                 // lane 2j: row j over this warp's centres
+        float bd1 = INF, bd2 = INF, bd3 = INF;                 // first lane of row j's run: row j over this warp's centres
         int bi1 = 0x7fffffff, bi2 = 0x7fffffff;
         const float4* wa = reinterpret_cast<const float4*>(wglob + (size_t)wid * d);
         float4 w0v = (wid < k && on0) ? wa[lane] : z4, w1v = (wid < k && on1) ? wa[32 + lane] : z4;
@@ -619,16 +622,18 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
               part[j] = keep + __shfl_xor_sync(0xffffffffu, send, o);
             }
           }
-          const float tot = part[0] + __shfl_xor_sync(0xffffffffu, part[0], 1);      // lanes 2j and 2j+1: row j
-          if ((lane & 1) == 0) {
+          float tot = part[0];                                  // lanes LPR * j .. : row j, each with a share of it
+#pragma unroll
+          for (int o = LPR / 2; o >= 1; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+          if ((lane & (LPR - 1)) == 0) {
             if (tot < bd1) { bd3 = bd2; bd2 = bd1; bi2 = bi1; bd1 = tot; bi1 = a; }
             else if (tot < bd2) { bd3 = bd2; bd2 = tot; bi2 = a; }
             else if (tot < bd3) { bd3 = tot; }
           }
           w0v = n0; w1v = n1;
         }
-        if ((lane & 1) == 0) {
-          const int j = lane >> 1;
+        if ((lane & (LPR - 1)) == 0) {
+          const int j = lane / LPR;
           float* o = res + (wid * RB + j) * 5;
           o[0] = bd1; o[1] = bd2; o[2] = bd3; o[3] = __int_as_float(bi1); o[4] = __int_as_float(bi2);
         }
@@ -692,8 +697,11 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           }
           if (lane == 0) best[order[b - 1 - (base + j)]] = (unsigned short)bi;
         }
-        __syncthreads();                                       // before the next rows overwrite the waiting area
-      }
+        __syncthreads();                                       // before the next batch overwrites the results
+      };
+      int base = 0;                                            // block-uniform trip counts
+      for (; nwide - base > 4; base += TC_SCAN_ROWS) scan_batch(std::integral_constant<int, TC_SCAN_ROWS>(), base, min(TC_SCAN_ROWS, nwide - base));
+      if (base < nwide) scan_batch(std::integral_constant<int, 4>(), base, nwide - base);
     }
     __syncthreads();
     if (p.assign_rec)
