@@ -113,6 +113,36 @@ def test_tensor_core_formats_decide_exactly(name, fmt):
     pr.close()
 
 
+@pytest.mark.parametrize("fmt", ["fp16", "bf16x3"])
+def test_tensor_core_rows_with_many_candidates(fmt):
+    """Bundles of five centres a hair apart: for the rows of their clusters the rounding bound of the 16-bit scores
+    leaves three, four or five candidates, so the triple settlement and the scans over all centres (batches of 16 and
+    of 4 rows) decide them; every decided row must still get the oracle's centre."""
+    rng = np.random.default_rng(77)
+    k, d, b, W = 200, 64, 256, 2
+    wl = scaled("dense", N=W * b * 3 + 9, k=k, d=d, b=b, W=W, comm_interval=2, eps=0.01)
+    mu = rng.standard_normal((8, d)) * 5.0
+    X = (mu[rng.integers(0, 8, wl.N)] + rng.standard_normal((wl.N, d))).astype(np.float32)
+    w0 = (rng.standard_normal((k, d)) * 5.0 + 40.0).astype(np.float32)            # far from every sample ...
+    for c in range(8):                                                             # ... but for a bundle of five per cluster
+        for j in range(5):
+            w0[5 * c + j] = (mu[c] + (2e-3 if fmt == "fp16" else 2e-4) * rng.standard_normal(d)).astype(np.float32)
+    pr = Pair(wl, X=X, w0=w0, dist_path=pkg.PATH_TC_FP16 if fmt == "fp16" else pkg.PATH_TC_BF16)
+    assert pr.gpu.path_name() == "tcgen05-" + fmt
+    pr.rounds(1)
+    pr.gpu.sync()
+    got = pr.gpu.get_assign().cpu().numpy()
+    decided_rows = 0
+    for i in range(wl.W):
+        tr = pr.cpu.last_step(i)
+        ok = decided(tr["d1"], tr["d2"])
+        assert (got[i][ok] == tr["assign"][ok]).all(), (fmt, i, int((got[i][ok] != tr["assign"][ok]).sum()))
+        decided_rows += int(ok.sum())
+    assert decided_rows > 0.5 * wl.W * wl.b
+    assert pr.max_rel_l2() < CENTRE_TOL
+    pr.close()
+
+
 def test_fp16_format_refuses_samples_outside_its_range():
     wl = scaled("dense", N=2 * 256 * 3, W=2, b=256, k=200, d=64, comm_interval=1)
     X = np.random.default_rng(3).standard_normal((wl.N, wl.d)).astype(np.float32) * 3.0e4      # ||x|| far beyond 65504 / 8
