@@ -40,6 +40,7 @@ struct Layout {
 constexpr size_t kAlign = 256;
 constexpr int kEvalBlocks = 148 * 8;
 constexpr size_t kMaxDynSmem = 227 * 1024;
+constexpr size_t kTwoBlockSmem = 113 * 1024;      // two blocks, each with its reserved kilobyte, in an SM's 228 KB
 
 inline size_t up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 
@@ -58,10 +59,17 @@ bool config_ok(const asgd_config* c) {
   return true;
 }
 
-// shapes the tensor-core path takes: d a multiple of 64 up to 256, more centres than the tiled path holds
-bool tc_eligible(const asgd_config* c) {
-  return c->d % TC_KC == 0 && c->d <= TC_MAX_D && c->k > 128 && c->k <= TC_MAX_K && c->b >= TC_M && c->b <= TC_MAX_B &&
-         tc_smem_bytes(c->k, c->d, c->b, 1) <= kMaxDynSmem && tc_smem_bytes(c->k, c->d, c->b, 3) <= kMaxDynSmem;
+// shapes the tensor-core path can take: d a multiple of 64 up to 256, a batch of at least one 128-row tile
+bool tc_supported(const asgd_config* c) {
+  return c->d % TC_KC == 0 && c->d <= TC_MAX_D && c->k >= 1 && c->k <= TC_MAX_K && c->b >= TC_M && c->b <= TC_MAX_B &&
+         tc_smem_bytes(c->k, c->d, c->b, 1, 1) <= kMaxDynSmem && tc_smem_bytes(c->k, c->d, c->b, 3, 1) <= kMaxDynSmem;
+}
+// ... and these are the library's own choice for them
+bool tc_eligible(const asgd_config* c) { return tc_supported(c); }
+// the path a configuration asks for is a tensor-core one
+bool tc_wanted(const asgd_config* c) {
+  if (c->dist_path == ASGD_PATH_TC_BF16 || c->dist_path == ASGD_PATH_TC_FP16) return tc_supported(c);
+  return c->dist_path == ASGD_PATH_AUTO && tc_eligible(c);
 }
 
 Layout make_layout(const asgd_config* c) {
@@ -91,7 +99,7 @@ Layout make_layout(const asgd_config* c) {
   L.xmax = take(64);
   // tensor-core path: 16-bit copies of -2w and of the samples (one FP16 term, or the two BF16 terms), the three
   // best per row, the row norms
-  const bool tc = tc_eligible(c) && (c->dist_path == ASGD_PATH_TC_BF16 || c->dist_path == ASGD_PATH_TC_FP16 || c->dist_path == ASGD_PATH_AUTO);
+  const bool tc = tc_wanted(c);
   const bool two_terms = tc && c->dist_path == ASGD_PATH_TC_BF16;
   L.wbf = take(tc ? (two_terms ? 2 : 1) * W * kd * 2 : 4);
   L.top2 = take(tc ? W * (size_t)c->b * 16 : 4);
@@ -114,6 +122,7 @@ struct asgd_ctx {
   int state_on_chip;
   int grid;               // blocks of the worker kernel (tiled path: a block may serve several workers)
   int tiled_shape;        // index into ASGD_TILED_SHAPES of the shape in use
+  int tc_two;             // tensor-core path: the instance that shares an SM between two blocks
   size_t smem_bytes;
   long long t_host;       // steps every worker has done (uniform across workers)
   long long launches;
@@ -225,14 +234,30 @@ int tc_prepare(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
   Params& p = c->p;
   const bool fp16 = (c->path == P_TC_FP16);
-  c->smem_bytes = tc_smem_bytes(cfg.k, cfg.d, cfg.b, fp16 ? 1 : 3);
-  if (fp16) {
-    CU(c, cudaFuncSetAttribute(asgd_tc_kernel<true, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
-    CU(c, cudaFuncSetAttribute(asgd_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
-  } else {
-    CU(c, cudaFuncSetAttribute(asgd_tc_kernel<true, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
-    CU(c, cudaFuncSetAttribute(asgd_tc_kernel<false, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes));
+  const int terms = fp16 ? 1 : 3;
+  const int bn = tc_block_rows(cfg.k, terms);
+  // Two blocks per SM (the half-register instance) when there are more workers than SMs, rows of at most 128 numbers,
+  // accumulators of at most 256 tensor-memory columns a block, and room for two blocks' shared memory; else one.
+  // The request is padded so that no more blocks than that share an SM (tensor memory has 512 columns).
+  {
+    const int grid2 = std::min(cfg.W, 2 * c->sm_count);
+    const size_t smem2 = tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, (cfg.W + grid2 - 1) / grid2);
+    c->tc_two = cfg.W > c->sm_count && cfg.d <= 128 && tc_tmem_cols(bn) <= 256 && smem2 <= kTwoBlockSmem;
+    if (c->tc_two) {
+      c->grid = grid2;
+      c->smem_bytes = std::max(smem2, (size_t)(kMaxDynSmem / 3 + 1024));
+    } else {
+      c->grid = std::min(cfg.W, c->sm_count);
+      c->smem_bytes = std::max(tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, (cfg.W + c->grid - 1) / c->grid), (size_t)(kMaxDynSmem / 2 + 1024));
+      if (c->smem_bytes > kMaxDynSmem) return ASGD_EUNSUPPORTED;
+    }
   }
+#define TC_SET(DET_, T_, D_) CU(c, cudaFuncSetAttribute(asgd_tc_kernel<DET_, T_, D_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes))
+  if (fp16 && c->tc_two) { TC_SET(true, 1, 128); TC_SET(false, 1, 128); }
+  else if (fp16) { TC_SET(true, 1, 256); TC_SET(false, 1, 256); }
+  else if (c->tc_two) { TC_SET(true, 3, 128); TC_SET(false, 3, 128); }
+  else { TC_SET(true, 3, 256); TC_SET(false, 3, 256); }
+#undef TC_SET
   p.wbf = c->ws + c->L.wbf;
   p.top2 = (float*)(c->ws + c->L.top2);
   { const int rc = compute_xmax2(c); if (rc != ASGD_OK) return rc; }
@@ -257,25 +282,23 @@ int tc_prepare(asgd_ctx* c) {
   p.xnorm = (const float*)(c->ws + c->L.xnorm);
   if (!encode_16bit_map(&c->mapXh, fp16, xh, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
   if (!encode_16bit_map(&c->mapXl, fp16, xl, (unsigned long long)cfg.N, (unsigned long long)cfg.d, TC_M)) return ASGD_ECUDA;
-  if (!encode_16bit_map(&c->mapW, fp16, p.wbf, (fp16 ? 1ull : 2ull) * cfg.W * cfg.k, (unsigned long long)cfg.d, (unsigned)tc_block_n(fp16 ? 1 : 3))) return ASGD_ECUDA;
+  if (!encode_16bit_map(&c->mapW, fp16, p.wbf, (fp16 ? 1ull : 2ull) * cfg.W * cfg.k, (unsigned long long)cfg.d, (unsigned)bn)) return ASGD_ECUDA;
   return ASGD_OK;
 }
 
 int launch_workers(asgd_ctx* c, bool det, long long steps) {
   const Params& p = c->p;
   switch (c->path) {
+#define TC_GO(DET_, T_, D_) asgd_tc_kernel<DET_, T_, D_><<<c->grid, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW)
     case P_TC_BF16:
-      if (det)
-        asgd_tc_kernel<true, 3><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
-      else
-        asgd_tc_kernel<false, 3><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
+      if (c->tc_two) { if (det) TC_GO(true, 3, 128); else TC_GO(false, 3, 128); }
+      else { if (det) TC_GO(true, 3, 256); else TC_GO(false, 3, 256); }
       break;
     case P_TC_FP16:
-      if (det)
-        asgd_tc_kernel<true, 1><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
-      else
-        asgd_tc_kernel<false, 1><<<p.W, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW);
+      if (c->tc_two) { if (det) TC_GO(true, 1, 128); else TC_GO(false, 1, 128); }
+      else { if (det) TC_GO(true, 1, 256); else TC_GO(false, 1, 256); }
       break;
+#undef TC_GO
     case P_TILED: {
       int idx = 0;
 #define X(D_, KP_, WS_, WK_, MB_) if (idx++ == c->tiled_shape) tiled_launch<D_, KP_, WS_, WK_, MB_>(c, det, steps);
@@ -305,7 +328,7 @@ int resolve_path(asgd_ctx* c) {
   const asgd_config& cfg = c->cfg;
   if (cfg.dist_path == ASGD_PATH_TC_BF16 || cfg.dist_path == ASGD_PATH_TC_FP16 ||
       (cfg.dist_path == ASGD_PATH_AUTO && tc_eligible(&cfg) && !c->no_tc)) {
-    if (!tc_eligible(&cfg)) return ASGD_EUNSUPPORTED;
+    if (!tc_supported(&cfg)) return ASGD_EUNSUPPORTED;
     c->path = (cfg.dist_path == ASGD_PATH_TC_BF16) ? P_TC_BF16 : P_TC_FP16;
     c->state_on_chip = 0;
     return ASGD_OK;                       // device-side set-up (tc_prepare) runs once the workspace is cleared

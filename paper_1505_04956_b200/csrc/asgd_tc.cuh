@@ -44,8 +44,13 @@ namespace asgd {
 constexpr int TC_THREADS = 256;
 constexpr int TC_WARPS = TC_THREADS / 32;
 constexpr int TC_M = 128, TC_KC = 64;                    // rows of an MMA's output tile; K chunk = 64 16-bit numbers = one swizzled 128-byte row
-// centres per block (the MMA's N): 256 with one term per operand, 128 with two (the sample tile then takes twice the room)
+// most centres per block (the MMA's N): 256 with one term per operand, 128 with two (the sample tile then takes twice the room)
 __host__ __device__ constexpr int tc_block_n(int terms) { return terms == 1 ? 256 : 128; }
+// centres per block for a state of k centres: a state that fits one block takes whole groups of 32 columns (the
+// accumulators are read 32 columns at a time, and every column read has been written by the MMA)
+__host__ __device__ constexpr int tc_block_rows(int k, int terms) { return k >= tc_block_n(terms) ? tc_block_n(terms) : (k + 31) / 32 * 32; }
+// tensor-memory columns of the two accumulator stages: a power of two, at least 32
+__host__ __device__ constexpr int tc_tmem_cols(int bn) { int c = 32; while (c < 2 * bn) c *= 2; return c; }
 constexpr int TC_A_STAGES = 4;                            // K chunks of the resident sample tile (d <= 256), each with a hi and a lo part
 constexpr int TC_B_STAGES = 4;                            // ring slots for the centre blocks (one K chunk of w_hi or of w_lo each)
 constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB per part
@@ -57,13 +62,19 @@ constexpr float TC_FAR = 1e30f;                          // stands for ||w_a||^2
 
 struct TcSmem {
   size_t B, A, cn, cnt, best, flagged, bars, misc, tail, total;
-  __host__ __device__ TcSmem(int k, int d, int b, int terms) {
-    const int nb = tc_block_n(terms);
+  int cn_stride;               // floats of ||w_a||^2 per worker of the block
+  // nv: workers the block serves in turn (their ||w_a||^2 stay on chip side by side)
+  __host__ __device__ TcSmem(int k, int d, int b, int terms, int nv) {
+    const int nb = tc_block_rows(k, terms);
     size_t off = 0;
     auto take = [&](size_t bytes, size_t align) { off = (off + align - 1) / align * align; size_t o = off; off += bytes; return o; };
-    A = take((size_t)TC_A_STAGES * (terms == 3 ? 2 : 1) * TC_A_STAGE_BYTES, 1024);   // [K chunk][hi, lo]; also the scratch of the grouping phase (<= 40 KB)
-    B = take((size_t)TC_B_STAGES * nb * TC_KC * 2, 1024);
-    cn = take((size_t)((k + nb - 1) / nb) * nb * 4, 16);
+    // [K chunk][hi, lo] of the resident sample tile; also the scratch of the grouping phase ([warps][k] counts, [b] ranks)
+    const size_t tile = (size_t)(d / TC_KC) * (terms == 3 ? 2 : 1) * TC_A_STAGE_BYTES;
+    const size_t scratch = (size_t)TC_WARPS * k * 4 + (size_t)b * 2;
+    A = take(tile > scratch ? tile : scratch, 1024);
+    B = take((size_t)TC_B_STAGES * nb * TC_KC * 2, 1024);                // also [k] group starts and the scans' results (nb >= 32: 16 KB)
+    cn_stride = (k + nb - 1) / nb * nb;
+    cn = take((size_t)nv * cn_stride * 4, 16);
     cnt = take((size_t)k * 4, 16);
     best = take((size_t)b * 2, 16);
     flagged = take((size_t)b * 2 + 16, 16);                          // pairs to settle from the front, rows for the full scan from the back
@@ -73,7 +84,7 @@ struct TcSmem {
     total = off + 1024;          // room to align the base to 1024 bytes
   }
 };
-inline size_t tc_smem_bytes(int k, int d, int b, int terms) { return TcSmem(k, d, b, terms).total; }
+inline size_t tc_smem_bytes(int k, int d, int b, int terms, int nv) { return TcSmem(k, d, b, terms, nv).total; }
 
 __device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -141,9 +152,9 @@ __global__ void tc_row_norms_kernel(const float* __restrict__ X, long long N, in
 
 // Adds the n listed sample rows (fp32 master) into S4, ROWS rows in flight, in list order.  Eight lanes share a
 // row: lane l8 holds dimensions 4*l8 + 32*q, q < nq <= QMAX.
-template <int ROWS, int QMAX>
+template <int ROWS, int QMAX, int SN>
 __device__ inline void tc_add_rows(const float* __restrict__ X, long long row0, int d, int nq, int l8,
-                                   const unsigned short* __restrict__ list, int n, float4 (&S4)[TC_MAX_D / 32]) {
+                                   const unsigned short* __restrict__ list, int n, float4 (&S4)[SN]) {
   for (int e0 = 0; e0 < n; e0 += ROWS) {
     float4 v[ROWS][QMAX];
 #pragma unroll
@@ -184,18 +195,22 @@ __device__ __forceinline__ void tc_top3_insert2(float& m1, float& m2, float& m3,
   m1 = fminf(m1, lo);
 }
 
-template <bool kDet, int kTerms>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+// kMaxD: the largest d the instance holds in registers.  256: one block per SM.  128: half the registers, so that two
+// blocks share an SM when their shared memory allows it; one block's scores then overlap the other's sums and update.
+template <bool kDet, int kTerms, int kMaxD>
+__global__ void __launch_bounds__(TC_THREADS, kMaxD <= 128 ? 2 : 1)
 asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CUtensorMap mapXh,
                const __grid_constant__ CUtensorMap mapXl, const __grid_constant__ CUtensorMap mapW) {
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
   unsigned char* smem = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
   const int k = p.k, d = p.d, b = p.b;
-  const TcSmem map(k, d, b, kTerms);
+  const int G = (int)gridDim.x;
+  const int nv = (p.W - (int)blockIdx.x + G - 1) / G;                   // workers of this block: blockIdx.x + v * G
+  const TcSmem map(k, d, b, kTerms, (p.W + G - 1) / G);
   unsigned char* sB = smem + map.B;
   unsigned char* sA = smem + map.A;
-  float* cn = reinterpret_cast<float*>(smem + map.cn);                 // ||w_a||^2; beyond k a large finite number (with index bits
-                                                                       // packed in, an infinity would read as a NaN and upset the min/max chain)
+  float* cn = reinterpret_cast<float*>(smem + map.cn);                 // ||w_a||^2 of the worker in turn; beyond k a large finite number (with
+                                                                       // index bits packed in, an infinity would read as a NaN and upset the min/max chain)
   int* cnt = reinterpret_cast<int*>(smem + map.cnt);
   unsigned short* best = reinterpret_cast<unsigned short*>(smem + map.best);
   unsigned short* flagged = reinterpret_cast<unsigned short*>(smem + map.flagged);
@@ -205,18 +220,30 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
 
   static_assert(kTerms == 1 || kTerms == 3, "one FP16 term or two BF16 terms per operand");
   constexpr int PPK = (kTerms == 3) ? 2 : 1;                            // parts (hi, lo) per K chunk of an operand
-  constexpr int TC_N = tc_block_n(kTerms);                              // centres per block
-  constexpr int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;                    // a ring slot: one K chunk of a centre block
-  constexpr int TC_TMEM_COLS = 2 * TC_N;                                // two accumulator stages
+  constexpr int QN = kMaxD / 32;                                        // float4 pieces of a row per lane of an eight-lane group
+  constexpr bool kWide = kMaxD > 128;                                   // rows of more than 128 numbers: a second float4 per lane in the scans
+  const int TC_N = tc_block_rows(k, kTerms);                            // centres per block
+  const int TC_B_CHUNK_BYTES = TC_N * TC_KC * 2;                        // a ring slot: one K chunk of a centre block
+  const int TC_TMEM_COLS = tc_tmem_cols(TC_N);                          // two accumulator stages
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-  const int i = blockIdx.x;
   const int nkc = d / TC_KC;                                           // K chunks per tile
   const int n_tiles = (k + TC_N - 1) / TC_N, m_tiles = (b + TC_M - 1) / TC_M;
-  float* wglob = p.state + (size_t)i * p.kd_pad;
-  float* gsum = p.gsum + (size_t)i * p.kd_pad;
-  unsigned short* wbf = reinterpret_cast<unsigned short*>(p.wbf) + (size_t)i * k * d;        // 16-bit -2w (w_hi) of this worker
-  unsigned short* wbl = wbf + (size_t)p.W * k * d;                                           // w_lo: second half of the array (two-term format)
-  float4* top3 = reinterpret_cast<float4*>(p.top2) + (size_t)i * b;        // per row: three smallest packed squared distances
+  // the worker in turn
+  int i = blockIdx.x;
+  float* wglob = nullptr;
+  float* gsum = nullptr;
+  unsigned short* wbf = nullptr;                                        // 16-bit -2w (w_hi) of the worker
+  unsigned short* wbl = nullptr;                                        // w_lo: second half of the array (two-term format)
+  float4* top3 = nullptr;                                               // per row: three smallest packed squared distances and the floor under the fourth
+  auto take_worker = [&](int v) {
+    i = (int)blockIdx.x + v * G;
+    wglob = p.state + (size_t)i * p.kd_pad;
+    gsum = p.gsum + (size_t)i * p.kd_pad;
+    wbf = reinterpret_cast<unsigned short*>(p.wbf) + (size_t)i * k * d;
+    wbl = wbf + (size_t)p.W * k * d;
+    top3 = reinterpret_cast<float4*>(p.top2) + (size_t)i * b;
+    cn = reinterpret_cast<float*>(smem + map.cn) + (size_t)v * map.cn_stride;
+  };
   const float INF = __int_as_float(0x7f800000);
   const float inv_b = 1.0f / (float)b;
 
@@ -228,16 +255,16 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     misc[2] = 0;
   }
   if (wid == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(misc)), "n"(TC_TMEM_COLS) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(misc)), "r"((unsigned)TC_TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // -2w as two BF16 terms and ||w_a||^2 of one centre held by eight lanes (lane l8: dimensions 4*l8 + 32*q)
   const int sub = lane >> 3, l8 = lane & 7;
   const int nq = d / 32;
-  auto refresh = [&](int a, const float4 (&w4)[TC_MAX_D / 32]) {
+  auto refresh = [&](int a, const float4 (&w4)[QN]) {
     float sq = 0.f;
 #pragma unroll
-    for (int q = 0; q < TC_MAX_D / 32; ++q) {
+    for (int q = 0; q < QN; ++q) {
       if (q < nq) {
         sq = fmaf(w4[q].x, w4[q].x, sq); sq = fmaf(w4[q].y, w4[q].y, sq); sq = fmaf(w4[q].z, w4[q].z, sq); sq = fmaf(w4[q].w, w4[q].w, sq);
         const size_t o = (size_t)a * d + 4 * l8 + 32 * q;
@@ -262,9 +289,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       const int a = a0 + sub;
       float sq = 0.f;
       if (a < k) {
-        float4 w4[TC_MAX_D / 32];
+        float4 w4[QN];
 #pragma unroll
-        for (int q = 0; q < TC_MAX_D / 32; ++q)
+        for (int q = 0; q < QN; ++q)
           if (q < nq) w4[q] = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q);
         sq = refresh(a, w4);
       }
@@ -273,8 +300,8 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       if (l8 == 0) cn[a] = (a < k) ? sq : TC_FAR;
     }
   };
-  refresh_all();
-  asm volatile("fence.proxy.async;" ::: "memory");                      // the BF16 terms written above are read by TMA
+  for (int v = 0; v < nv; ++v) { take_worker(v); refresh_all(); }
+  asm volatile("fence.proxy.async;" ::: "memory");                      // the 16-bit terms written above are read by TMA
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -283,11 +310,14 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   const unsigned fmt = (kTerms == 3) ? 1u : 0u;
   const unsigned idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((unsigned)(TC_N >> 3) << 17) | ((unsigned)(TC_M >> 4) << 24);
 
-  unsigned long long t = p.stats[(size_t)i * ST_STRIDE + ST_STEPS];
   // running phase counters of the pipelines (each role keeps its own copies in step)
   unsigned it_m = 0, it_bc = 0, it_acc = 0;
 
-  for (long long step = 0; step < steps; ++step, ++t) {
+  bool gave_up = false;
+  for (long long step = 0; step < steps && !gave_up; ++step)
+  for (int v = 0; v < nv; ++v) {                          // the block's workers take the step one after the other
+    take_worker(v);
+    const unsigned long long t = *reinterpret_cast<volatile unsigned long long*>(p.stats + (size_t)i * ST_STRIDE + ST_STEPS);   // written by this block at the end of the worker's last step
     const long long batch = p.perm[(size_t)i * p.B + (size_t)(t % (unsigned long long)p.B)];
     const long long row0 = (long long)i * p.H + batch * b;
 
@@ -443,7 +473,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (misc[2]) break;                                   // a wait ran out: report and leave (uniform)
+    if (misc[2]) { gave_up = true; break; }               // a wait ran out: report and leave (uniform)
 
     // ================= decide =================
     float wmax2 = 0.f;
@@ -507,9 +537,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         const float* w1 = wglob + (size_t)i1 * d + 4 * l8;
         const float* w2 = wglob + (size_t)i2 * d + 4 * l8;
         const float* w3 = wglob + (size_t)i3 * d + 4 * l8;
-        float4 xv[TC_MAX_D / 32], c1[TC_MAX_D / 32], c2[TC_MAX_D / 32], c3[TC_MAX_D / 32];
+        float4 xv[QN], c1[QN], c2[QN], c3[QN];
 #pragma unroll
-        for (int q = 0; q < TC_MAX_D / 32; ++q) {
+        for (int q = 0; q < QN; ++q) {
           if (q < nq && r >= 0) {
             xv[q] = __ldg(reinterpret_cast<const float4*>(x + 32 * q));
             c1[q] = *reinterpret_cast<const float4*>(w1 + 32 * q);
@@ -523,7 +553,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         // above (4 d + 16) u of the larger one decides; only rows closer than that are summed again in fp64
         float f1 = 0.f, f2 = 0.f, f3 = 0.f;
 #pragma unroll
-        for (int q = 0; q < TC_MAX_D / 32; ++q) {
+        for (int q = 0; q < QN; ++q) {
           float u;
           u = xv[q].x - c1[q].x; f1 = fmaf(u, u, f1); u = xv[q].y - c1[q].y; f1 = fmaf(u, u, f1);
           u = xv[q].z - c1[q].z; f1 = fmaf(u, u, f1); u = xv[q].w - c1[q].w; f1 = fmaf(u, u, f1);
@@ -544,7 +574,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         if (__any_sync(0xffffffffu, close && r >= 0)) {       // warp-uniform: the shuffles below need every lane
           double d1 = 0.0, d2 = 0.0, d3 = 0.0;
 #pragma unroll
-          for (int q = 0; q < TC_MAX_D / 32; ++q) {
+          for (int q = 0; q < QN; ++q) {
             double u;
             u = (double)xv[q].x - (double)c1[q].x; d1 = fma(u, u, d1); u = (double)xv[q].y - (double)c1[q].y; d1 = fma(u, u, d1);
             u = (double)xv[q].z - (double)c1[q].z; d1 = fma(u, u, d1); u = (double)xv[q].w - (double)c1[q].w; d1 = fma(u, u, d1);
@@ -578,7 +608,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       __syncthreads();                                         // the pairs' readers of `order` and `top3` are done; the ring is idle
       const int nwide = misc[5];
       const int d4 = d / 4;
-      const bool on0 = lane < d4, on1 = 32 + lane < d4;
+      const bool on0 = lane < d4, on1 = kWide && 32 + lane < d4;
       const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
       // one batch of R <= RB rows (RB = 16, or 4 for the usual handful: a quarter of the arithmetic per centre)
       auto scan_batch = [&](auto rb_tag, const int base, const int R) {
@@ -607,8 +637,10 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             float s0 = 0.f, s1 = 0.f, e;
             e = x0.x - w0v.x; s0 = fmaf(e, e, s0); e = x0.y - w0v.y; s1 = fmaf(e, e, s1);
             e = x0.z - w0v.z; s0 = fmaf(e, e, s0); e = x0.w - w0v.w; s1 = fmaf(e, e, s1);
-            e = x1.x - w1v.x; s0 = fmaf(e, e, s0); e = x1.y - w1v.y; s1 = fmaf(e, e, s1);
-            e = x1.z - w1v.z; s0 = fmaf(e, e, s0); e = x1.w - w1v.w; s1 = fmaf(e, e, s1);
+            if (kWide) {
+              e = x1.x - w1v.x; s0 = fmaf(e, e, s0); e = x1.y - w1v.y; s1 = fmaf(e, e, s1);
+              e = x1.z - w1v.z; s0 = fmaf(e, e, s0); e = x1.w - w1v.w; s1 = fmaf(e, e, s1);
+            }
             part[j] = s0 + s1;
           }
           // halving exchange: at offset o the lanes with that bit clear keep the lower half of the rows still held
@@ -676,8 +708,10 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             double sacc = 0.0, e;
             e = (double)x0.x - (double)u0.x; sacc = fma(e, e, sacc); e = (double)x0.y - (double)u0.y; sacc = fma(e, e, sacc);
             e = (double)x0.z - (double)u0.z; sacc = fma(e, e, sacc); e = (double)x0.w - (double)u0.w; sacc = fma(e, e, sacc);
-            e = (double)x1.x - (double)u1.x; sacc = fma(e, e, sacc); e = (double)x1.y - (double)u1.y; sacc = fma(e, e, sacc);
-            e = (double)x1.z - (double)u1.z; sacc = fma(e, e, sacc); e = (double)x1.w - (double)u1.w; sacc = fma(e, e, sacc);
+            if (kWide) {
+              e = (double)x1.x - (double)u1.x; sacc = fma(e, e, sacc); e = (double)x1.y - (double)u1.y; sacc = fma(e, e, sacc);
+              e = (double)x1.z - (double)u1.z; sacc = fma(e, e, sacc); e = (double)x1.w - (double)u1.w; sacc = fma(e, e, sacc);
+            }
 #pragma unroll
             for (int sh = 16; sh > 0; sh >>= 1) sacc += __shfl_xor_sync(0xffffffffu, sacc, sh);
             return sacc;
@@ -778,23 +812,23 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         const int a = a0 + sub;
         const bool on = a < k;
         const int n = on ? cnt[a] : 0, p0 = on ? start[a] : 0;
-        float4 S4[TC_MAX_D / 32];
+        float4 S4[QN];
 #pragma unroll
-        for (int q = 0; q < TC_MAX_D / 32; ++q) S4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (nq <= TC_MAX_D / 64) tc_add_rows<2 * TC_SUM_ROWS, TC_MAX_D / 64>(p.X, row0, d, nq, l8, order + p0, n, S4);
-        else tc_add_rows<TC_SUM_ROWS, TC_MAX_D / 32>(p.X, row0, d, nq, l8, order + p0, n, S4);
+        for (int q = 0; q < QN; ++q) S4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (nq <= QN / 2) tc_add_rows<2 * TC_SUM_ROWS, QN / 2>(p.X, row0, d, nq, l8, order + p0, n, S4);
+        else tc_add_rows<TC_SUM_ROWS, QN>(p.X, row0, d, nq, l8, order + p0, n, S4);
         float sq = 0.f;
         if (on) {
           if (plain) {
-            float4 w4[TC_MAX_D / 32];
+            float4 w4[QN];
             const float fn = (float)n;
             // all of the centre's row first, then the stores: a store between two loads from the same array would keep
             // the second load behind it (they might alias), one L2 round trip per piece instead of one per row
 #pragma unroll
-            for (int q = 0; q < TC_MAX_D / 32; ++q)
+            for (int q = 0; q < QN; ++q)
               if (q < nq) w4[q] = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q);
 #pragma unroll
-            for (int q = 0; q < TC_MAX_D / 32; ++q) {
+            for (int q = 0; q < QN; ++q) {
               if (q < nq) {
                 float4 u = w4[q];
                 u.x -= p.eps * ((fn * u.x - S4[q].x) * inv_b); u.y -= p.eps * ((fn * u.y - S4[q].y) * inv_b);
@@ -806,7 +840,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             sq = refresh(a, w4);
           } else {
 #pragma unroll
-            for (int q = 0; q < TC_MAX_D / 32; ++q)
+            for (int q = 0; q < QN; ++q)
               if (q < nq) *reinterpret_cast<float4*>(gsum + (size_t)a * d + 4 * l8 + 32 * q) = S4[q];
           }
         }
@@ -850,7 +884,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   }
   tc_fence_before();
   __syncthreads();
-  if (wid == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TC_TMEM_COLS) : "memory");
+  if (wid == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((unsigned)TC_TMEM_COLS) : "memory");
 }
 
 }  // namespace asgd

@@ -18,6 +18,8 @@
 // shared memory.  The order of every sum is fixed by row position.
 #pragma once
 
+#include <type_traits>
+
 #include "asgd_step_tail.cuh"
 #include "asgd_stream.cuh"   // bulk-copy and mbarrier helpers
 
@@ -201,23 +203,33 @@ asgd_tiled_kernel(const Params p, const long long steps) {
             for (int c = 0; c < 4; ++c) acc[m][c] = 0.f;
           const float* xrow = xb + (size_t)(rb * 4 + sg) * QS + (size_t)(wsi * 4) * XS;    // rows rb*TS0 + sg*QR + wsi*4 + m
           const float* wrow = wR + (size_t)(wk * 32 + cg) * WST;
+          // the warp's 32 centres come in four groups of eight (centres 8c + cg); a group that lies wholly past k is
+          // padding and is left out (k = 100 in 128 columns: three of the last warp's four groups)
+          auto score_groups = [&](auto ng_tag) {
+            constexpr int NG = decltype(ng_tag)::value;
   #pragma unroll 2
-          for (int j = 0; j < D; j += 4) {
-            float4 xv[4], wv[4];
+            for (int j = 0; j < D; j += 4) {
+              float4 xv[4], wv[NG];
   #pragma unroll
-            for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xrow + (size_t)m * XS + j);
+              for (int m = 0; m < 4; ++m) xv[m] = *reinterpret_cast<const float4*>(xrow + (size_t)m * XS + j);
   #pragma unroll
-            for (int c = 0; c < 4; ++c) wv[c] = *reinterpret_cast<const float4*>(wrow + (size_t)(8 * c) * WST + j);
+              for (int c = 0; c < NG; ++c) wv[c] = *reinterpret_cast<const float4*>(wrow + (size_t)(8 * c) * WST + j);
   #pragma unroll
-            for (int m = 0; m < 4; ++m)
+              for (int m = 0; m < 4; ++m)
   #pragma unroll
-              for (int c = 0; c < 4; ++c) {
-                acc[m][c] = fmaf(xv[m].x, wv[c].x, acc[m][c]);
-                acc[m][c] = fmaf(xv[m].y, wv[c].y, acc[m][c]);
-                acc[m][c] = fmaf(xv[m].z, wv[c].z, acc[m][c]);
-                acc[m][c] = fmaf(xv[m].w, wv[c].w, acc[m][c]);
-              }
-          }
+                for (int c = 0; c < NG; ++c) {
+                  acc[m][c] = fmaf(xv[m].x, wv[c].x, acc[m][c]);
+                  acc[m][c] = fmaf(xv[m].y, wv[c].y, acc[m][c]);
+                  acc[m][c] = fmaf(xv[m].z, wv[c].z, acc[m][c]);
+                  acc[m][c] = fmaf(xv[m].w, wv[c].w, acc[m][c]);
+                }
+            }
+          };
+          const int ngroups = min(4, max(0, (k - wk * 32 + 7) / 8));          // the same for every lane of the warp
+          if (ngroups == 4) score_groups(std::integral_constant<int, 4>());
+          else if (ngroups == 3) score_groups(std::integral_constant<int, 3>());
+          else if (ngroups == 2) score_groups(std::integral_constant<int, 2>());
+          else if (ngroups == 1) score_groups(std::integral_constant<int, 1>());
           // minimum and runner-up over the lane's 4 centres, then over the 8 lanes that share the rows
           float cnv[4];
   #pragma unroll

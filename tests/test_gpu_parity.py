@@ -205,11 +205,16 @@ EDGE_CASES = {
     "tiled_32_k37_ragged_tile": dict(N=5 * 100 * 3 + 1, d=32, k=37, W=5, b=100, comm_interval=2, fanout=2),
     "tiled_32_many_workers": dict(N=700 * 12, d=32, k=8, W=700, b=4, comm_interval=1, fanout=1),
     "tiled_32_small_blocks_one_worker_each": dict(N=592 * 70 * 2, d=32, k=64, W=592, b=70, comm_interval=2, fanout=1),
-    "tiled_128_k128": dict(N=3 * 200 * 2, d=128, k=128, W=3, b=200, comm_interval=1, fanout=1),
+    "tiled_128_k128": dict(N=3 * 200 * 2, d=128, k=128, W=3, b=200, comm_interval=1, fanout=1, path=pkg.PATH_FP32),
     "tiled_128_k5_tiny_batch": dict(N=4 * 7 * 3, d=128, k=5, W=4, b=7, comm_interval=1, fanout=3),
     # shapes of the tensor-core kernel: a centre block that is not full, one K chunk, a ragged last sample tile
     "tc_d64_k300_ragged": dict(N=3 * 200 * 3 + 5, d=64, k=300, W=3, b=200, comm_interval=2, fanout=1),
     "tc_d128_k129": dict(N=2 * 128 * 4, d=128, k=129, W=2, b=128, comm_interval=1, fanout=1),
+    # ... a state of one centre block (narrower MMA), two blocks per SM, a block's workers taking turns
+    "tc_d128_k128_one_block": dict(N=3 * 200 * 2, d=128, k=128, W=3, b=200, comm_interval=1, fanout=1),
+    "tc_d64_k17_one_block": dict(N=4 * 150 * 3 + 2, d=64, k=17, W=4, b=150, comm_interval=2, fanout=2),
+    "tc_d128_k100_two_blocks_per_sm_workers_in_turn": dict(N=310 * 128 * 2, d=128, k=100, W=310, b=128, comm_interval=1, fanout=2),
+    "tc_d256_k40_workers_in_turn": dict(N=320 * 128 * 2 + 9, d=256, k=40, W=320, b=128, comm_interval=2, fanout=1),
     "general_10x10_big_batch": dict(N=2 * 700 * 3, d=10, k=10, W=2, b=700, comm_interval=2, fanout=1),
 }
 
@@ -218,9 +223,12 @@ EDGE_CASES = {
 @pytest.mark.parametrize("parzen", [1, 0])
 def test_edge_cases(case, parzen):
     kw = dict(EDGE_CASES[case])
+    path = kw.pop("path", pkg.PATH_AUTO)
     wl = scaled("tiny", eps=0.1, **kw)
     slots = 3 if case in ("fanout_all_peers", "ragged_rows") else None
-    pr = Pair(wl, parzen=parzen, slots=slots)
+    pr = Pair(wl, parzen=parzen, slots=slots, dist_path=path)
+    if case.startswith(("tiled_", "tc_", "stream_")):
+        assert pr.gpu.path_name().startswith({"tiled_": "fp32-tiled", "tc_": "tcgen05", "stream_": "fp32-stream"}[case[:case.index("_") + 1]])
     rounds = 2 * wl.B + 3
     pr.rounds(rounds)
     pr.gpu.sync()

@@ -24,7 +24,8 @@ CASES = {
     "stream_10x10": (dict(N=6 * 100 * 5, d=10, k=10, W=6, b=100, comm_interval=1, fanout=2), 4, 12),
     "stream_16x16_all_rows": (dict(N=4 * 175 * 4, d=16, k=16, W=4, b=175, comm_interval=2, fanout=1), 16, 8),
     "tiled_32x37": (dict(N=5 * 100 * 4 + 1, d=32, k=37, W=5, b=100, comm_interval=1, fanout=2), 5, 8),
-    "tiled_128x100": (dict(N=3 * 200 * 3, d=128, k=100, W=3, b=200, comm_interval=1, fanout=1), 33, 6),
+    "tiled_128x100": (dict(N=3 * 100 * 3, d=128, k=100, W=3, b=100, comm_interval=1, fanout=1), 33, 6),
+    "tc_d128_k100_one_block": (dict(N=3 * 200 * 3, d=128, k=100, W=3, b=200, comm_interval=1, fanout=1), 33, 6),
     "tc_d64_k300": (dict(N=3 * 200 * 4 + 5, d=64, k=300, W=3, b=200, comm_interval=1, fanout=2), 70, 6),
 }
 
