@@ -276,8 +276,14 @@ def measure(args, wl, dev, rank, world, dist, keep=False):
             with open(ppath) as f:
                 tpeak, tkind = float(json.load(f)["bf16_tflops_sustained"]), "measured (sustained)"
         ach = flops / (launch_ms * 1e-3) / 1e12
-        roofline = dict(common, bound="tensor", achieved=ach, peak=tpeak, unit="TFLOP/s", frac=ach / tpeak,
-                        peak_kind="of " + tkind, algorithmic_flops_per_launch=flops, hbm_GBs=hbm_gbs)
+        if flops / (tpeak * 1e12) >= bytes_per_launch / (hbm_peak * 1e9):
+            roofline = dict(common, bound="tensor", achieved=ach, peak=tpeak, unit="TFLOP/s", frac=ach / tpeak,
+                            peak_kind="of " + tkind, algorithmic_flops_per_launch=flops, hbm_GBs=hbm_gbs)
+        else:
+            # few centres: reading the samples takes longer than the contraction, the launch is bound by HBM
+            roofline = dict(common, bound="hbm", achieved=hbm_gbs, peak=hbm_peak, unit="GB/s", frac=hbm_gbs / hbm_peak,
+                            peak_kind="of " + peak_kind, frac_of_nominal_8TBs=hbm_gbs / NOMINAL_HBM_GBS,
+                            algorithmic_flops_per_launch=flops, tensor_TFLOPs=ach)
         dtype = "f16" if kernel.endswith("fp16") else "bf16"
     else:
         roofline = dict(common, bound="hbm", achieved=hbm_gbs, peak=hbm_peak, unit="GB/s", frac=hbm_gbs / hbm_peak,

@@ -610,12 +610,14 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       const int d4 = d / 4;
       const bool on0 = lane < d4, on1 = kWide && 32 + lane < d4;
       const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
-      // one batch of R <= RB rows (RB = 16, or 4 for the usual handful: a quarter of the arithmetic per centre)
-      auto scan_batch = [&](auto rb_tag, const int base, const int R) {
-        constexpr int RB = decltype(rb_tag)::value;
-        constexpr int LPR = 32 / RB;                           // lanes that end up with the same row: LPR * j .. LPR * j + LPR - 1
-        float* res = reinterpret_cast<float*>(sB);             // [TC_WARPS][RB][5] per warp and row: the three smallest, indices of the first two
-        int* need64 = reinterpret_cast<int*>(res + TC_WARPS * RB * 5);    // [RB][3]: 0 decided, 1 compare two in fp64, 2 scan all in fp64; the two indices
+      // one batch of R <= RB rows against CB centres per warp at a time: RB x CB = 16 (row, centre) pairs either way
+      // (16 rows x 1 centre, or for the usual handful 4 rows x 4 centres, whose four rows of the state are on their way together)
+      auto scan_batch = [&](auto rb_tag, auto cb_tag, const int base, const int R) {
+        constexpr int RB = decltype(rb_tag)::value, CB = decltype(cb_tag)::value;
+        constexpr int VR = RB * CB;                            // (centre slot c, row j) pairs, pair c * RB + j
+        constexpr int LPR = 32 / VR;                           // lanes that end up with the same pair: LPR * v .. LPR * v + LPR - 1
+        float* res = reinterpret_cast<float*>(sB);             // [TC_WARPS][VR][5] per warp and pair: the three smallest, indices of the first two
+        int* need64 = reinterpret_cast<int*>(res + TC_WARPS * VR * 5);    // [RB][3]: 0 decided, 1 compare two in fp64, 2 scan all in fp64; the two indices
         float4 xr0[RB], xr1[RB];                               // this lane's dimensions of the rows (zeros past the last row)
 #pragma unroll
         for (int j = 0; j < RB; ++j) {
@@ -623,29 +625,43 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           xr0[j] = (j < R && on0) ? __ldg(xrow + lane) : z4;
           xr1[j] = (j < R && on1) ? __ldg(xrow + 32 + lane) : z4;
         }
-        float bd1 = INF, bd2 = INF, bd3 = INF;                 // first lane of row j's run: row j over this warp's centres
+        float bd1 = INF, bd2 = INF, bd3 = INF;                 // first lane of a pair's run: row j over the centres of slot c of this warp
         int bi1 = 0x7fffffff, bi2 = 0x7fffffff;
-        const float4* wa = reinterpret_cast<const float4*>(wglob + (size_t)wid * d);
-        float4 w0v = (wid < k && on0) ? wa[lane] : z4, w1v = (wid < k && on1) ? wa[32 + lane] : z4;
-        for (int a = wid; a < k; a += TC_WARPS) {              // ascending inside a warp: a strict "<" keeps the lowest index of a tie
-          const float4* wn = reinterpret_cast<const float4*>(wglob + (size_t)min(a + TC_WARPS, k - 1) * d);
-          const float4 n0 = on0 ? wn[lane] : z4, n1 = on1 ? wn[32 + lane] : z4;      // the next centre's row
-          float part[RB];
+        const int c_mine = (lane / LPR) / RB;                  // the centre slot of the pair this lane ends up with
+        // the warp's centres are wid, wid + 8, ...; an iteration takes CB of them, slot c the centre a + 8 c
+        float4 w0v[CB], w1v[CB];
 #pragma unroll
-          for (int j = 0; j < RB; ++j) {
-            const float4 x0 = xr0[j], x1 = xr1[j];
-            float s0 = 0.f, s1 = 0.f, e;
-            e = x0.x - w0v.x; s0 = fmaf(e, e, s0); e = x0.y - w0v.y; s1 = fmaf(e, e, s1);
-            e = x0.z - w0v.z; s0 = fmaf(e, e, s0); e = x0.w - w0v.w; s1 = fmaf(e, e, s1);
-            if (kWide) {
-              e = x1.x - w1v.x; s0 = fmaf(e, e, s0); e = x1.y - w1v.y; s1 = fmaf(e, e, s1);
-              e = x1.z - w1v.z; s0 = fmaf(e, e, s0); e = x1.w - w1v.w; s1 = fmaf(e, e, s1);
-            }
-            part[j] = s0 + s1;
+        for (int c = 0; c < CB; ++c) {
+          const float4* wa = reinterpret_cast<const float4*>(wglob + (size_t)min(wid + TC_WARPS * c, k - 1) * d);
+          w0v[c] = on0 ? wa[lane] : z4;
+          w1v[c] = on1 ? wa[32 + lane] : z4;
+        }
+        for (int a = wid; a < k; a += TC_WARPS * CB) {         // ascending inside a slot: a strict "<" keeps the lowest index of a tie
+          float4 n0[CB], n1[CB];                               // the next iteration's rows of the state
+#pragma unroll
+          for (int c = 0; c < CB; ++c) {
+            const float4* wn = reinterpret_cast<const float4*>(wglob + (size_t)min(a + TC_WARPS * (CB + c), k - 1) * d);
+            n0[c] = on0 ? wn[lane] : z4;
+            n1[c] = on1 ? wn[32 + lane] : z4;
           }
-          // halving exchange: at offset o the lanes with that bit clear keep the lower half of the rows still held
+          float part[VR];
 #pragma unroll
-          for (int o = 16, n = RB / 2; n >= 1; o >>= 1, n >>= 1) {
+          for (int c = 0; c < CB; ++c)
+#pragma unroll
+            for (int j = 0; j < RB; ++j) {
+              const float4 x0 = xr0[j], x1 = xr1[j];
+              float s0 = 0.f, s1 = 0.f, e;
+              e = x0.x - w0v[c].x; s0 = fmaf(e, e, s0); e = x0.y - w0v[c].y; s1 = fmaf(e, e, s1);
+              e = x0.z - w0v[c].z; s0 = fmaf(e, e, s0); e = x0.w - w0v[c].w; s1 = fmaf(e, e, s1);
+              if (kWide) {
+                e = x1.x - w1v[c].x; s0 = fmaf(e, e, s0); e = x1.y - w1v[c].y; s1 = fmaf(e, e, s1);
+                e = x1.z - w1v[c].z; s0 = fmaf(e, e, s0); e = x1.w - w1v[c].w; s1 = fmaf(e, e, s1);
+              }
+              part[c * RB + j] = s0 + s1;
+            }
+          // halving exchange: at offset o the lanes with that bit clear keep the lower half of the pairs still held
+#pragma unroll
+          for (int o = 16, n = VR / 2; n >= 1; o >>= 1, n >>= 1) {
             const bool up = (lane & o) != 0;
 #pragma unroll
             for (int j = 0; j < n; ++j) {
@@ -654,19 +670,21 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
               part[j] = keep + __shfl_xor_sync(0xffffffffu, send, o);
             }
           }
-          float tot = part[0];                                  // lanes LPR * j .. : row j, each with a share of it
+          float tot = part[0];                                  // lanes LPR * v .. : pair v, each with a share of it
 #pragma unroll
           for (int o = LPR / 2; o >= 1; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
-          if ((lane & (LPR - 1)) == 0) {
-            if (tot < bd1) { bd3 = bd2; bd2 = bd1; bi2 = bi1; bd1 = tot; bi1 = a; }
-            else if (tot < bd2) { bd3 = bd2; bd2 = tot; bi2 = a; }
+          const int a_mine = a + TC_WARPS * c_mine;
+          if ((lane & (LPR - 1)) == 0 && a_mine < k) {
+            if (tot < bd1) { bd3 = bd2; bd2 = bd1; bi2 = bi1; bd1 = tot; bi1 = a_mine; }
+            else if (tot < bd2) { bd3 = bd2; bd2 = tot; bi2 = a_mine; }
             else if (tot < bd3) { bd3 = tot; }
           }
-          w0v = n0; w1v = n1;
+#pragma unroll
+          for (int c = 0; c < CB; ++c) { w0v[c] = n0[c]; w1v[c] = n1[c]; }
         }
         if ((lane & (LPR - 1)) == 0) {
-          const int j = lane / LPR;
-          float* o = res + (wid * RB + j) * 5;
+          const int v = lane / LPR;
+          float* o = res + (wid * VR + v) * 5;
           o[0] = bd1; o[1] = bd2; o[2] = bd3; o[3] = __int_as_float(bi1); o[4] = __int_as_float(bi2);
         }
         __syncthreads();
@@ -679,7 +697,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             else if (v < fd2 || (v == fd2 && idx < fi2)) { fd3 = fd2; fd2 = v; fi2 = idx; }
             else if (v < fd3) { fd3 = v; }
           };
-          for (int q = 0; q < TC_WARPS; ++q) {
+          for (int q = 0; q < TC_WARPS * CB; ++q) {             // every warp's every centre slot
             const float* o = res + (q * RB + tid) * 5;
             put(o[0], __float_as_int(o[3]));
             put(o[1], __float_as_int(o[4]));
@@ -734,8 +752,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         __syncthreads();                                       // before the next batch overwrites the results
       };
       int base = 0;                                            // block-uniform trip counts
-      for (; nwide - base > 4; base += TC_SCAN_ROWS) scan_batch(std::integral_constant<int, TC_SCAN_ROWS>(), base, min(TC_SCAN_ROWS, nwide - base));
-      if (base < nwide) scan_batch(std::integral_constant<int, 4>(), base, nwide - base);
+      for (; nwide - base > 4; base += TC_SCAN_ROWS)
+        scan_batch(std::integral_constant<int, TC_SCAN_ROWS>(), std::integral_constant<int, 1>(), base, min(TC_SCAN_ROWS, nwide - base));
+      if (base < nwide) scan_batch(std::integral_constant<int, 4>(), std::integral_constant<int, 4>(), base, nwide - base);
     }
     __syncthreads();
     if (p.assign_rec)
