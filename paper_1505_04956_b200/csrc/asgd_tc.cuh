@@ -54,7 +54,6 @@ __host__ __device__ constexpr int tc_tmem_cols(int bn) { int c = 32; while (c < 
 constexpr int TC_A_STAGES = 4;                            // K chunks of the resident sample tile (d <= 256), each with a hi and a lo part
 constexpr int TC_B_STAGES = 4;                            // ring slots for the centre blocks (one K chunk of w_hi or of w_lo each)
 constexpr int TC_A_STAGE_BYTES = TC_M * TC_KC * 2;       // 16 KB per part
-constexpr int TC_SUM_ROWS = 4;                            // sample rows a centre's adders keep in flight
 constexpr int TC_MAX_K = 1024, TC_MAX_D = 256, TC_MAX_B = 4096;
 constexpr unsigned TC_INDEX_MASK = 1023u;
 constexpr int TC_SCAN_ROWS = 16;                          // rows the full scan measures at a time
@@ -150,28 +149,6 @@ __global__ void tc_row_norms_kernel(const float* __restrict__ X, long long N, in
   }
 }
 
-// Adds the n listed sample rows (fp32 master) into S4, ROWS rows in flight, in list order.  Eight lanes share a
-// row: lane l8 holds dimensions 4*l8 + 32*q, q < nq <= QMAX.
-template <int ROWS, int QMAX, int SN>
-__device__ inline void tc_add_rows(const float* __restrict__ X, long long row0, int d, int nq, int l8,
-                                   const unsigned short* __restrict__ list, int n, float4 (&S4)[SN]) {
-  for (int e0 = 0; e0 < n; e0 += ROWS) {
-    float4 v[ROWS][QMAX];
-#pragma unroll
-    for (int u = 0; u < ROWS; ++u) {
-      const bool have = e0 + u < n;
-      const float* x = X + (size_t)(row0 + (have ? (int)list[e0 + u] : 0)) * d + 4 * l8;
-#pragma unroll
-      for (int q = 0; q < QMAX; ++q)
-        v[u][q] = (q < nq && have) ? __ldg(reinterpret_cast<const float4*>(x + 32 * q)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int u = 0; u < ROWS; ++u)
-#pragma unroll
-      for (int q = 0; q < QMAX; ++q) { S4[q].x += v[u][q].x; S4[q].y += v[u][q].y; S4[q].z += v[u][q].z; S4[q].w += v[u][q].w; }
-  }
-}
-
 // barrier slots
 enum { TCB_BFULL = 0, TCB_BEMPTY = TC_B_STAGES, TCB_AFULL = 2 * TC_B_STAGES, TCB_AEMPTY = 2 * TC_B_STAGES + TC_A_STAGES,
        TCB_ACCFULL = 2 * TC_B_STAGES + 2 * TC_A_STAGES, TCB_ACCEMPTY = TCB_ACCFULL + 2, TCB_COUNT = TCB_ACCFULL + 4 };
@@ -215,7 +192,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   unsigned short* best = reinterpret_cast<unsigned short*>(smem + map.best);
   unsigned short* flagged = reinterpret_cast<unsigned short*>(smem + map.flagged);
   unsigned long long* bars = reinterpret_cast<unsigned long long*>(smem + map.bars);
-  int* misc = reinterpret_cast<int*>(smem + map.misc);                 // [0] tmem base, [1] pairs to settle, [2] abort, [4] news, [5] rows for the full scan, [6] rows with three candidates
+  int* misc = reinterpret_cast<int*>(smem + map.misc);                 // [0] tmem base, [1] pairs to settle, [2] abort, [4] news, [5] rows for the full scan, [6] rows with three candidates, [7] next centre of the sum phase
   TailScratch* ts = reinterpret_cast<TailScratch*>(smem + map.tail);
 
   static_assert(kTerms == 1 || kTerms == 3, "one FP16 term or two BF16 terms per operand");
@@ -261,27 +238,29 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   // -2w as two BF16 terms and ||w_a||^2 of one centre held by eight lanes (lane l8: dimensions 4*l8 + 32*q)
   const int sub = lane >> 3, l8 = lane & 7;
   const int nq = d / 32;
+  // 16-bit terms of -2w for four numbers of the state at element offset o (a multiple of 4): one 8-byte store per
+  // term; returns the four numbers' sum of squares
+  auto put16 = [&](size_t o, const float4& w) {
+    const float v[4] = {-2.f * w.x, -2.f * w.y, -2.f * w.z, -2.f * w.w};     // exact
+    if (kTerms == 1) {
+      const __half2 h01 = __floats2half2_rn(v[0], v[1]), h23 = __floats2half2_rn(v[2], v[3]);
+      *reinterpret_cast<uint2*>(wbf + o) = make_uint2(*reinterpret_cast<const unsigned*>(&h01), *reinterpret_cast<const unsigned*>(&h23));
+    } else {
+      const __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
+      const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+      const __nv_bfloat162 l01 = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y), l23 = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
+      *reinterpret_cast<uint2*>(wbf + o) = make_uint2(*reinterpret_cast<const unsigned*>(&h01), *reinterpret_cast<const unsigned*>(&h23));
+      *reinterpret_cast<uint2*>(wbl + o) = make_uint2(*reinterpret_cast<const unsigned*>(&l01), *reinterpret_cast<const unsigned*>(&l23));
+    }
+    float sq = w.x * w.x;
+    sq = fmaf(w.y, w.y, sq); sq = fmaf(w.z, w.z, sq); sq = fmaf(w.w, w.w, sq);
+    return sq;
+  };
   auto refresh = [&](int a, const float4 (&w4)[QN]) {
     float sq = 0.f;
 #pragma unroll
-    for (int q = 0; q < QN; ++q) {
-      if (q < nq) {
-        sq = fmaf(w4[q].x, w4[q].x, sq); sq = fmaf(w4[q].y, w4[q].y, sq); sq = fmaf(w4[q].z, w4[q].z, sq); sq = fmaf(w4[q].w, w4[q].w, sq);
-        const size_t o = (size_t)a * d + 4 * l8 + 32 * q;
-        const float v[4] = {-2.f * w4[q].x, -2.f * w4[q].y, -2.f * w4[q].z, -2.f * w4[q].w};     // exact
-        // four 16-bit numbers per store (8 bytes; o is a multiple of 4)
-        if (kTerms == 1) {
-          const __half2 h01 = __floats2half2_rn(v[0], v[1]), h23 = __floats2half2_rn(v[2], v[3]);
-          *reinterpret_cast<uint2*>(wbf + o) = make_uint2(*reinterpret_cast<const unsigned*>(&h01), *reinterpret_cast<const unsigned*>(&h23));
-        } else {
-          const __nv_bfloat162 h01 = __floats2bfloat162_rn(v[0], v[1]), h23 = __floats2bfloat162_rn(v[2], v[3]);
-          const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
-          const __nv_bfloat162 l01 = __floats2bfloat162_rn(v[0] - f01.x, v[1] - f01.y), l23 = __floats2bfloat162_rn(v[2] - f23.x, v[3] - f23.y);
-          *reinterpret_cast<uint2*>(wbf + o) = make_uint2(*reinterpret_cast<const unsigned*>(&h01), *reinterpret_cast<const unsigned*>(&h23));
-          *reinterpret_cast<uint2*>(wbl + o) = make_uint2(*reinterpret_cast<const unsigned*>(&l01), *reinterpret_cast<const unsigned*>(&l23));
-        }
-      }
-    }
+    for (int q = 0; q < QN; ++q)
+      if (q < nq) sq += put16((size_t)a * d + 4 * l8 + 32 * q, w4[q]);
     return sq;
   };
   auto refresh_all = [&]() {                                            // every centre from the fp32 state in HBM
@@ -468,7 +447,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     it_m += (unsigned)m_tiles;
     it_bc += (unsigned)(m_tiles * n_tiles * PPK * nkc);
     it_acc += (unsigned)(n_tiles * m_tiles);
-    if (tid == 0) { misc[1] = 0; misc[5] = 0; misc[6] = 0; }
+    if (tid == 0) { misc[1] = 0; misc[5] = 0; misc[6] = 0; misc[7] = TC_WARPS * 4; }
     for (int a = tid; a < k; a += TC_THREADS) cnt[a] = 0;
     tc_fence_before();
     __syncthreads();
@@ -824,51 +803,84 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     const bool plain = (misc[4] == 0);                    // no message waiting: the fused update below, then the send if one is due
 
     // ---- Eq. 9 and the update: eight lanes per centre add its rows (fp32 master, ascending row order);
-    //      plain step: w <- w - eps (n w - S) / b at once; otherwise S goes to the sum buffer for the general tail ----
+    //      plain step: w <- w - eps (n w - S) / b at once; otherwise S goes to the sum buffer for the general tail.
+    //      The 32 eight-lane groups of the block work through the centres independently: a group takes a few rows of
+    //      its centre per turn, and when the centre is done it finishes it and draws the next centre from a counter, so
+    //      that a group with a large centre does not hold up the three it shares a warp with (all lanes run the same
+    //      instructions; what a group does not need is predicated off) ----
     {
       const int* start = reinterpret_cast<const int*>(sB);
-      for (int a0 = (wid * 4) ; a0 < k; a0 += TC_WARPS * 4) {
-        const int a = a0 + sub;
-        const bool on = a < k;
-        const int n = on ? cnt[a] : 0, p0 = on ? start[a] : 0;
-        float4 S4[QN];
+      const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      auto sum_and_update = [&](auto rows_tag, auto qmax_tag) {
+        constexpr int ROWS = decltype(rows_tag)::value, QMAX = decltype(qmax_tag)::value;   // rows per turn, float4 pieces per lane (nq <= QMAX)
+        int a = wid * 4 + sub;                                 // the group's centre; the next ones come from the counter
+        int n = (a < k) ? cnt[a] : 0, p0 = (a < k) ? start[a] : 0, e = 0;
+        float4 S4[QMAX];
 #pragma unroll
-        for (int q = 0; q < QN; ++q) S4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (nq <= QN / 2) tc_add_rows<2 * TC_SUM_ROWS, QN / 2>(p.X, row0, d, nq, l8, order + p0, n, S4);
-        else tc_add_rows<TC_SUM_ROWS, QN>(p.X, row0, d, nq, l8, order + p0, n, S4);
-        float sq = 0.f;
-        if (on) {
-          if (plain) {
-            float4 w4[QN];
-            const float fn = (float)n;
-            // all of the centre's row first, then the stores: a store between two loads from the same array would keep
-            // the second load behind it (they might alias), one L2 round trip per piece instead of one per row
+        for (int q = 0; q < QMAX; ++q) S4[q] = z4;
+        while (__any_sync(0xffffffffu, a < k)) {
+          const bool live = a < k;
+          // a centre that ends with this turn's rows: its row of the state is asked for together with them
+          const bool moves = plain && live && n > 0 && e + ROWS >= n;                 // (an empty centre stays where it is)
+          float4 w4[QMAX];
 #pragma unroll
-            for (int q = 0; q < QN; ++q)
-              if (q < nq) w4[q] = *reinterpret_cast<const float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q);
+          for (int q = 0; q < QMAX; ++q)
+            w4[q] = (q < nq && moves) ? *reinterpret_cast<const float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q) : z4;
+          {
+            float4 v[ROWS][QMAX];
 #pragma unroll
-            for (int q = 0; q < QN; ++q) {
-              if (q < nq) {
-                float4 u = w4[q];
-                u.x -= p.eps * ((fn * u.x - S4[q].x) * inv_b); u.y -= p.eps * ((fn * u.y - S4[q].y) * inv_b);
-                u.z -= p.eps * ((fn * u.z - S4[q].z) * inv_b); u.w -= p.eps * ((fn * u.w - S4[q].w) * inv_b);
-                *reinterpret_cast<float4*>(wglob + (size_t)a * d + 4 * l8 + 32 * q) = u;
-                w4[q] = u;
-              }
+            for (int u = 0; u < ROWS; ++u) {
+              const bool have = live && e + u < n;
+              const float* x = p.X + (size_t)(row0 + (have ? (int)order[p0 + e + u] : 0)) * d + 4 * l8;
+#pragma unroll
+              for (int q = 0; q < QMAX; ++q) v[u][q] = (q < nq && have) ? __ldg(reinterpret_cast<const float4*>(x + 32 * q)) : z4;
             }
-            sq = refresh(a, w4);
-          } else {
 #pragma unroll
-            for (int q = 0; q < QN; ++q)
-              if (q < nq) *reinterpret_cast<float4*>(gsum + (size_t)a * d + 4 * l8 + 32 * q) = S4[q];
+            for (int u = 0; u < ROWS; ++u)
+#pragma unroll
+              for (int q = 0; q < QMAX; ++q) { S4[q].x += v[u][q].x; S4[q].y += v[u][q].y; S4[q].z += v[u][q].z; S4[q].w += v[u][q].w; }
+          }
+          e += ROWS;
+          const bool done = live && e >= n;
+          if (__any_sync(0xffffffffu, done)) {
+            float sq = 0.f;
+            if (plain) {
+              const float fn = (float)n;
+#pragma unroll
+              for (int q = 0; q < QMAX; ++q) {
+                if (q < nq && moves) {
+                  float4 u = w4[q];
+                  u.x -= p.eps * ((fn * u.x - S4[q].x) * inv_b); u.y -= p.eps * ((fn * u.y - S4[q].y) * inv_b);
+                  u.z -= p.eps * ((fn * u.z - S4[q].z) * inv_b); u.w -= p.eps * ((fn * u.w - S4[q].w) * inv_b);
+                  const size_t o = (size_t)a * d + 4 * l8 + 32 * q;
+                  *reinterpret_cast<float4*>(wglob + o) = u;
+                  sq += put16(o, u);
+                }
+              }
+#pragma unroll
+              for (int o = 1; o < 8; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+              if (moves && l8 == 0) cn[a] = sq;
+            } else if (done) {
+#pragma unroll
+              for (int q = 0; q < QMAX; ++q)
+                if (q < nq) *reinterpret_cast<float4*>(gsum + (size_t)a * d + 4 * l8 + 32 * q) = S4[q];
+            }
+            int nxt = 0;
+            if (done && l8 == 0) nxt = atomicAdd(&misc[7], 1);
+            nxt = __shfl_sync(0xffffffffu, nxt, lane & ~7);
+            if (done) {
+              a = nxt;
+              e = 0;
+              n = (a < k) ? cnt[a] : 0;
+              p0 = (a < k) ? start[a] : 0;
+#pragma unroll
+              for (int q = 0; q < QMAX; ++q) S4[q] = z4;
+            }
           }
         }
-        if (plain) {
-#pragma unroll
-          for (int o = 1; o < 8; o <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-          if (on && l8 == 0) cn[a] = sq;
-        }
-      }
+      };
+      if (nq <= QN / 2) sum_and_update(std::integral_constant<int, 8>(), std::integral_constant<int, QN / 2>());
+      else sum_and_update(std::integral_constant<int, 4>(), std::integral_constant<int, QN>());
     }
     if (!plain) {
       __syncthreads();
