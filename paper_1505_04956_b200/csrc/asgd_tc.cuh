@@ -85,9 +85,28 @@ struct TcSmem {
 };
 inline size_t tc_smem_bytes(int k, int d, int b, int terms, int nv) { return TcSmem(k, d, b, terms, nv).total; }
 
-__device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+// L2 policies: the samples stream through once per pass (first out), a worker's 16-bit state is read again for
+// every sample tile (last out)
+__device__ inline unsigned long long l2_policy_evict_first() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ inline unsigned long long l2_policy_evict_last() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ inline void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, unsigned long long* bar, unsigned long long policy) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+               ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy) : "memory");
+}
+// a float4 of the fp32 samples, read once: first out of L2, not kept in L1
+__device__ inline float4 ldg_stream4(const float4* p, unsigned long long policy) {
+  float4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p), "l"(policy));
+  return v;
 }
 // Shared-memory operand descriptor: K-major rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ inline unsigned long long tc_smem_desc(const void* smem, unsigned byte_off) {
@@ -307,6 +326,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
       if (lane == 0) {
         unsigned um = it_m, ibc = it_bc;
         bool ok = true;
+        const unsigned long long pol_x = l2_policy_evict_first(), pol_w = l2_policy_evict_last();
         for (int m = 0; m < m_tiles && ok; ++m, ++um) {
           for (int kc = 0; kc < nkc && ok; ++kc) {
             if (um > 0) ok = mbar_wait_bounded(bars + TCB_AEMPTY + kc, (um - 1) & 1, p.wait_limit);     // last use of the chunk by the previous tile
@@ -314,9 +334,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             mbar_expect_tx(bars + TCB_AFULL + kc, (unsigned)(PPK * TC_A_STAGE_BYTES));
             const bool withheld = (m == 0 && kc == 0 && step == p.withhold_step);   // failure drill: announced, never copied
             if (!withheld) {
-              tma_load_2d(sA + (size_t)(kc * PPK + 0) * TC_A_STAGE_BYTES, &mapXh, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc);
+              tma_load_2d(sA + (size_t)(kc * PPK + 0) * TC_A_STAGE_BYTES, &mapXh, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc, pol_x);
               if (kTerms == 3)
-                tma_load_2d(sA + (size_t)(kc * PPK + 1) * TC_A_STAGE_BYTES, &mapXl, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc);
+                tma_load_2d(sA + (size_t)(kc * PPK + 1) * TC_A_STAGE_BYTES, &mapXl, kc * TC_KC, (int)(row0 + (long long)m * TC_M), bars + TCB_AFULL + kc, pol_x);
             }
           }
           for (int n = 0; n < n_tiles && ok; ++n) {
@@ -325,7 +345,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
               if (ibc >= TC_B_STAGES) ok = mbar_wait_bounded(bars + TCB_BEMPTY + st, ((ibc / TC_B_STAGES) - 1) & 1, p.wait_limit);
               if (!ok) break;
               mbar_expect_tx(bars + TCB_BFULL + st, (unsigned)TC_B_CHUNK_BYTES);
-              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, (g / PPK) * TC_KC, (g % PPK) * p.W * k + i * k + n * TC_N, bars + TCB_BFULL + st);
+              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, (g / PPK) * TC_KC, (g % PPK) * p.W * k + i * k + n * TC_N, bars + TCB_BFULL + st, pol_w);
             }
           }
         }
@@ -811,6 +831,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     {
       const int* start = reinterpret_cast<const int*>(sB);
       const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+      const unsigned long long pol_x = l2_policy_evict_first();
       auto sum_and_update = [&](auto rows_tag, auto qmax_tag) {
         constexpr int ROWS = decltype(rows_tag)::value, QMAX = decltype(qmax_tag)::value;   // rows per turn, float4 pieces per lane (nq <= QMAX)
         int a = wid * 4 + sub;                                 // the group's centre; the next ones come from the counter
@@ -833,7 +854,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
               const bool have = live && e + u < n;
               const float* x = p.X + (size_t)(row0 + (have ? (int)order[p0 + e + u] : 0)) * d + 4 * l8;
 #pragma unroll
-              for (int q = 0; q < QMAX; ++q) v[u][q] = (q < nq && have) ? __ldg(reinterpret_cast<const float4*>(x + 32 * q)) : z4;
+              for (int q = 0; q < QMAX; ++q) v[u][q] = (q < nq && have) ? ldg_stream4(reinterpret_cast<const float4*>(x + 32 * q), pol_x) : z4;
             }
 #pragma unroll
             for (int u = 0; u < ROWS; ++u)
