@@ -30,7 +30,7 @@ enum PathId { P_GENERIC = 0, P_STREAM = 1, P_TILED = 2, P_TC_BF16 = 3, P_TC_FP16
 // Among the shapes with the same d and enough centres the one that keeps the most threads busy for the given
 // number of workers is taken (small blocks when there are enough workers to fill the GPU with them: a block that
 // serves one worker keeps its state on chip between steps); ties go to the later entry.
-#define ASGD_TILED_SHAPES(X) X(32, 64, 4, 2, 2) X(32, 64, 2, 2, 4) X(128, 128, 4, 4, 1)
+#define ASGD_TILED_SHAPES(X) X(32, 64, 8, 2, 1) X(32, 64, 4, 2, 2) X(32, 64, 2, 2, 4) X(128, 128, 4, 4, 1)
 
 struct Layout {
   size_t state, mail, seq, seen, arb_win, arb_cnt, mail_rows, rowacc, rowin, stats, perm, status, assign_rec, accept_rec, gsum,
