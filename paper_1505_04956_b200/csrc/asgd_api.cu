@@ -62,7 +62,7 @@ bool config_ok(const asgd_config* c) {
 // shapes the tensor-core path can take: d a multiple of 64 up to 256, a batch of at least one 128-row tile
 bool tc_supported(const asgd_config* c) {
   return c->d % TC_KC == 0 && c->d <= TC_MAX_D && c->k >= 1 && c->k <= TC_MAX_K && c->b >= TC_M && c->b <= TC_MAX_B &&
-         tc_smem_bytes(c->k, c->d, c->b, 1, 1) <= kMaxDynSmem && tc_smem_bytes(c->k, c->d, c->b, 3, 1) <= kMaxDynSmem;
+         tc_smem_bytes(c->k, c->d, c->b, 1, 1, TC_THREADS) <= kMaxDynSmem && tc_smem_bytes(c->k, c->d, c->b, 3, 1, TC_THREADS) <= kMaxDynSmem;
 }
 // ... and these are the library's own choice for them
 bool tc_eligible(const asgd_config* c) { return tc_supported(c); }
@@ -122,7 +122,7 @@ struct asgd_ctx {
   int state_on_chip;
   int grid;               // blocks of the worker kernel (tiled path: a block may serve several workers)
   int tiled_shape;        // index into ASGD_TILED_SHAPES of the shape in use
-  int tc_two;             // tensor-core path: the instance that shares an SM between two blocks
+  int tc_inst;            // tensor-core path: 0 = 256 threads, one block per SM; 1 = two blocks share an SM; 2 = 512 threads
   size_t smem_bytes;
   long long t_host;       // steps every worker has done (uniform across workers)
   long long launches;
@@ -236,27 +236,38 @@ int tc_prepare(asgd_ctx* c) {
   const bool fp16 = (c->path == P_TC_FP16);
   const int terms = fp16 ? 1 : 3;
   const int bn = tc_block_rows(cfg.k, terms);
-  // Two blocks per SM (the half-register instance) when there are more workers than SMs, rows of at most 128 numbers,
-  // accumulators of at most 256 tensor-memory columns a block, and room for two blocks' shared memory; else one.
-  // The request is padded so that no more blocks than that share an SM (tensor memory has 512 columns).
+  // Three instances.  Two blocks per SM (half the registers a thread) when there are more workers than SMs, rows of at
+  // most 128 numbers, accumulators of at most 256 tensor-memory columns a block, and room for two blocks' shared
+  // memory.  Else, for rows of at most 128 numbers, one block of 512 threads per SM if its shared memory fits.  Else one
+  // block of 256 threads.  The request is padded so that no more blocks than meant share an SM (tensor memory has 512
+  // columns).
   {
     const int grid2 = std::min(cfg.W, 2 * c->sm_count);
-    const size_t smem2 = tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, (cfg.W + grid2 - 1) / grid2);
-    c->tc_two = cfg.W > c->sm_count && cfg.d <= 128 && tc_tmem_cols(bn) <= 256 && smem2 <= kTwoBlockSmem;
-    if (c->tc_two) {
+    const size_t smem2 = tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, (cfg.W + grid2 - 1) / grid2, TC_THREADS);
+    c->grid = std::min(cfg.W, c->sm_count);
+    const int nv1 = (cfg.W + c->grid - 1) / c->grid;
+    const size_t smem_wide = tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, nv1, TC_THREADS_WIDE);
+    c->tc_inst = 0;
+    if (cfg.W > c->sm_count && cfg.d <= 128 && tc_tmem_cols(bn) <= 256 && smem2 <= kTwoBlockSmem) {
+      c->tc_inst = 1;
       c->grid = grid2;
       c->smem_bytes = std::max(smem2, (size_t)(kMaxDynSmem / 3 + 1024));
+    } else if (cfg.d <= 128 && smem_wide <= kMaxDynSmem) {
+      c->tc_inst = 2;
+      c->smem_bytes = std::max(smem_wide, (size_t)(kMaxDynSmem / 2 + 1024));
     } else {
-      c->grid = std::min(cfg.W, c->sm_count);
-      c->smem_bytes = std::max(tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, (cfg.W + c->grid - 1) / c->grid), (size_t)(kMaxDynSmem / 2 + 1024));
+      c->smem_bytes = std::max(tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, nv1, TC_THREADS), (size_t)(kMaxDynSmem / 2 + 1024));
       if (c->smem_bytes > kMaxDynSmem) return ASGD_EUNSUPPORTED;
     }
   }
-#define TC_SET(DET_, T_, D_) CU(c, cudaFuncSetAttribute(asgd_tc_kernel<DET_, T_, D_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes))
-  if (fp16 && c->tc_two) { TC_SET(true, 1, 128); TC_SET(false, 1, 128); }
-  else if (fp16) { TC_SET(true, 1, 256); TC_SET(false, 1, 256); }
-  else if (c->tc_two) { TC_SET(true, 3, 128); TC_SET(false, 3, 128); }
-  else { TC_SET(true, 3, 256); TC_SET(false, 3, 256); }
+#define TC_SET(DET_, T_, D_, NT_) CU(c, cudaFuncSetAttribute(asgd_tc_kernel<DET_, T_, D_, NT_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes))
+#define TC_SET_BOTH(T_, D_, NT_) { TC_SET(true, T_, D_, NT_); TC_SET(false, T_, D_, NT_); }
+  if (fp16) {
+    if (c->tc_inst == 1) TC_SET_BOTH(1, 128, TC_THREADS) else if (c->tc_inst == 2) TC_SET_BOTH(1, 128, TC_THREADS_WIDE) else TC_SET_BOTH(1, 256, TC_THREADS)
+  } else {
+    if (c->tc_inst == 1) TC_SET_BOTH(3, 128, TC_THREADS) else if (c->tc_inst == 2) TC_SET_BOTH(3, 128, TC_THREADS_WIDE) else TC_SET_BOTH(3, 256, TC_THREADS)
+  }
+#undef TC_SET_BOTH
 #undef TC_SET
   p.wbf = c->ws + c->L.wbf;
   p.top2 = (float*)(c->ws + c->L.top2);
@@ -289,15 +300,15 @@ int tc_prepare(asgd_ctx* c) {
 int launch_workers(asgd_ctx* c, bool det, long long steps) {
   const Params& p = c->p;
   switch (c->path) {
-#define TC_GO(DET_, T_, D_) asgd_tc_kernel<DET_, T_, D_><<<c->grid, TC_THREADS, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW)
+#define TC_GO(DET_, T_, D_, NT_) asgd_tc_kernel<DET_, T_, D_, NT_><<<c->grid, NT_, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW)
+#define TC_GO_BOTH(T_, D_, NT_) { if (det) TC_GO(true, T_, D_, NT_); else TC_GO(false, T_, D_, NT_); }
     case P_TC_BF16:
-      if (c->tc_two) { if (det) TC_GO(true, 3, 128); else TC_GO(false, 3, 128); }
-      else { if (det) TC_GO(true, 3, 256); else TC_GO(false, 3, 256); }
+      if (c->tc_inst == 1) TC_GO_BOTH(3, 128, TC_THREADS) else if (c->tc_inst == 2) TC_GO_BOTH(3, 128, TC_THREADS_WIDE) else TC_GO_BOTH(3, 256, TC_THREADS)
       break;
     case P_TC_FP16:
-      if (c->tc_two) { if (det) TC_GO(true, 1, 128); else TC_GO(false, 1, 128); }
-      else { if (det) TC_GO(true, 1, 256); else TC_GO(false, 1, 256); }
+      if (c->tc_inst == 1) TC_GO_BOTH(1, 128, TC_THREADS) else if (c->tc_inst == 2) TC_GO_BOTH(1, 128, TC_THREADS_WIDE) else TC_GO_BOTH(1, 256, TC_THREADS)
       break;
+#undef TC_GO_BOTH
 #undef TC_GO
     case P_TILED: {
       int idx = 0;

@@ -41,8 +41,8 @@
 
 namespace asgd {
 
-constexpr int TC_THREADS = 256;
-constexpr int TC_WARPS = TC_THREADS / 32;
+constexpr int TC_THREADS = 256, TC_THREADS_WIDE = 512;    // threads of a block: the usual instance, and the one for rows of at most 128 numbers (half the registers a thread)
+constexpr int TC_GROUP_WARPS = 8;                         // row blocks of the grouping phase (whatever the block's size)
 constexpr int TC_M = 128, TC_KC = 64;                    // rows of an MMA's output tile; K chunk = 64 16-bit numbers = one swizzled 128-byte row
 // most centres per block (the MMA's N): 256 with one term per operand, 128 with two (the sample tile then takes twice the room)
 __host__ __device__ constexpr int tc_block_n(int terms) { return terms == 1 ? 256 : 128; }
@@ -62,14 +62,16 @@ constexpr float TC_FAR = 1e30f;                          // stands for ||w_a||^2
 struct TcSmem {
   size_t B, A, cn, cnt, best, flagged, bars, misc, tail, total;
   int cn_stride;               // floats of ||w_a||^2 per worker of the block
-  // nv: workers the block serves in turn (their ||w_a||^2 stay on chip side by side)
-  __host__ __device__ TcSmem(int k, int d, int b, int terms, int nv) {
+  // (the workers' ||w_a||^2 stay on chip side by side)
+  size_t stage;                // epilogue warps that share a row hand their parts to the first of them here
+  // nv: workers the block serves in turn; threads: the block's size
+  __host__ __device__ TcSmem(int k, int d, int b, int terms, int nv, int threads) {
     const int nb = tc_block_rows(k, terms);
     size_t off = 0;
     auto take = [&](size_t bytes, size_t align) { off = (off + align - 1) / align * align; size_t o = off; off += bytes; return o; };
     // [K chunk][hi, lo] of the resident sample tile; also the scratch of the grouping phase ([warps][k] counts, [b] ranks)
     const size_t tile = (size_t)(d / TC_KC) * (terms == 3 ? 2 : 1) * TC_A_STAGE_BYTES;
-    const size_t scratch = (size_t)TC_WARPS * k * 4 + (size_t)b * 2;
+    const size_t scratch = (size_t)TC_GROUP_WARPS * k * 4 + (size_t)b * 2;
     A = take(tile > scratch ? tile : scratch, 1024);
     B = take((size_t)TC_B_STAGES * nb * TC_KC * 2, 1024);                // also [k] group starts and the scans' results (nb >= 32: 16 KB)
     cn_stride = (k + nb - 1) / nb * nb;
@@ -77,13 +79,15 @@ struct TcSmem {
     cnt = take((size_t)k * 4, 16);
     best = take((size_t)b * 2, 16);
     flagged = take((size_t)b * 2 + 16, 16);                          // pairs to settle from the front, rows for the full scan from the back
+    const int per_row = (threads / 32 - 4) / 4;                       // epilogue warps per quarter of a sample tile
+    stage = take(per_row > 1 ? (size_t)2 * per_row * TC_M * 16 : 0, 16);   // [tile parity][part][row] (s1, s2, s3, floor)
     bars = take(32 * 8, 16);
     misc = take(64, 16);
     tail = take(sizeof(TailScratch), 16);
     total = off + 1024;          // room to align the base to 1024 bytes
   }
 };
-inline size_t tc_smem_bytes(int k, int d, int b, int terms, int nv) { return TcSmem(k, d, b, terms, nv).total; }
+inline size_t tc_smem_bytes(int k, int d, int b, int terms, int nv, int threads) { return TcSmem(k, d, b, terms, nv, threads).total; }
 
 // L2 policies: the samples stream through once per pass (first out), a worker's 16-bit state is read again for
 // every sample tile (last out)
@@ -193,8 +197,10 @@ __device__ __forceinline__ void tc_top3_insert2(float& m1, float& m2, float& m3,
 
 // kMaxD: the largest d the instance holds in registers.  256: one block per SM.  128: half the registers, so that two
 // blocks share an SM when their shared memory allows it; one block's scores then overlap the other's sums and update.
-template <bool kDet, int kTerms, int kMaxD>
-__global__ void __launch_bounds__(TC_THREADS, kMaxD <= 128 ? 2 : 1)
+// kThreads: 256, or 512 for a block that has an SM to itself and rows of at most 128 numbers: three epilogue warps per
+// quarter of a sample tile instead of one, and twice the warps in every later phase.
+template <bool kDet, int kTerms, int kMaxD, int kThreads>
+__global__ void __launch_bounds__(kThreads, (kMaxD <= 128 && kThreads == TC_THREADS) ? 2 : 1)
 asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CUtensorMap mapXh,
                const __grid_constant__ CUtensorMap mapXl, const __grid_constant__ CUtensorMap mapW) {
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
@@ -202,7 +208,10 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   const int k = p.k, d = p.d, b = p.b;
   const int G = (int)gridDim.x;
   const int nv = (p.W - (int)blockIdx.x + G - 1) / G;                   // workers of this block: blockIdx.x + v * G
-  const TcSmem map(k, d, b, kTerms, (p.W + G - 1) / G);
+  constexpr int NT = kThreads, NW = kThreads / 32;                      // threads and warps of the block
+  constexpr int GW = TC_GROUP_WARPS;
+  static_assert(kThreads == TC_THREADS || (kThreads == TC_THREADS_WIDE && kMaxD <= 128), "512 threads only with 128 registers a thread");
+  const TcSmem map(k, d, b, kTerms, (p.W + G - 1) / G, NT);
   unsigned char* sB = smem + map.B;
   unsigned char* sA = smem + map.A;
   float* cn = reinterpret_cast<float*>(smem + map.cn);                 // ||w_a||^2 of the worker in turn; beyond k a large finite number (with
@@ -246,7 +255,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   if (tid == 0) {
     for (int q = 0; q < TC_B_STAGES; ++q) { mbar_init(bars + TCB_BFULL + q, 1); mbar_init(bars + TCB_BEMPTY + q, 1); }
     for (int q = 0; q < TC_A_STAGES; ++q) { mbar_init(bars + TCB_AFULL + q, 1); mbar_init(bars + TCB_AEMPTY + q, 1); }
-    for (int q = 0; q < 2; ++q) { mbar_init(bars + TCB_ACCFULL + q, 1); mbar_init(bars + TCB_ACCEMPTY + q, 4); }
+    for (int q = 0; q < 2; ++q) { mbar_init(bars + TCB_ACCFULL + q, 1); mbar_init(bars + TCB_ACCEMPTY + q, NW - 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     misc[2] = 0;
   }
@@ -283,7 +292,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     return sq;
   };
   auto refresh_all = [&]() {                                            // every centre from the fp32 state in HBM
-    for (int a0 = wid * 4; a0 < n_tiles * TC_N; a0 += TC_WARPS * 4) {
+    for (int a0 = wid * 4; a0 < n_tiles * TC_N; a0 += NW * 4) {
       const int a = a0 + sub;
       float sq = 0.f;
       if (a < k) {
@@ -392,8 +401,11 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         if (!ok) atomicExch(&misc[2], 1);
       }
     } else if (wid >= 4) {
-      // four warps read the accumulators: warp q of them owns TMEM lanes 32q .. 32q+31, i.e. one row per thread
-      const int quarter = wid & 3;
+      // the other warps read the accumulators: a warp can reach the TMEM lanes 32q .. 32q+31 with q = warp mod 4, i.e.
+      // one row per thread; the EPW warps of a quarter take the 32-column groups of a centre block in turn
+      constexpr int EPW = (NW - 4) / 4;
+      const int quarter = wid & 3, part = (wid - 4) >> 2;
+      float4* stage = reinterpret_cast<float4*>(smem + map.stage);    // [tile parity][part][row of the tile]
       unsigned iacc = it_acc;
       bool ok = true;
       for (int m = 0; m < m_tiles; ++m) {
@@ -407,8 +419,12 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           if (ok) ok = __all_sync(0xffffffffu, mbar_wait_bounded(bars + TCB_ACCFULL + buf, (iacc >> 1) & 1, p.wait_limit));
           if (!ok) continue;
           tc_fence_after();
+          if (32 * part >= TC_N) {                        // fewer column groups than warps: nothing to read here
+            tc_fence_before();
+            if (lane == 0) mbar_arrive(bars + TCB_ACCEMPTY + buf);
+          }
 #pragma unroll 1
-          for (int c0 = 0; c0 < TC_N; c0 += 32) {
+          for (int c0 = 32 * part; c0 < TC_N; c0 += 32 * EPW) {
             unsigned v[32];
             const unsigned taddr = tmem + ((unsigned)(quarter * 32) << 16) + (unsigned)(buf * TC_N + c0);
             asm volatile(
@@ -419,7 +435,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
                   "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
                 : "r"(taddr) : "memory");
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (c0 + 32 == TC_N) {                        // last read of this accumulator stage: hand it back
+            if (c0 + 32 * EPW >= TC_N) {                  // this warp's last read of the accumulator stage: hand it back
               tc_fence_before();
               if (lane == 0) mbar_arrive(bars + TCB_ACCEMPTY + buf);
             }
@@ -445,7 +461,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             }
           }
         }
-        if (ok && r < b) {
+        {
           // the four smallest of the twelve kept values.  Every value that was not kept is at least the largest of its
           // triple, so the fourth smallest of ALL values is at least min(fourth smallest kept, smallest of the four
           // triples' largest): a floor under the fourth candidate that costs nothing in the loop above
@@ -458,8 +474,26 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           };
 #pragma unroll
           for (int q = 0; q < 4; ++q) { put4(m1[q]); put4(m2[q]); put4(m3[q]); }
-          const float floor4 = fminf(a4, fminf(fminf(m3[0], m3[1]), fminf(m3[2], m3[3])));
-          __stcg(top3 + r, make_float4(a1, a2, a3, floor4));
+          float floor4 = fminf(a4, fminf(fminf(m3[0], m3[1]), fminf(m3[2], m3[3])));
+          if (EPW > 1) {
+            // the parts of a row meet in shared memory (every warp of the quarter comes to the barrier, whatever its
+            // waits did): the three smallest of all parts are among the parts' three smallest, and the fourth smallest
+            // of all is one of those or at least some part's floor
+            float4* mine = stage + ((size_t)(m & 1) * EPW + part) * TC_M + quarter * 32 + lane;
+            if (part > 0) *mine = make_float4(a1, a2, a3, floor4);
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + quarter), "r"(32 * EPW) : "memory");
+            if (part == 0) {
+              a4 = __int_as_float(0x7f800000);
+#pragma unroll
+              for (int q = 1; q < EPW; ++q) {
+                const float4 o = mine[(size_t)q * TC_M];
+                put4(o.x); put4(o.y); put4(o.z);
+                floor4 = fminf(floor4, o.w);
+              }
+              floor4 = fminf(floor4, a4);
+            }
+          }
+          if (ok && r < b && part == 0) __stcg(top3 + r, make_float4(a1, a2, a3, floor4));
         }
       }
       if (!ok && lane == 0) atomicExch(&misc[2], 1);
@@ -467,8 +501,8 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     it_m += (unsigned)m_tiles;
     it_bc += (unsigned)(m_tiles * n_tiles * PPK * nkc);
     it_acc += (unsigned)(n_tiles * m_tiles);
-    if (tid == 0) { misc[1] = 0; misc[5] = 0; misc[6] = 0; misc[7] = TC_WARPS * 4; }
-    for (int a = tid; a < k; a += TC_THREADS) cnt[a] = 0;
+    if (tid == 0) { misc[1] = 0; misc[5] = 0; misc[6] = 0; misc[7] = NW * 4; }
+    for (int a = tid; a < k; a += NT) cnt[a] = 0;
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -497,14 +531,14 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     };
     auto inside = [&](float lo, float hi_, float err) { return (hi_ - lo) <= 2.f * err + 2.4415e-4f * fmaxf(fabsf(lo), fabsf(hi_)); };
     // Scratch for the rest of the step lives in the sample ring, which is idle until the next step's loads.
-    int* wcnt = reinterpret_cast<int*>(sA);                                   // [TC_WARPS][k] rows of a centre in a warp's row block
-    unsigned short* lrank = reinterpret_cast<unsigned short*>(sA + (size_t)TC_WARPS * k * 4);   // [b] rank of a row among its warp's rows of the centre
+    int* wcnt = reinterpret_cast<int*>(sA);                                   // [GW][k] rows of a centre in a row block
+    unsigned short* lrank = reinterpret_cast<unsigned short*>(sA + (size_t)GW * k * 4);   // [b] rank of a row among its block's rows of the centre
     unsigned short* order = flagged;                                          // [b] rows grouped by centre, ascending inside a group
     unsigned short* triples = lrank;                                          // until the grouping: rows with exactly three candidates
 
     // ---- decide: the minimum, unless the runner-up lies inside the bound (settle the pair) or the third does too (scan all) ----
-    for (int e = tid; e < TC_WARPS * k; e += TC_THREADS) wcnt[e] = 0;
-    for (int r = tid; r < b; r += TC_THREADS) {
+    for (int e = tid; e < GW * k; e += NT) wcnt[e] = 0;
+    for (int r = tid; r < b; r += NT) {
       const float4 s = __ldcg(top3 + r);
       best[r] = (unsigned short)(__float_as_uint(s.x) & TC_INDEX_MASK);
       const float err = row_err(__ldg(p.xnorm + row0 + r));
@@ -523,7 +557,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     //      dimensions 4*l8 + 32*q), a warp settles four rows at a time ----
     {
       const int npair = misc[1], ntrip = misc[6];
-      const int groups = TC_WARPS * 4;
+      const int groups = NW * 4;
       for (int fb = wid * 4; fb < npair + ntrip; fb += groups) {   // the same trip count for all lanes of a warp (shuffles inside)
         const int f = fb + sub;
         const bool have = f < npair + ntrip;
@@ -615,8 +649,8 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         constexpr int RB = decltype(rb_tag)::value, CB = decltype(cb_tag)::value;
         constexpr int VR = RB * CB;                            // (centre slot c, row j) pairs, pair c * RB + j
         constexpr int LPR = 32 / VR;                           // lanes that end up with the same pair: LPR * v .. LPR * v + LPR - 1
-        float* res = reinterpret_cast<float*>(sB);             // [TC_WARPS][VR][5] per warp and pair: the three smallest, indices of the first two
-        int* need64 = reinterpret_cast<int*>(res + TC_WARPS * VR * 5);    // [RB][3]: 0 decided, 1 compare two in fp64, 2 scan all in fp64; the two indices
+        float* res = reinterpret_cast<float*>(sB);             // [NW][VR][5] per warp and pair: the three smallest, indices of the first two
+        int* need64 = reinterpret_cast<int*>(res + NW * VR * 5);    // [RB][3]: 0 decided, 1 compare two in fp64, 2 scan all in fp64; the two indices
         float4 xr0[RB], xr1[RB];                               // this lane's dimensions of the rows (zeros past the last row)
 #pragma unroll
         for (int j = 0; j < RB; ++j) {
@@ -631,15 +665,15 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         float4 w0v[CB], w1v[CB];
 #pragma unroll
         for (int c = 0; c < CB; ++c) {
-          const float4* wa = reinterpret_cast<const float4*>(wglob + (size_t)min(wid + TC_WARPS * c, k - 1) * d);
+          const float4* wa = reinterpret_cast<const float4*>(wglob + (size_t)min(wid + NW * c, k - 1) * d);
           w0v[c] = on0 ? wa[lane] : z4;
           w1v[c] = on1 ? wa[32 + lane] : z4;
         }
-        for (int a = wid; a < k; a += TC_WARPS * CB) {         // ascending inside a slot: a strict "<" keeps the lowest index of a tie
+        for (int a = wid; a < k; a += NW * CB) {         // ascending inside a slot: a strict "<" keeps the lowest index of a tie
           float4 n0[CB], n1[CB];                               // the next iteration's rows of the state
 #pragma unroll
           for (int c = 0; c < CB; ++c) {
-            const float4* wn = reinterpret_cast<const float4*>(wglob + (size_t)min(a + TC_WARPS * (CB + c), k - 1) * d);
+            const float4* wn = reinterpret_cast<const float4*>(wglob + (size_t)min(a + NW * (CB + c), k - 1) * d);
             n0[c] = on0 ? wn[lane] : z4;
             n1[c] = on1 ? wn[32 + lane] : z4;
           }
@@ -672,7 +706,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           float tot = part[0];                                  // lanes LPR * v .. : pair v, each with a share of it
 #pragma unroll
           for (int o = LPR / 2; o >= 1; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
-          const int a_mine = a + TC_WARPS * c_mine;
+          const int a_mine = a + NW * c_mine;
           if ((lane & (LPR - 1)) == 0 && a_mine < k) {
             if (tot < bd1) { bd3 = bd2; bd2 = bd1; bi2 = bi1; bd1 = tot; bi1 = a_mine; }
             else if (tot < bd2) { bd3 = bd2; bd2 = tot; bi2 = a_mine; }
@@ -696,7 +730,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             else if (v < fd2 || (v == fd2 && idx < fi2)) { fd3 = fd2; fd2 = v; fi2 = idx; }
             else if (v < fd3) { fd3 = v; }
           };
-          for (int q = 0; q < TC_WARPS * CB; ++q) {             // every warp's every centre slot
+          for (int q = 0; q < NW * CB; ++q) {                   // every warp's every centre slot
             const float* o = res + (q * RB + tid) * 5;
             put(o[0], __float_as_int(o[3]));
             put(o[1], __float_as_int(o[4]));
@@ -712,7 +746,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
           if (tid < R && how == 0) best[order[b - 1 - (base + tid)]] = (unsigned short)fi1;
         }
         __syncthreads();
-        for (int j = wid; j < R; j += TC_WARPS) {              // warp-uniform: need64[j] is the same for every lane
+        for (int j = wid; j < R; j += NW) {                    // warp-uniform: need64[j] is the same for every lane
           const int how = need64[j * 3 + 0];
           if (how == 0) continue;
           const float4* xrow = reinterpret_cast<const float4*>(p.X + (size_t)(row0 + (int)order[b - 1 - (base + j)]) * d);
@@ -757,13 +791,13 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     }
     __syncthreads();
     if (p.assign_rec)
-      for (int r = tid; r < b; r += TC_THREADS) p.assign_rec[(size_t)i * b + r] = best[r];
+      for (int r = tid; r < b; r += NT) p.assign_rec[(size_t)i * b + r] = best[r];
 
     // ---- rows grouped by centre, in row order (stable): ranks inside each warp's block of rows, then offsets ----
     {
-      const int R = ((b + TC_WARPS - 1) / TC_WARPS + 31) / 32 * 32;           // rows per warp, whole chunks of 32
-      int* mine = wcnt + wid * k;
-      for (int r0 = wid * R; r0 < min(b, (wid + 1) * R); r0 += 32) {
+      const int R = ((b + GW - 1) / GW + 31) / 32 * 32;                       // rows per block of rows, whole chunks of 32
+      int* mine = wcnt + min(wid, GW - 1) * k;
+      for (int r0 = wid * R; wid < GW && r0 < min(b, (wid + 1) * R); r0 += 32) {
         const int r = r0 + lane;
         const int a = (r < b) ? (int)best[r] : -1;
         const unsigned grp = __match_any_sync(0xffffffffu, a);
@@ -785,7 +819,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         const int a = tid * 4 + u;
         int c = 0;
         if (a < k)
-          for (int w8 = 0; w8 < TC_WARPS; ++w8) { const int v = wcnt[w8 * k + a]; wcnt[w8 * k + a] = c; c += v; }   // per-warp offsets
+          for (int w8 = 0; w8 < GW; ++w8) { const int v = wcnt[w8 * k + a]; wcnt[w8 * k + a] = c; c += v; }   // per-block offsets
         tot[u] = c;
         run += c;
       }
@@ -807,8 +841,8 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
     __syncthreads();
     {
       const int* start = reinterpret_cast<const int*>(sB);
-      const int R = ((b + TC_WARPS - 1) / TC_WARPS + 31) / 32 * 32;
-      for (int r = tid; r < b; r += TC_THREADS) {
+      const int R = ((b + GW - 1) / GW + 31) / 32 * 32;
+      for (int r = tid; r < b; r += NT) {
         const int a = best[r];
         order[start[a] + wcnt[(r / R) * k + a] + lrank[r]] = (unsigned short)r;
       }
@@ -915,7 +949,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
         n_sent = step_send_any<kDet>(p, i, t, wglob, d, ts);
       }
       if (kDet && p.rows_m > 0)                            // per-row record of a step that looked at no message
-        for (int a = tid; a < p.k; a += TC_THREADS) p.rowin[(size_t)i * p.k + a] = 0;
+        for (int a = tid; a < p.k; a += NT) p.rowin[(size_t)i * p.k + a] = 0;
       if (tid == 0) {
         if (kDet)
           for (int s = 0; s < p.S; ++s) p.accept_rec[(size_t)i * p.S + s] = -1;
