@@ -62,7 +62,7 @@ bool config_ok(const asgd_config* c) {
 // shapes the tensor-core path can take: d a multiple of 64 up to 256, a batch of at least one 128-row tile
 bool tc_supported(const asgd_config* c) {
   return c->d % TC_KC == 0 && c->d <= TC_MAX_D && c->k >= 1 && c->k <= TC_MAX_K && c->b >= TC_M && c->b <= TC_MAX_B &&
-         tc_smem_bytes(c->k, c->d, c->b, 1, 1, TC_THREADS) <= kMaxDynSmem && tc_smem_bytes(c->k, c->d, c->b, 3, 1, TC_THREADS) <= kMaxDynSmem;
+         tc_smem_bytes(c->k, c->d, c->b, 1, 1, TC_THREADS_MID) <= kMaxDynSmem && tc_smem_bytes(c->k, c->d, c->b, 3, 1, TC_THREADS_MID) <= kMaxDynSmem;
 }
 // ... and these are the library's own choice for them
 bool tc_eligible(const asgd_config* c) { return tc_supported(c); }
@@ -122,7 +122,7 @@ struct asgd_ctx {
   int state_on_chip;
   int grid;               // blocks of the worker kernel (tiled path: a block may serve several workers)
   int tiled_shape;        // index into ASGD_TILED_SHAPES of the shape in use
-  int tc_inst;            // tensor-core path: 0 = 256 threads, one block per SM; 1 = two blocks share an SM; 2 = 512 threads
+  int tc_inst;            // tensor-core path: 0 = 384 threads, one block per SM; 1 = 256 threads, two blocks share an SM; 2 = 512 threads
   size_t smem_bytes;
   long long t_host;       // steps every worker has done (uniform across workers)
   long long launches;
@@ -236,10 +236,10 @@ int tc_prepare(asgd_ctx* c) {
   const bool fp16 = (c->path == P_TC_FP16);
   const int terms = fp16 ? 1 : 3;
   const int bn = tc_block_rows(cfg.k, terms);
-  // Three instances.  Two blocks per SM (half the registers a thread) when there are more workers than SMs, rows of at
-  // most 128 numbers, accumulators of at most 256 tensor-memory columns a block, and room for two blocks' shared
-  // memory.  Else, for rows of at most 128 numbers, one block of 512 threads per SM if its shared memory fits.  Else one
-  // block of 256 threads.  The request is padded so that no more blocks than meant share an SM (tensor memory has 512
+  // Three instances.  Two blocks of 256 threads per SM when there are more workers than SMs, rows of at most 128
+  // numbers, accumulators of at most 256 tensor-memory columns a block, and room for two blocks' shared memory.  Else,
+  // for rows of at most 128 numbers, one block of 512 threads per SM if its shared memory fits.  Else one block of 384
+  // threads.  The request is padded so that no more blocks than meant share an SM (tensor memory has 512
   // columns).
   {
     const int grid2 = std::min(cfg.W, 2 * c->sm_count);
@@ -256,16 +256,16 @@ int tc_prepare(asgd_ctx* c) {
       c->tc_inst = 2;
       c->smem_bytes = std::max(smem_wide, (size_t)(kMaxDynSmem / 2 + 1024));
     } else {
-      c->smem_bytes = std::max(tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, nv1, TC_THREADS), (size_t)(kMaxDynSmem / 2 + 1024));
+      c->smem_bytes = std::max(tc_smem_bytes(cfg.k, cfg.d, cfg.b, terms, nv1, TC_THREADS_MID), (size_t)(kMaxDynSmem / 2 + 1024));
       if (c->smem_bytes > kMaxDynSmem) return ASGD_EUNSUPPORTED;
     }
   }
 #define TC_SET(DET_, T_, D_, NT_) CU(c, cudaFuncSetAttribute(asgd_tc_kernel<DET_, T_, D_, NT_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->smem_bytes))
 #define TC_SET_BOTH(T_, D_, NT_) { TC_SET(true, T_, D_, NT_); TC_SET(false, T_, D_, NT_); }
   if (fp16) {
-    if (c->tc_inst == 1) TC_SET_BOTH(1, 128, TC_THREADS) else if (c->tc_inst == 2) TC_SET_BOTH(1, 128, TC_THREADS_WIDE) else TC_SET_BOTH(1, 256, TC_THREADS)
+    if (c->tc_inst == 1) TC_SET_BOTH(1, 128, TC_THREADS) else if (c->tc_inst == 2) TC_SET_BOTH(1, 128, TC_THREADS_WIDE) else TC_SET_BOTH(1, 256, TC_THREADS_MID)
   } else {
-    if (c->tc_inst == 1) TC_SET_BOTH(3, 128, TC_THREADS) else if (c->tc_inst == 2) TC_SET_BOTH(3, 128, TC_THREADS_WIDE) else TC_SET_BOTH(3, 256, TC_THREADS)
+    if (c->tc_inst == 1) TC_SET_BOTH(3, 128, TC_THREADS) else if (c->tc_inst == 2) TC_SET_BOTH(3, 128, TC_THREADS_WIDE) else TC_SET_BOTH(3, 256, TC_THREADS_MID)
   }
 #undef TC_SET_BOTH
 #undef TC_SET
@@ -303,10 +303,10 @@ int launch_workers(asgd_ctx* c, bool det, long long steps) {
 #define TC_GO(DET_, T_, D_, NT_) asgd_tc_kernel<DET_, T_, D_, NT_><<<c->grid, NT_, c->smem_bytes, c->stream>>>(p, steps, c->mapXh, c->mapXl, c->mapW)
 #define TC_GO_BOTH(T_, D_, NT_) { if (det) TC_GO(true, T_, D_, NT_); else TC_GO(false, T_, D_, NT_); }
     case P_TC_BF16:
-      if (c->tc_inst == 1) TC_GO_BOTH(3, 128, TC_THREADS) else if (c->tc_inst == 2) TC_GO_BOTH(3, 128, TC_THREADS_WIDE) else TC_GO_BOTH(3, 256, TC_THREADS)
+      if (c->tc_inst == 1) TC_GO_BOTH(3, 128, TC_THREADS) else if (c->tc_inst == 2) TC_GO_BOTH(3, 128, TC_THREADS_WIDE) else TC_GO_BOTH(3, 256, TC_THREADS_MID)
       break;
     case P_TC_FP16:
-      if (c->tc_inst == 1) TC_GO_BOTH(1, 128, TC_THREADS) else if (c->tc_inst == 2) TC_GO_BOTH(1, 128, TC_THREADS_WIDE) else TC_GO_BOTH(1, 256, TC_THREADS)
+      if (c->tc_inst == 1) TC_GO_BOTH(1, 128, TC_THREADS) else if (c->tc_inst == 2) TC_GO_BOTH(1, 128, TC_THREADS_WIDE) else TC_GO_BOTH(1, 256, TC_THREADS_MID)
       break;
 #undef TC_GO_BOTH
 #undef TC_GO

@@ -41,7 +41,9 @@
 
 namespace asgd {
 
-constexpr int TC_THREADS = 256, TC_THREADS_WIDE = 512;    // threads of a block: the usual instance, and the one for rows of at most 128 numbers (half the registers a thread)
+// threads of a block: two blocks per SM; one block per SM with rows of up to 256 numbers (168 registers a thread); one
+// block per SM with rows of at most 128 numbers (128 registers a thread)
+constexpr int TC_THREADS = 256, TC_THREADS_MID = 384, TC_THREADS_WIDE = 512;
 constexpr int TC_GROUP_WARPS = 8;                         // row blocks of the grouping phase (whatever the block's size)
 constexpr int TC_M = 128, TC_KC = 64;                    // rows of an MMA's output tile; K chunk = 64 16-bit numbers = one swizzled 128-byte row
 // most centres per block (the MMA's N): 256 with one term per operand, 128 with two (the sample tile then takes twice the room)
@@ -77,10 +79,14 @@ struct TcSmem {
     cn_stride = (k + nb - 1) / nb * nb;
     cn = take((size_t)nv * cn_stride * 4, 16);
     cnt = take((size_t)k * 4, 16);
-    best = take((size_t)b * 2, 16);
-    flagged = take((size_t)b * 2 + 16, 16);                          // pairs to settle from the front, rows for the full scan from the back
+    // best[b] and flagged[b + 8] (pairs to settle from the front, rows for the full scan from the back) are dead while
+    // the scores are computed: the epilogue's hand-over area [tile parity][part][row] of (s1, s2, s3, floor) shares their room
     const int per_row = (threads / 32 - 4) / 4;                       // epilogue warps per quarter of a sample tile
-    stage = take(per_row > 1 ? (size_t)2 * per_row * TC_M * 16 : 0, 16);   // [tile parity][part][row] (s1, s2, s3, floor)
+    const size_t best_bytes = ((size_t)b * 2 + 15) / 16 * 16, flag_bytes = ((size_t)b * 2 + 16 + 15) / 16 * 16;
+    const size_t stage_bytes = per_row > 1 ? (size_t)2 * per_row * TC_M * 16 : 0;
+    best = take(best_bytes + flag_bytes > stage_bytes ? best_bytes + flag_bytes : stage_bytes, 16);
+    flagged = best + best_bytes;
+    stage = best;
     bars = take(32 * 8, 16);
     misc = take(64, 16);
     tail = take(sizeof(TailScratch), 16);
@@ -197,8 +203,8 @@ __device__ __forceinline__ void tc_top3_insert2(float& m1, float& m2, float& m3,
 
 // kMaxD: the largest d the instance holds in registers.  256: one block per SM.  128: half the registers, so that two
 // blocks share an SM when their shared memory allows it; one block's scores then overlap the other's sums and update.
-// kThreads: 256, or 512 for a block that has an SM to itself and rows of at most 128 numbers: three epilogue warps per
-// quarter of a sample tile instead of one, and twice the warps in every later phase.
+// kThreads: 256 where two blocks share an SM; a block that has an SM to itself takes 384 threads (two epilogue warps per
+// quarter of a sample tile), or 512 with rows of at most 128 numbers (three), and as many more warps in every later phase.
 template <bool kDet, int kTerms, int kMaxD, int kThreads>
 __global__ void __launch_bounds__(kThreads, (kMaxD <= 128 && kThreads == TC_THREADS) ? 2 : 1)
 asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CUtensorMap mapXh,
@@ -210,7 +216,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   const int nv = (p.W - (int)blockIdx.x + G - 1) / G;                   // workers of this block: blockIdx.x + v * G
   constexpr int NT = kThreads, NW = kThreads / 32;                      // threads and warps of the block
   constexpr int GW = TC_GROUP_WARPS;
-  static_assert(kThreads == TC_THREADS || (kThreads == TC_THREADS_WIDE && kMaxD <= 128), "512 threads only with 128 registers a thread");
+  static_assert(kThreads <= TC_THREADS_MID || kMaxD <= 128, "512 threads only with 128 registers a thread");
   const TcSmem map(k, d, b, kTerms, (p.W + G - 1) / G, NT);
   unsigned char* sB = smem + map.B;
   unsigned char* sA = smem + map.A;
