@@ -45,7 +45,10 @@ typedef enum asgd_status {
   ASGD_ETIMEOUT = -5      /* a bounded device-side wait expired (reported by asgd_sync)     */
 } asgd_status;
 
-/* Distance paths (a2).  AUTO picks by k and d. */
+/* Distance paths of the assignment (Eq. 8).  AUTO takes, in this order: the streaming kernel for the small shapes
+ * it is compiled for (k, d <= 16, b <= 512); the tensor-core path with FP16 operands where d is a multiple of 64 up
+ * to 256, k <= 1024 and 128 <= b <= 4096 (and the samples fit FP16, see below); the register-tiled kernel (d = 32
+ * with k <= 64, d = 128 with k <= 128); else the shape-independent kernel.  Every path decides Eq. 8 exactly. */
 enum {
   ASGD_PATH_AUTO = 0,
   ASGD_PATH_FP32 = 1,       /* CUDA cores, fp32 (the specialised kernel for the shape, if any) */

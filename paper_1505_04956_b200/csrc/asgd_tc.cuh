@@ -1,33 +1,33 @@
-// Tensor-core path (tcgen05, BF16 operands in two terms each, FP32 accumulate in tensor memory) for large
-// states (k up to 1024, d a multiple of 64 up to 256): the shapes where the scores of Eq. 8 are a dense
-// contraction  -2 X W^T  of a 4096 x 256 mini-batch against a 1024 x 256 centre matrix.
-//
-// Split precision: x = x_hi + x_lo and -2w = w_hi + w_lo with every term a BF16 number (x_lo, w_lo hold the
-// rounding residues), and the score takes three products  x_hi.w_hi + x_lo.w_hi + x_hi.w_lo  into the same
-// accumulator.  What is left out (x_lo.w_lo and the residues of the residues) is below 6 * 2^-18 ||x|| ||w||, so
-// the scores are good to about 16 bits, the Eq. 8 decision falls to the exact fp32 comparison only for a fraction
-// of a percent of the rows, and every such row is decided among ALL centres that the bound cannot rule out.
+// Tensor-core path (tcgen05, 16-bit operands, FP32 accumulate in tensor memory) for states of up to 1024 centres with
+// d a multiple of 64 up to 256 and batches of at least 128 rows: the shapes where the scores of Eq. 8 are a dense
+// contraction  -2 X W^T, e.g. of a 4096 x 256 mini-batch against a 1024 x 256 centre matrix.
 //
 // Two operand formats (template parameter kTerms):
 //   1  FP16, one term per operand: x and -2w rounded to FP16 (11 significant bits), one product.  A score is good to
 //      2^-10 ||x|| ||w||; the rows whose candidates lie closer than that (a few per cent) are decided exactly afterwards.
 //      Needs |x|, |2w| inside FP16's range.
-//   3  BF16, two terms per operand, three products as above (about 16 bits): any fp32 range, three times the tensor work
-//      and twice the operand bytes.
+//   3  BF16, two terms per operand: x = x_hi + x_lo and -2w = w_hi + w_lo (x_lo, w_lo hold the rounding residues),
+//      three products  x_hi.w_hi + x_lo.w_hi + x_hi.w_lo  into the same accumulator.  What is left out (x_lo.w_lo and
+//      the residues of the residues) is below 6 * 2^-18 ||x|| ||w||: about 16 bits, any fp32 range, three times the
+//      tensor work and twice the operand bytes.
+// Either way Eq. 8 is decided exactly: a row is settled among ALL centres that the format's error bound cannot rule out.
 //
-// One worker = one thread block = one SM.  Warp roles while the scores are computed:
-//   warp 0   one lane issues the TMA loads: a 128-row sample tile (hi and lo) in 128-byte-swizzled K-chunks of 64,
-//            resident while all centre blocks pass, and 128-centre blocks of w_hi, w_lo through a ring of
-//            K-chunks (they come from L2);
-//   warp 1   allocates tensor memory; one lane issues tcgen05.mma (128 x 128 x 16 per instruction) into one
-//            of two 128-column accumulator stages and commits to mbarriers;
-//   warps 4-7  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread), add ||w_a||^2 and
-//            ||x||^2 and keep, per sample, the three smallest squared distances with the centre index packed
-//            into the low mantissa bits, carried in registers over the centre blocks.
+// A block serves its workers in turn (one worker when there are as many blocks as workers).  Warp roles while the
+// scores are computed:
+//   warp 0   one lane issues the TMA loads: a 128-row sample tile in 128-byte-swizzled K-chunks of 64, resident while
+//            all centre blocks pass, and the centre blocks (256 centres with one term, 128 with two, or the whole
+//            state rounded up to 32 when it is smaller) through a ring of K-chunks (they come from L2);
+//   warp 1   allocates tensor memory; one lane issues tcgen05.mma (128 x N x 16 per instruction) into one of two
+//            accumulator stages and commits to mbarriers;
+//   warps 4 and up  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread; one, two or three warps
+//            per quarter of the tile, taking the 32-column groups in turn), add ||w_a||^2 and ||x||^2 and keep, per
+//            sample, the three smallest squared distances with the centre index packed into the low mantissa bits,
+//            and a floor under the fourth, carried in registers over the centre blocks.
 // Then all warps: a sample whose runner-up is inside the error bound is decided between its two candidates with
-// fp32 inputs (fp64 sums when still close); one whose third candidate is inside the bound as well is decided
-// over all centres the same way.  Rows are grouped by centre and each centre's sum of fp32 master samples,
-// update, new w_hi, w_lo and ||w_a||^2 come from one pass.  Every wait is bounded.
+// fp32 inputs (fp64 sums when still close), likewise among three when the third is inside and the floor is not; one
+// whose fourth candidate may be inside as well is measured against all centres the same way.  Rows are grouped by
+// centre and each centre's sum of fp32 master samples, update, new 16-bit copy and ||w_a||^2 come from one pass.
+// Every wait is bounded.
 #pragma once
 
 #include <cuda.h>
