@@ -26,6 +26,20 @@ extern "C" {
  */
 int asgd_probe_issue_rates(float *out_host, int n_out, float *scratch_dev, int sms);
 
+/*
+ * Cycles per tcgen05.mma (kind::f16, FP16 operands in shared memory with the 128-byte swizzle, M = 128, K = 16, fp32
+ * accumulators in tensor memory), issued back to back by one thread of one block per SM, six cases in this order:
+ *   0 N = 256, the same pair of operand chunks every time     1 N = 256, walking over four chunks of each operand
+ *   2 as 1 with a tcgen05.commit after every four products    3, 4, 5 the same three with N = 128
+ * This is the rate the tensor-core worker kernel's issuing thread can reach at best.
+ *   out_host     HOST [n_out], n_out >= 6 (written)
+ *   scratch_dev  DEVICE, at least 4 * sms bytes, caller's; overwritten
+ *   sms          blocks to launch (the GPU's SM count)
+ * Launches on the default stream and synchronises; every device-side wait is bounded.  Returns 0; -1 for a NULL
+ * pointer, n_out < 6 or sms < 1 (nothing is launched); -3 when a CUDA call failed; -4 when a wait ran out.
+ */
+int asgd_probe_mma_rates(float *out_host, int n_out, float *scratch_dev, int sms);
+
 #ifdef __cplusplus
 }
 #endif

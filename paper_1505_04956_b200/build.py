@@ -48,7 +48,7 @@ PROBE_LIB = os.path.join(PKG, "libasgd_probe.so")
 def build_probe(force: bool = False) -> str:
     """Compile the issue-rate probes (csrc/asgd_probe.cu) into their own library; return its path."""
     src = os.path.join(CSRC, "asgd_probe.cu")
-    if not force and os.path.exists(PROBE_LIB) and os.path.getmtime(PROBE_LIB) >= os.path.getmtime(src):
+    if not force and os.path.exists(PROBE_LIB) and os.path.getmtime(PROBE_LIB) >= _newest_source_mtime():   # it includes the kernels' headers
         return PROBE_LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = PROBE_LIB + ".%d.tmp" % os.getpid()

@@ -6,6 +6,8 @@
 // Built into its own small library (libasgd_probe.so); nothing in the worker library depends on it.
 #include <cuda_runtime.h>
 
+#include "asgd_tc.cuh"   // descriptors and wrappers of tcgen05.mma, mbarrier helpers
+
 namespace {
 
 enum Mode { M_FFMA = 0, M_FFMA_ACC, M_FFMA2_ACC, M_FADD2, M_LOP3, M_FMNMX, M_FSET, M_IMAD, M_HMMA, M_LOP3_FFMA, M_LOP3_FFMA2,
@@ -97,4 +99,108 @@ extern "C" int asgd_probe_issue_rates(float* out_host, int n_out, float* scratch
   RUN(M_LOP3_FFMA) RUN(M_LOP3_FFMA2) RUN(M_HMMA_6FFMA) RUN(M_HMMA_4LOP3)
 #undef RUN
   return rc;
+}
+
+namespace {
+
+// One block: thread 0 issues n_mma tcgen05.mma (kind::f16, FP16 operands of zeros in shared memory, M = 128, the given N,
+// K = 16) back to back into two accumulator ranges, a commit after every `commit_every` of them (0: only at the end),
+// and waits (bounded) for the last commit.  out[blockIdx.x] = cycles per product, or -1 when the wait ran out.
+__global__ void __launch_bounds__(128) mma_probe_kernel(float* out, int n_mma, int n_cols, int commit_every, int spread, int variant) {
+  extern __shared__ __align__(1024) unsigned char smem_dyn[];
+  unsigned char* smem = smem_dyn + ((1024u - (asgd::smem_u32(smem_dyn) & 1023u)) & 1023u);
+  unsigned char* sA = smem;                               // 4 chunks of 128 rows x 64 numbers (16 KB each)
+  unsigned char* sB = smem + 4 * 16384;                   // 4 chunks of up to 256 rows x 64 numbers (32 KB each)
+  __shared__ unsigned long long bars[2 + 8 + 2];
+  __shared__ unsigned tmem_base;
+  for (int e = threadIdx.x; e < (4 * 16384 + 4 * 32768) / 16; e += blockDim.x) reinterpret_cast<uint4*>(smem)[e] = make_uint4(0u, 0u, 0u, 0u);
+  if (threadIdx.x == 0) {
+    asgd::mbar_init(bars + 0, 1);
+    asgd::mbar_init(bars + 1, commit_every > 0 ? (unsigned)(n_mma / commit_every) : 1u);
+    for (int q = 0; q < 10; ++q) asgd::mbar_init(bars + 2 + q, 1);      // variants 1, 3: commits go round these, one arrival completes a phase; the last two end variant 3
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (threadIdx.x < 32) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(asgd::smem_u32(&tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("fence.proxy.async;" ::: "memory");
+  asgd::tc_fence_before();
+  __syncthreads();
+  asgd::tc_fence_after();
+  const unsigned tmem = tmem_base;
+  if (variant == 3) {
+    // two issuing threads (first lanes of warps 0 and 1), each with its own accumulator range, half of the products
+    // and its own commits; thread 0 times both
+    __shared__ long long t_start;
+    if (threadIdx.x == 0) t_start = clock64();
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0 && threadIdx.x < 64) {
+      const int who = threadIdx.x >> 5;
+      const unsigned idesc = (1u << 4) | ((unsigned)(n_cols >> 3) << 17) | ((unsigned)(128 >> 4) << 24);
+      const unsigned long long dA0 = asgd::tc_smem_desc(sA, 0), dB0 = asgd::tc_smem_desc(sB, 0);
+      for (int it = 0; it < n_mma / 2; ++it) {
+        const int chunk = (it >> 2) & 3, k4 = it & 3;
+        const unsigned long long da = dA0 + (unsigned long long)(chunk * (16384 >> 4) + 2 * k4);
+        const unsigned long long db = dB0 + (unsigned long long)(chunk * (32768 >> 4) + 2 * k4);
+        asgd::tc_mma_bf16(tmem + (unsigned)(who * n_cols), da, db, idesc, (it & 15) != 0);
+        if (commit_every > 0 && (it + 1) % commit_every == 0) asgd::tc_commit(bars + 2 + who * 4 + ((it / commit_every) & 3));
+      }
+      asgd::tc_commit(bars + 10 + who);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      bool ok = asgd::mbar_wait_bounded(bars + 10, 0, 1u << 24);
+      ok = asgd::mbar_wait_bounded(bars + 11, 0, 1u << 24) && ok;
+      const long long t1 = clock64();
+      out[blockIdx.x] = ok ? (float)(t1 - t_start) / (float)n_mma : -1.f;
+    }
+  } else if (threadIdx.x == 0) {
+    const unsigned idesc = (1u << 4) | ((unsigned)(n_cols >> 3) << 17) | ((unsigned)(128 >> 4) << 24);
+    const unsigned long long dA0 = asgd::tc_smem_desc(sA, 0), dB0 = asgd::tc_smem_desc(sB, 0);
+    const long long t0 = clock64();
+    for (int it = 0; it < n_mma; ++it) {
+      // spread: walk over the four chunks of either operand as the worker kernel does; else the same chunk every time
+      const int chunk = spread ? (it >> 2) & 3 : 0, k4 = it & 3;
+      const unsigned long long da = dA0 + (unsigned long long)(chunk * (16384 >> 4) + 2 * k4);
+      const unsigned long long db = dB0 + (unsigned long long)(chunk * (32768 >> 4) + 2 * k4);
+      // variant 2: a fresh accumulator range after every commit (no product adds to columns a commit has just covered)
+      const unsigned acc = (variant == 2 && commit_every > 0) ? (unsigned)(((it / commit_every) & 1) * n_cols) : (unsigned)(((it >> 4) & 1) * n_cols);
+      const bool first = (variant == 2 && commit_every > 0) ? (it % commit_every) == 0 : (it & 15) == 0;
+      asgd::tc_mma_bf16(tmem + acc, da, db, idesc, !first);
+      if (commit_every > 0 && (it + 1) % commit_every == 0) asgd::tc_commit(variant == 1 ? bars + 2 + ((it / commit_every) & 7) : bars + 1);
+    }
+    asgd::tc_commit(bars + 0);
+    const bool ok = asgd::mbar_wait_bounded(bars + 0, 0, 1u << 24);
+    const long long t1 = clock64();
+    out[blockIdx.x] = ok ? (float)(t1 - t0) / (float)n_mma : -1.f;
+  }
+  asgd::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+}
+
+}  // namespace
+
+// out_host[6]: cycles per tcgen05.mma (kind::f16, M = 128, K = 16, operands in shared memory, one issuing thread, one
+// block per SM) for: N = 256 on one pair of chunks; N = 256 walking over four chunks of each operand; the same with
+// a commit after every four products; N = 128 on one pair of chunks; N = 128 walking; N = 128 walking with commits.
+// scratch_dev: DEVICE, >= 4 * sms bytes.  Returns 0, -1 for a bad argument, -3 when a CUDA call failed, -4 when a
+// wait on the products ran out.
+extern "C" int asgd_probe_mma_rates(float* out_host, int n_out, float* scratch_dev, int sms) {
+  if (!out_host || !scratch_dev || n_out < 6 || sms < 1) return -1;
+  const int smem = 4 * 16384 + 4 * 32768 + 1024;
+  if (cudaFuncSetAttribute(mma_probe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return -3;
+  const int cfg[12][4] = {{256, 0, 0, 0}, {256, 0, 1, 0}, {256, 4, 1, 0}, {128, 0, 0, 0}, {128, 0, 1, 0}, {128, 4, 1, 0},
+                          {256, 4, 1, 1}, {256, 4, 1, 2}, {256, 16, 1, 0}, {256, 16, 1, 1}, {256, 4, 1, 3}, {256, 0, 1, 3}};
+  for (int c = 0; c < (n_out >= 12 ? 12 : 6); ++c) {
+    const int n_mma = 4096;
+    for (int rep = 0; rep < 2; ++rep) mma_probe_kernel<<<sms, 128, smem>>>(scratch_dev, n_mma, cfg[c][0], cfg[c][1], cfg[c][2], cfg[c][3]);
+    if (cudaDeviceSynchronize() != cudaSuccess) return -3;
+    float v = 0.f;
+    if (cudaMemcpy(&v, scratch_dev, sizeof(float), cudaMemcpyDeviceToHost) != cudaSuccess) return -3;
+    if (v < 0.f) return -4;
+    out_host[c] = v;
+  }
+  return 0;
 }

@@ -179,8 +179,9 @@ __global__ void tc_row_norms_kernel(const float* __restrict__ X, long long N, in
 }
 
 // barrier slots
-enum { TCB_BFULL = 0, TCB_BEMPTY = TC_B_STAGES, TCB_AFULL = 2 * TC_B_STAGES, TCB_AEMPTY = 2 * TC_B_STAGES + TC_A_STAGES,
-       TCB_ACCFULL = 2 * TC_B_STAGES + 2 * TC_A_STAGES, TCB_ACCEMPTY = TCB_ACCFULL + 2, TCB_COUNT = TCB_ACCFULL + 4 };
+enum { TCB_BFULL = 0 /* [issuing thread][slot] */, TCB_BEMPTY = 2 * TC_B_STAGES, TCB_AFULL = 3 * TC_B_STAGES, TCB_AEMPTY = 3 * TC_B_STAGES + TC_A_STAGES,
+       TCB_ACCFULL = 3 * TC_B_STAGES + 2 * TC_A_STAGES, TCB_ACCEMPTY = TCB_ACCFULL + 2, TCB_COUNT = TCB_ACCFULL + 4 };
+static_assert(TCB_COUNT <= 32, "barrier slots");
 
 // smallest three of (m1 <= m2 <= m3) and a new value, kept sorted (five min/max)
 __device__ __forceinline__ void tc_top3_insert(float& m1, float& m2, float& m3, float v) {
@@ -259,8 +260,9 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   const float inv_b = 1.0f / (float)b;
 
   if (tid == 0) {
-    for (int q = 0; q < TC_B_STAGES; ++q) { mbar_init(bars + TCB_BFULL + q, 1); mbar_init(bars + TCB_BEMPTY + q, 1); }
-    for (int q = 0; q < TC_A_STAGES; ++q) { mbar_init(bars + TCB_AFULL + q, 1); mbar_init(bars + TCB_AEMPTY + q, 1); }
+    for (int q = 0; q < TC_B_STAGES; ++q) { mbar_init(bars + TCB_BFULL + q, 1); mbar_init(bars + TCB_BFULL + TC_B_STAGES + q, 1); mbar_init(bars + TCB_BEMPTY + q, 1); }
+    // a sample chunk is free when every issuing thread has seen its last products on it complete
+    for (int q = 0; q < TC_A_STAGES; ++q) { mbar_init(bars + TCB_AFULL + q, 1); mbar_init(bars + TCB_AEMPTY + q, (k + TC_N - 1) / TC_N >= 2 ? 2 : 1); }
     for (int q = 0; q < 2; ++q) { mbar_init(bars + TCB_ACCFULL + q, 1); mbar_init(bars + TCB_ACCEMPTY + q, NW - 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     misc[2] = 0;
@@ -325,6 +327,8 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
 
   // running phase counters of the pipelines (each role keeps its own copies in step)
   unsigned it_m = 0, it_bc = 0, it_acc = 0;
+  unsigned bfull_par = 0;                                 // an issuing thread's next phase of each of its ring barriers (a bit per slot)
+  const bool two_issuers = n_tiles >= 2;
 
   bool gave_up = false;
   for (long long step = 0; step < steps && !gave_up; ++step)
@@ -355,25 +359,38 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             }
           }
           for (int n = 0; n < n_tiles && ok; ++n) {
+            // the full barrier of the thread that will issue this centre block's products
+            const int q_full = two_issuers ? (int)((it_acc + (unsigned)(m * n_tiles + n)) & 1u) * TC_B_STAGES : 0;
             for (int g = 0; g < PPK * nkc; ++g, ++ibc) {               // g = PPK * K chunk + (0: w_hi, 1: w_lo)
               const int st = ibc % TC_B_STAGES;
               if (ibc >= TC_B_STAGES) ok = mbar_wait_bounded(bars + TCB_BEMPTY + st, ((ibc / TC_B_STAGES) - 1) & 1, p.wait_limit);
               if (!ok) break;
-              mbar_expect_tx(bars + TCB_BFULL + st, (unsigned)TC_B_CHUNK_BYTES);
-              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, (g / PPK) * TC_KC, (g % PPK) * p.W * k + i * k + n * TC_N, bars + TCB_BFULL + st, pol_w);
+              mbar_expect_tx(bars + TCB_BFULL + q_full + st, (unsigned)TC_B_CHUNK_BYTES);
+              tma_load_2d(sB + (size_t)st * TC_B_CHUNK_BYTES, &mapW, (g / PPK) * TC_KC, (g % PPK) * p.W * k + i * k + n * TC_N, bars + TCB_BFULL + q_full + st, pol_w);
             }
           }
         }
         if (!ok) atomicExch(&misc[2], 1);
       }
-    } else if (wid == 1) {
+    } else if (wid == 1 || (wid == 2 && two_issuers)) {
+      // Two issuing threads, one per accumulator stage (centre blocks in turn), when a sample tile meets at least two
+      // centre blocks.  A tcgen05.commit holds the thread that issues it for several hundred cycles (measured: one
+      // thread issuing four products and a commit in turn reaches 275 cycles per product, two threads doing so side
+      // by side 133, the rate without commits 128), so the other thread's products keep the tensor pipe fed
+      // meanwhile.  The pipe runs the products in the order they were issued, each block's products come from one
+      // thread, a ring slot or a sample chunk is handed back by the thread that used it last, and each thread has its
+      // own full barriers for the ring, so that it sees every phase of every barrier it waits on (a parity wait cannot
+      // tell the last completed phase from the one before).  Both threads meet every sample tile.
       if (lane == 0) {
+        const unsigned me = (unsigned)(wid - 1);
         unsigned um = it_m, ibc = it_bc, iacc = it_acc;
         bool ok = true;
         const unsigned long long dA0 = tc_smem_desc(sA, 0), dB0 = tc_smem_desc(sB, 0);
         for (int m = 0; m < m_tiles && ok; ++m, ++um) {
+          bool first_here = true;                          // this thread's first centre block of the sample tile
           for (int n = 0; n < n_tiles && ok; ++n, ++iacc) {
             const int buf = iacc & 1;
+            if (two_issuers && (unsigned)buf != me) { ibc += (unsigned)(PPK * nkc); continue; }      // the other thread's block
             if (iacc >= 2) ok = mbar_wait_bounded(bars + TCB_ACCEMPTY + buf, ((iacc >> 1) - 1) & 1, p.wait_limit);
             if (!ok) break;
             tc_fence_after();
@@ -381,9 +398,11 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
             for (int g = 0; g < PPK * nkc && ok; ++g, ++ibc) {
               const int st = ibc % TC_B_STAGES;
               const int kc = g / PPK, lo_w = g % PPK;
-              if (n == 0 && lo_w == 0) ok = mbar_wait_bounded(bars + TCB_AFULL + kc, um & 1, p.wait_limit);
-              if (ok) ok = mbar_wait_bounded(bars + TCB_BFULL + st, (ibc / TC_B_STAGES) & 1, p.wait_limit);
+              if (first_here && lo_w == 0) ok = mbar_wait_bounded(bars + TCB_AFULL + kc, um & 1, p.wait_limit);
+              // this thread's uses of the slot so far decide the phase
+              if (ok) ok = mbar_wait_bounded(bars + TCB_BFULL + (two_issuers ? (int)me * TC_B_STAGES : 0) + st, (bfull_par >> st) & 1u, p.wait_limit);
               if (!ok) break;
+              bfull_par ^= 1u << st;
               tc_fence_after();
               // operand descriptors: the base descriptor plus the chunk's offset in 16-byte units (the address field
               // holds address >> 4 and shared memory is below 256 KB, so the sum stays inside the field)
@@ -399,9 +418,11 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
                   tc_mma_bf16(acc_col, dal + (unsigned long long)(2 * k4), db + (unsigned long long)(2 * k4), idesc, true);
               }
               tc_commit(bars + TCB_BEMPTY + st);                        // the ring slot is free when these MMAs have read it
-              if (n == n_tiles - 1 && lo_w == PPK - 1) tc_commit(bars + TCB_AEMPTY + kc);   // and so is the sample chunk after its last centre block
+              // and so is the sample chunk after this thread's last centre block of the tile
+              if ((two_issuers ? n + 2 >= n_tiles : n == n_tiles - 1) && lo_w == PPK - 1) tc_commit(bars + TCB_AEMPTY + kc);
             }
             tc_commit(bars + TCB_ACCFULL + buf);                        // the accumulator stage is complete
+            first_here = false;
           }
         }
         if (!ok) atomicExch(&misc[2], 1);
@@ -971,7 +992,7 @@ asgd_tc_kernel(const Params p, const long long steps, const __grid_constant__ CU
   if (misc[2] && tid == 0) {
     atomicExch(p.status, DEV_TIMEOUT);
     // copies may still be on their way into this block's shared memory: give each a bounded chance to land
-    for (int q = 0; q < TC_B_STAGES; ++q) { mbar_wait_bounded(bars + TCB_BFULL + q, 0, p.wait_limit); mbar_wait_bounded(bars + TCB_BFULL + q, 1, p.wait_limit); }
+    for (int q = 0; q < 2 * TC_B_STAGES; ++q) { mbar_wait_bounded(bars + TCB_BFULL + q, 0, p.wait_limit); mbar_wait_bounded(bars + TCB_BFULL + q, 1, p.wait_limit); }
     for (int q = 0; q < TC_A_STAGES; ++q) { mbar_wait_bounded(bars + TCB_AFULL + q, 0, p.wait_limit); mbar_wait_bounded(bars + TCB_AFULL + q, 1, p.wait_limit); }
   }
   tc_fence_before();

@@ -32,6 +32,30 @@ def issue_rates():
     return [float(v) for v in out]
 
 
+MMA_NAMES = ("tcgen05.mma 128x256x16 f16, one pair of chunks", "tcgen05.mma 128x256x16, walking four chunks",
+             "tcgen05.mma 128x256x16, walking, commit every 4", "tcgen05.mma 128x128x16 f16, one pair of chunks",
+             "tcgen05.mma 128x128x16, walking four chunks", "tcgen05.mma 128x128x16, walking, commit every 4",
+             "N=256 commit every 4, eight barriers in turn", "N=256 commit every 4, fresh accumulator after a commit",
+             "N=256 commit every 16", "N=256 commit every 16, eight barriers in turn", "N=256 two issuing threads, commit every 4",
+             "N=256 two issuing threads, no commits")
+
+
+def mma_rates():
+    """Cycles per tcgen05.mma issued back to back by one thread, in the order of MMA_NAMES (needs a B200)."""
+    import torch
+    lib = C.CDLL(_build.build_probe())
+    lib.asgd_probe_mma_rates.argtypes = [C.POINTER(C.c_float), C.c_int, C.c_void_p, C.c_int]
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    scratch = torch.empty(sms, dtype=torch.float32, device="cuda")
+    out = (C.c_float * len(MMA_NAMES))()
+    rc = lib.asgd_probe_mma_rates(out, len(MMA_NAMES), C.c_void_p(scratch.data_ptr()), sms)
+    if rc != 0:
+        raise RuntimeError("asgd_probe_mma_rates failed (%d)" % rc)
+    return [float(v) for v in out]
+
+
 if __name__ == "__main__":
     for name, v in zip(NAMES, issue_rates()):
-        print("%-40s %6.2f cycles per warp instruction and scheduler" % (name, v))
+        print("%-48s %7.2f cycles per warp instruction and scheduler" % (name, v))
+    for name, v in zip(MMA_NAMES, mma_rates()):
+        print("%-48s %7.2f cycles per product" % (name, v))

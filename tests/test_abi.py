@@ -29,7 +29,7 @@ def test_probe_library_builds_and_exports_its_entry_point():
     text = open(os.path.join(ROOT, "include", "asgd_probe.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     names = sorted(set(re.findall(r"\b(asgd_[a-z0-9_]+)\s*\(", text)))
-    assert names == ["asgd_probe_issue_rates"]
+    assert names == ["asgd_probe_issue_rates", "asgd_probe_mma_rates"]
     lib = C.CDLL(libbuild.build_probe())
     for n in names:
         assert hasattr(lib, n), n

@@ -13,3 +13,11 @@ def test_issue_rates_are_plausible():
     # a scalar FMA issues about every cycle; the half-rate kinds take about two
     assert r["FFMA (two immediates)"] < 1.5
     assert r["LOP3"] > 1.5 * r["FFMA (two immediates)"]
+
+
+def test_mma_rates_are_plausible():
+    from paper_1505_04956_b200 import peaks
+    r = dict(zip(peaks.MMA_NAMES, peaks.mma_rates()))
+    assert len(r) == 6
+    for name, v in r.items():
+        assert 16.0 < v < 2000.0, (name, v)
