@@ -18,7 +18,8 @@
 //            all centre blocks pass, and the centre blocks (256 centres with one term, 128 with two, or the whole
 //            state rounded up to 32 when it is smaller) through a ring of K-chunks (they come from L2);
 //   warp 1   allocates tensor memory; one lane issues tcgen05.mma (128 x N x 16 per instruction) into one of two
-//            accumulator stages and commits to mbarriers;
+//            accumulator stages and commits to mbarriers; with two or more centre blocks one lane of warp 2 does the
+//            same for every other block (a commit holds its thread for a while; the other thread keeps the pipe fed);
 //   warps 4 and up  read the accumulators (tcgen05.ld, one TMEM lane = one sample per thread; one, two or three warps
 //            per quarter of the tile, taking the 32-column groups in turn), add ||w_a||^2 and ||x||^2 and keep, per
 //            sample, the three smallest squared distances with the centre index packed into the low mantissa bits,
