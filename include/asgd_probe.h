@@ -28,11 +28,17 @@ int asgd_probe_issue_rates(float *out_host, int n_out, float *scratch_dev, int s
 
 /*
  * Cycles per tcgen05.mma (kind::f16, FP16 operands in shared memory with the 128-byte swizzle, M = 128, K = 16, fp32
- * accumulators in tensor memory), issued back to back by one thread of one block per SM, six cases in this order:
+ * accumulators in tensor memory), issued back to back by one thread of one block per SM (two threads in the last two
+ * cases), twelve cases in this order:
  *   0 N = 256, the same pair of operand chunks every time     1 N = 256, walking over four chunks of each operand
  *   2 as 1 with a tcgen05.commit after every four products    3, 4, 5 the same three with N = 128
- * This is the rate the tensor-core worker kernel's issuing thread can reach at best.
- *   out_host     HOST [n_out], n_out >= 6 (written)
+ *   6 as 2 with the commits going round eight barriers        7 as 2 with a fresh accumulator range after every commit
+ *   8 as 1 with a commit after every 16 products              9 as 8 with the commits going round eight barriers
+ *  10 two issuing threads (first lanes of two warps), each with its own accumulator range: four products and a
+ *     commit in turn                                          11 the same without commits
+ * These are the rates the tensor-core worker kernel's issuing threads can reach at best; cases 2 and 10 are why it
+ * has two of them.
+ *   out_host     HOST [n_out]; n_out >= 12: all cases, 6 <= n_out < 12: the first six (written)
  *   scratch_dev  DEVICE, at least 4 * sms bytes, caller's; overwritten
  *   sms          blocks to launch (the GPU's SM count)
  * Launches on the default stream and synchronises; every device-side wait is bounded.  Returns 0; -1 for a NULL

@@ -182,11 +182,13 @@ __global__ void __launch_bounds__(128) mma_probe_kernel(float* out, int n_mma, i
 
 }  // namespace
 
-// out_host[6]: cycles per tcgen05.mma (kind::f16, M = 128, K = 16, operands in shared memory, one issuing thread, one
-// block per SM) for: N = 256 on one pair of chunks; N = 256 walking over four chunks of each operand; the same with
-// a commit after every four products; N = 128 on one pair of chunks; N = 128 walking; N = 128 walking with commits.
-// scratch_dev: DEVICE, >= 4 * sms bytes.  Returns 0, -1 for a bad argument, -3 when a CUDA call failed, -4 when a
-// wait on the products ran out.
+// out_host[12] (the first six with 6 <= n_out < 12): cycles per tcgen05.mma (kind::f16, M = 128, K = 16, operands in
+// shared memory, one block per SM) for: N = 256 on one pair of chunks; N = 256 walking over four chunks of each operand;
+// the same with a commit after every four products; the same three with N = 128; N = 256 with a commit after every
+// four, the commits going round eight barriers; with a fresh accumulator range after every commit; with a commit after
+// every 16; the same on eight barriers; two issuing threads, four products and a commit in turn each; two issuing
+// threads without commits.  scratch_dev: DEVICE, >= 4 * sms bytes.  Returns 0, -1 for a bad argument, -3 when a CUDA
+// call failed, -4 when a wait on the products ran out.
 extern "C" int asgd_probe_mma_rates(float* out_host, int n_out, float* scratch_dev, int sms) {
   if (!out_host || !scratch_dev || n_out < 6 || sms < 1) return -1;
   const int smem = 4 * 16384 + 4 * 32768 + 1024;
