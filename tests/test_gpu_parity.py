@@ -335,6 +335,44 @@ def test_free_running_mode_reaches_the_oracles_error():
     pr.close()
 
 
+# One persistent launch of several steps with no messages (c = 0) is deterministic: a worker's states after it are
+# those of the oracle's synchronous rounds.  The shapes take every worker kernel and every instance of the
+# tensor-core one through what only a multi-step launch exercises: pipeline phases that run on from step to step, the
+# two product-issuing threads with odd numbers of centre blocks and of sample tiles, three K chunks in a four-slot ring,
+# the two-term format, workers that share a block in turn, two blocks on an SM.
+SILENT_LAUNCHES = {
+    "stream": (dict(N=4 * 100 * 4 + 3, d=10, k=10, W=4, b=100), pkg.PATH_AUTO, "fp32-stream"),
+    "tiled_d32": (dict(N=5 * 100 * 3 + 1, d=32, k=37, W=5, b=100), pkg.PATH_AUTO, "fp32-tiled"),
+    "tc_512_threads_three_blocks": (dict(N=2 * 300 * 3 + 5, d=128, k=600, W=2, b=300), pkg.PATH_AUTO, "tcgen05-fp16"),
+    "tc_512_threads_one_chunk": (dict(N=2 * 256 * 3, d=64, k=520, W=2, b=256), pkg.PATH_AUTO, "tcgen05-fp16"),
+    "tc_384_threads_three_chunks": (dict(N=2 * 300 * 3 + 5, d=192, k=600, W=2, b=300), pkg.PATH_AUTO, "tcgen05-fp16"),
+    "tc_384_threads_d256": (dict(N=2 * 384 * 2 + 1, d=256, k=700, W=2, b=384), pkg.PATH_AUTO, "tcgen05-fp16"),
+    "tc_two_terms_three_blocks": (dict(N=2 * 200 * 3, d=256, k=300, W=2, b=200), pkg.PATH_TC_BF16, "tcgen05-bf16x3"),
+    "tc_two_terms_d128": (dict(N=3 * 200 * 3, d=128, k=300, W=3, b=200), pkg.PATH_TC_BF16, "tcgen05-bf16x3"),
+    "tc_two_blocks_per_sm_workers_in_turn": (dict(N=310 * 128 * 2, d=128, k=100, W=310, b=128), pkg.PATH_AUTO, "tcgen05-fp16"),
+    "general": (dict(N=3 * 50 * 4 + 2, d=9, k=7, W=3, b=50), pkg.PATH_AUTO, "fp32-generic"),
+}
+
+
+@pytest.mark.parametrize("case", list(SILENT_LAUNCHES))
+def test_silent_multi_step_launch_equals_the_oracles_rounds(case):
+    over, path, want = SILENT_LAUNCHES[case]
+    wl = scaled("tiny", eps=0.1, comm_interval=0, fanout=1, **over)
+    pr = Pair(wl, dist_path=path, record_assign=0)
+    assert pr.gpu.path_name() == want, (case, pr.gpu.path_name())
+    steps = 2 * wl.B + 3
+    pr.gpu.run(steps)
+    pr.gpu.sync()
+    pr.cpu.rounds(steps)
+    assert pr.max_rel_l2() < pr.centre_tol(), (case, pr.max_rel_l2())
+    assert all(pr.gpu.get_stats(i)["steps"] == steps for i in range(wl.W))
+    pr.gpu.run(2)                                         # a second launch picks the counters up where the first left them
+    pr.gpu.sync()
+    pr.cpu.rounds(2)
+    assert pr.max_rel_l2() < pr.centre_tol(), (case, pr.max_rel_l2())
+    pr.close()
+
+
 def test_mixing_deterministic_rounds_and_free_running():
     wl = scaled("tiny", N=20_000)
     pr = Pair(wl, record_assign=0)
